@@ -1,0 +1,176 @@
+"""CPU fp64 oracle for standard attention -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes front end of ``attention_oracle.c`` (plain C, compiled with gcc on
+first use).  It states the paper's definition of standard attention (Section
+5.1), its lower-triangular mask (Section 4.1) and the decode-stage form
+(Appendix C) and is what the CUDA library is compared against.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the product never does, and this package never imports the
+product.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "attention_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lock = threading.Lock()
+_lib = None
+
+_DTYPE_CODE = {torch.float16: 0, torch.bfloat16: 1, torch.float32: 2, torch.float64: 3}
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle into ``liboracle.so`` next to its source."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = _LIB + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+               "-ffp-contract=off", _SRC, "-o", tmp, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            lib = ctypes.CDLL(_LIB)
+            i32, f64, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+            lib.oracle_attention_full.restype = i32
+            lib.oracle_attention_full.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                                  i32, f64, vp, vp, vp, i32]
+            lib.oracle_attention_rows.restype = i32
+            lib.oracle_attention_rows.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                                  i32, f64, vp, vp, i32, vp, vp, i32]
+            lib.oracle_decode.restype = i32
+            lib.oracle_decode.argtypes = [vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, f64, vp,
+                                          vp, vp, i32]
+            lib.oracle_bruteforce.restype = i32
+            lib.oracle_bruteforce.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f64,
+                                              vp, vp]
+            lib.oracle_num_threads.restype = i32
+            _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the oracle's parallel loops use by default (OpenMP's count)."""
+    return int(_load().oracle_num_threads())
+
+
+def _as_cpu(t) -> torch.Tensor:
+    if isinstance(t, np.ndarray):
+        t = torch.from_numpy(t)
+    if t.device.type != "cpu":
+        raise ValueError("the oracle takes host tensors only")
+    if t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError("expected a [B, S, H, d] tensor with contiguous d")
+    return t
+
+
+def _strides9(q, k, v):
+    s = [q.stride(0), q.stride(1), q.stride(2), k.stride(0), k.stride(1), k.stride(2),
+         v.stride(0), v.stride(1), v.stride(2)]
+    return np.asarray(s, dtype=np.int64)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with code {rc}")
+
+
+def _common(q, k, v):
+    q, k, v = _as_cpu(q), _as_cpu(k), _as_cpu(v)
+    if not (q.dtype == k.dtype == v.dtype) or q.dtype not in _DTYPE_CODE:
+        raise ValueError("q, k, v must share one of fp16 / bf16 / fp32 / fp64")
+    B, Sq, Hq, d = q.shape
+    Bk, Skv, Hkv, dk = k.shape
+    if Bk != B or dk != d or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("shape mismatch between q, k, v")
+    return q, k, v, B, Sq, Hq, Skv, Hkv, d
+
+
+def attention_full(q, k, v, causal: bool, scale: float, nthreads: int = 0):
+    """Standard attention on the whole problem.
+
+    q ``[B,Sq,Hq,d]``, k and v ``[B,Skv,Hkv,d]`` host tensors.  Returns
+    ``(O [B,Sq,Hq,d], LSE [B,Hq,Sq])`` as float64 tensors.
+    """
+    q, k, v, B, Sq, Hq, Skv, Hkv, d = _common(q, k, v)
+    O = torch.zeros(B, Sq, Hq, d, dtype=torch.float64)
+    LSE = torch.zeros(B, Hq, Sq, dtype=torch.float64)
+    st = _strides9(q, k, v)
+    rc = _load().oracle_attention_full(q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                       _DTYPE_CODE[q.dtype], B, Hq, Hkv, Sq, Skv, d,
+                                       int(bool(causal)), float(scale), st.ctypes.data,
+                                       O.data_ptr(), LSE.data_ptr(), int(nthreads))
+    _check(rc, "oracle_attention_full")
+    return O, LSE
+
+
+def attention_rows(q, k, v, causal: bool, scale: float, rows, nthreads: int = 0):
+    """Standard attention for chosen rows only.
+
+    ``rows`` is an ``[n,3]`` integer array of (b, h, i).  Returns
+    ``(O [n,d], LSE [n])`` as float64 tensors.
+    """
+    q, k, v, B, Sq, Hq, Skv, Hkv, d = _common(q, k, v)
+    rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int32).reshape(-1, 3))
+    n = rows.shape[0]
+    O = torch.zeros(n, d, dtype=torch.float64)
+    LSE = torch.zeros(n, dtype=torch.float64)
+    st = _strides9(q, k, v)
+    rc = _load().oracle_attention_rows(q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                       _DTYPE_CODE[q.dtype], B, Hq, Hkv, Sq, Skv, d,
+                                       int(bool(causal)), float(scale), st.ctypes.data,
+                                       rows.ctypes.data, n, O.data_ptr(), LSE.data_ptr(),
+                                       int(nthreads))
+    _check(rc, "oracle_attention_rows")
+    return O, LSE
+
+
+def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
+    """Decode-stage attention: q ``[B,1,Hq,d]`` over the first ``seqlens[b]`` rows of
+    the ``[B,Smax,Hkv,d]`` caches.  Returns ``(O [B,Hq,d], LSE [B,Hq])`` float64."""
+    q, k, v, B, Sq, Hq, Smax, Hkv, d = _common(q, k_cache, v_cache)
+    if Sq != 1:
+        raise ValueError("decode takes one query row per sequence")
+    sl = np.ascontiguousarray(np.asarray(seqlens, dtype=np.int32).reshape(-1))
+    if sl.shape[0] != B:
+        raise ValueError("seqlens must have B entries")
+    O = torch.zeros(B, Hq, d, dtype=torch.float64)
+    LSE = torch.zeros(B, Hq, dtype=torch.float64)
+    st = _strides9(q, k, v)
+    rc = _load().oracle_decode(q.data_ptr(), k.data_ptr(), v.data_ptr(), _DTYPE_CODE[q.dtype],
+                               sl.ctypes.data, B, Hq, Hkv, Smax, d, float(scale),
+                               st.ctypes.data, O.data_ptr(), LSE.data_ptr(), int(nthreads))
+    _check(rc, "oracle_decode")
+    return O, LSE
+
+
+def bruteforce(q, k, v, causal: bool, scale: float):
+    """Extended-precision direct evaluation for tiny inputs (d <= 64): exp(s)/sum exp(s)
+    with no max subtraction.  Inputs are converted to contiguous float64."""
+    q = torch.as_tensor(q).to(torch.float64).contiguous()
+    k = torch.as_tensor(k).to(torch.float64).contiguous()
+    v = torch.as_tensor(v).to(torch.float64).contiguous()
+    B, Sq, Hq, d = q.shape
+    _, Skv, Hkv, _ = k.shape
+    O = torch.zeros(B, Sq, Hq, d, dtype=torch.float64)
+    LSE = torch.zeros(B, Hq, Sq, dtype=torch.float64)
+    rc = _load().oracle_bruteforce(q.data_ptr(), k.data_ptr(), v.data_ptr(), B, Hq, Hkv, Sq,
+                                   Skv, d, int(bool(causal)), float(scale), O.data_ptr(),
+                                   LSE.data_ptr())
+    _check(rc, "oracle_bruteforce")
+    return O, LSE

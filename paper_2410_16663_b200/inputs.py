@@ -1,0 +1,160 @@
+"""Seeded synthetic inputs for the attention workloads.
+
+This module only draws random numbers and shapes them; it contains none of the
+attention arithmetic, so both the CUDA tests and the CPU oracle can be fed from
+it.  Values are N(0,1) rounded to the storage type, the distribution the
+benchmark configurations name; sequence lengths for decode are uniform integers
+in a closed range.  Small problems are drawn on the host (identical bits on any
+machine); problems too large for that are drawn on the device with torch's
+seeded generator and the rows the oracle needs are copied back by the caller.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import torch
+
+FP16_NAN_BITS = 0x7E00  # quiet NaN in binary16, used to poison cache padding
+BF16_NAN_BITS = 0x7FC0
+
+
+@dataclass(frozen=True)
+class PrefillConfig:
+    name: str
+    B: int
+    Hq: int
+    Hkv: int
+    Sq: int
+    Skv: int
+    d: int = 128
+    dtype: str = "fp16"
+    causal: bool = True
+    seed: int = 0
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.d)
+
+    @property
+    def torch_dtype(self):
+        return torch.float16 if self.dtype == "fp16" else torch.bfloat16
+
+    def flops(self) -> float:
+        """Credited FLOPs: 4*B*Hq*Sq*Skv*d, halved when causal (the masked half is not credited)."""
+        f = 4.0 * self.B * self.Hq * self.Sq * self.Skv * self.d
+        return f / 2 if self.causal else f
+
+
+@dataclass(frozen=True)
+class DecodeConfig:
+    name: str
+    B: int
+    Hq: int
+    Hkv: int
+    Smax: int
+    len_lo: int
+    len_hi: int
+    d: int = 128
+    dtype: str = "fp16"
+    seed: int = 0
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.d)
+
+
+# The five benchmark configurations (C1..C5) with fixed seeds.
+C1 = PrefillConfig("C1", 1, 2, 2, 512, 512, dtype="fp16", causal=True, seed=1001)
+C2 = PrefillConfig("C2", 4, 32, 32, 2048, 2048, dtype="fp16", causal=True, seed=1002)
+C3 = {s: PrefillConfig(f"C3-{s // 1024}K", 1, 32, 32, s, s, dtype="bf16", causal=True,
+                       seed=1003 + i)
+      for i, s in enumerate((8192, 32768, 131072, 262144))}
+C4 = PrefillConfig("C4", 2, 64, 8, 8192, 8192, dtype="bf16", causal=True, seed=1010)
+C4_NC = PrefillConfig("C4-noncausal", 2, 64, 8, 1024, 8192, dtype="bf16", causal=False, seed=1011)
+C5_MHA = DecodeConfig("C5-mha", 64, 32, 32, 32768, 1024, 32768, seed=1020)
+C5_GQA = DecodeConfig("C5-gqa", 64, 32, 8, 32768, 1024, 32768, seed=1021)
+
+
+def _gen(seed: int, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def _randn(shape, dtype, gen, device) -> torch.Tensor:
+    """N(0,1) in fp32 rounded to ``dtype``, drawn in slabs along dim 0/1 to bound temporaries."""
+    out = torch.empty(shape, dtype=dtype, device=device)
+    flat = out.view(-1)
+    n = flat.numel()
+    step = 1 << 26
+    for s in range(0, n, step):
+        e = min(n, s + step)
+        flat[s:e] = torch.randn(e - s, dtype=torch.float32, device=device, generator=gen).to(dtype)
+    return out
+
+
+def prefill_inputs(cfg: PrefillConfig, device="cpu"):
+    """q [B,Sq,Hq,d], k and v [B,Skv,Hkv,d] for a prefill configuration."""
+    device = torch.device(device)
+    gen = _gen(cfg.seed, device)
+    dt = cfg.torch_dtype
+    q = _randn((cfg.B, cfg.Sq, cfg.Hq, cfg.d), dt, gen, device)
+    k = _randn((cfg.B, cfg.Skv, cfg.Hkv, cfg.d), dt, gen, device)
+    v = _randn((cfg.B, cfg.Skv, cfg.Hkv, cfg.d), dt, gen, device)
+    return q, k, v
+
+
+def decode_seqlens(cfg: DecodeConfig) -> torch.Tensor:
+    """Per-sequence cache lengths, uniform integers in [len_lo, len_hi], drawn on the host."""
+    gen = _gen(cfg.seed + 7, "cpu")
+    return torch.randint(cfg.len_lo, cfg.len_hi + 1, (cfg.B,), generator=gen, dtype=torch.int32)
+
+
+def decode_inputs(cfg: DecodeConfig, device="cpu", poison: bool = True):
+    """q [B,1,Hq,d], k_cache and v_cache [B,Smax,Hkv,d], seqlens [B] (int32, host).
+
+    Cache rows at or beyond ``seqlens[b]`` hold NaN bit patterns when ``poison`` is set, so a
+    kernel that lets padding reach its result is caught.
+    """
+    device = torch.device(device)
+    gen = _gen(cfg.seed, device)
+    dt = torch.float16 if cfg.dtype == "fp16" else torch.bfloat16
+    seqlens = decode_seqlens(cfg)
+    q = _randn((cfg.B, 1, cfg.Hq, cfg.d), dt, gen, device)
+    k = _randn((cfg.B, cfg.Smax, cfg.Hkv, cfg.d), dt, gen, device)
+    v = _randn((cfg.B, cfg.Smax, cfg.Hkv, cfg.d), dt, gen, device)
+    if poison:
+        bits = FP16_NAN_BITS if dt == torch.float16 else BF16_NAN_BITS
+        for b in range(cfg.B):
+            n = int(seqlens[b])
+            if n < cfg.Smax:
+                k[b, n:].view(torch.int16).fill_(bits)
+                v[b, n:].view(torch.int16).fill_(bits)
+    return q, k, v, seqlens
+
+
+def sample_rows(cfg: PrefillConfig, n_random: int, seed: int, pairs=None, tile: int = 128):
+    """Rows (b, h, i) for row-sampled checks: the first four and the last row, both sides of
+    tile boundaries near the start, middle and end, and uniformly random rows, over a few
+    (b, h) pairs that include both ends of a GQA group."""
+    gen = _gen(seed, "cpu")
+    if pairs is None:
+        g = cfg.Hq // cfg.Hkv
+        pairs = {(0, 0), (0, g - 1), (cfg.B - 1, cfg.Hq - 1), (cfg.B - 1, cfg.Hq - g),
+                 (0, cfg.Hq // 2)}
+        pairs = sorted(pairs)
+    fixed = {0, 1, 2, 3, cfg.Sq - 1}
+    ntile = (cfg.Sq + tile - 1) // tile
+    for t in {1, 2, ntile // 2, ntile - 1}:
+        for dlt in (-1, 0):
+            i = t * tile + dlt
+            if 0 <= i < cfg.Sq:
+                fixed.add(i)
+    rows = []
+    for (b, h) in pairs:
+        mine = set(fixed)
+        if n_random > 0:
+            mine.update(int(x) for x in torch.randint(0, cfg.Sq, (n_random,), generator=gen))
+        rows.extend((b, h, i) for i in sorted(mine))
+    return rows
