@@ -1,0 +1,145 @@
+/*
+ * fa.h -- C ABI of the B200 (sm_100a) fused attention forward library.
+ *
+ * The library computes, for every batch b, query head h and query row i,
+ *
+ *     O[b,i,h,:] = sum_j softmax_j( scale * <Q[b,i,h,:], K[b,j,hk,:]> + mask(i,j) ) * V[b,j,hk,:]
+ *     LSE[b,h,i] = ln sum_j exp( scale * <Q[b,i,h,:], K[b,j,hk,:]> + mask(i,j) )
+ *
+ * i.e. the paper's attention operator Softmax(Q K^T / sqrt(d)) V (Section 5.1), evaluated
+ * with the FlashAttention2-style fused, blocked, online-softmax method the paper builds on
+ * (Section 4.1; Appendix A: per block Q*K^T, Exp, Exp*V, update of rowmax/rowsum), so that
+ * neither the score matrix nor the attention_mask is ever stored (Section 4.1, tiling-mask:
+ * the mask is lower triangular; fully masked blocks are skipped, fully visible blocks are
+ * not masked).  The decode entry point evaluates the decode-stage form of Appendix C
+ * (one query row per sequence over the cached keys and values).
+ *
+ * Conventions shared by every entry point
+ *   - All q/k/v/o/lse/seqlens/workspace pointers are DEVICE pointers owned by the caller,
+ *     unless an argument is explicitly named *_host.  The library never allocates or frees
+ *     device memory and never keeps a pointer after the call returns.
+ *   - Layout: q and o are [B, Sq, Hq, d], k and v are [B, Skv, Hkv, d], d contiguous
+ *     (the paper's B*S*N*D layout, Section 4.2).  lse is [B, Hq, Sq] float, natural log.
+ *   - Head mapping: query head h reads kv head h / (Hq / Hkv); Hq % Hkv must be 0.
+ *   - causal != 0 applies the lower-triangular mask aligned to the last key:
+ *     row i sees key j iff j <= i + (Skv - Sq).
+ *   - scale is used as given (callers pass 1/sqrt(d)).
+ *   - stream is a cudaStream_t passed as void*.  Calls only enqueue work on it; they do
+ *     not synchronise.  Two calls that write the same buffers must be ordered by the caller.
+ *   - Return value: FA_OK or a negative FA_ERR_* code.  Arguments are validated before any
+ *     CUDA call; on a validation error nothing has been enqueued.  No entry point throws,
+ *     aborts or traps.
+ *   - Device-side waits are bounded.  If one ever expires the kernel records it in a status
+ *     word, drains and returns; fa_device_status() reports it after the stream is idle.
+ */
+#ifndef FA_H_
+#define FA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FA_OK 0
+#define FA_ERR_NULL (-1)        /* a required pointer is NULL                                 */
+#define FA_ERR_SHAPE (-2)       /* negative dims, Hq % Hkv != 0, bad stride                  */
+#define FA_ERR_UNSUPPORTED (-3) /* d != 128, causal with Sq > Skv, unknown dtype             */
+#define FA_ERR_ALIGN (-4)       /* a pointer or stride is not 16-byte aligned                */
+#define FA_ERR_WORKSPACE (-5)   /* workspace missing or too small                            */
+#define FA_ERR_DEVICE (-6)      /* current device is not compute capability 10.x             */
+#define FA_ERR_CUDA (-7)        /* a CUDA call failed; see fa_last_cuda_error()              */
+#define FA_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired (fa_device_status)     */
+
+#define FA_DTYPE_FP16 0
+#define FA_DTYPE_BF16 1
+#define FA_DTYPE_FP32 2 /* only as fa_params.o_dtype */
+
+/*
+ * Prefill / general forward, fp16 inputs and output (Section 5.1 operator; Section 4.1 method).
+ *   q [B,Sq,Hq,d], k,v [B,Skv,Hkv,d], o [B,Sq,Hq,d] fp16, contiguous; lse [B,Hq,Sq] float or NULL.
+ *   d must be 128.  B == 0 or Sq == 0 is a successful no-op.  Skv == 0 gives O = 0, LSE = -inf.
+ *   o and lse must not alias the inputs.
+ */
+int fa_forward(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+               int Hkv, int Sq, int Skv, int d, int causal, float scale, void* stream);
+
+/* Same operation with bfloat16 inputs and output. */
+int fa_forward_bf16(const void* q, const void* k, const void* v, void* o, float* lse, int B,
+                    int Hq, int Hkv, int Sq, int Skv, int d, int causal, float scale,
+                    void* stream);
+
+/*
+ * Extended form: explicit element strides (batch, sequence, head; d is contiguous) so that
+ * [B,H,S,d] storage can be passed too, and a choice of output type (the input type, or
+ * FA_DTYPE_FP32 to read the fp32 accumulator without the final 16-bit rounding).
+ * A stride of 0 means "contiguous [B,S,H,d]".  Strides must be multiples of 8 elements.
+ */
+typedef struct fa_params {
+    const void* q;
+    const void* k;
+    const void* v;
+    void* o;
+    float* lse; /* may be NULL */
+    int B, Hq, Hkv, Sq, Skv, d;
+    int causal;
+    float scale;
+    int dtype;   /* FA_DTYPE_FP16 or FA_DTYPE_BF16: type of q, k, v */
+    int o_dtype; /* same as dtype, or FA_DTYPE_FP32 */
+    int64_t q_stride[3]; /* batch, sequence, head -- in elements */
+    int64_t k_stride[3];
+    int64_t v_stride[3];
+    int64_t o_stride[3];
+    int variant; /* 0 = default kernel; other values select alternates kept for A/B timing */
+} fa_params;
+
+int fa_forward_ex(const fa_params* p, void* stream);
+
+/*
+ * Decode stage (Appendix C): one query row per sequence over that sequence's cached keys
+ * and values, split along the cache into chunks whose partial results (fp32 O and LSE) are
+ * merged by a second kernel with the same rowmax/rowsum recurrence (Appendix A) applied
+ * across chunks.
+ *   q [B,1,Hq,d] fp16, k_cache,v_cache [B,Skv_max,Hkv,d] fp16, o [B,1,Hq,d] fp16,
+ *   lse [B,Hq] float or NULL, seqlens_k [B] int32 on the DEVICE: only the first
+ *   seqlens_k[b] cache rows of sequence b are read; rows beyond may hold anything (NaN too).
+ *   A sequence with seqlens_k[b] == 0 gives O = 0 and LSE = -inf.  Values of seqlens_k
+ *   outside [0, Skv_max] are clamped.
+ *   workspace: at least fa_decode_workspace_bytes(...) bytes, 16-byte aligned, contents
+ *   need no initialisation and are overwritten.
+ */
+int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+              const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
+              void* workspace, size_t workspace_bytes, void* stream);
+
+size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
+
+/*
+ * Host-buffer form of fa_forward for callers whose tensors live in host memory (pinned memory
+ * makes the copies asynchronous): copies q, k, v to the device staging area, runs the forward,
+ * copies o and lse back, all on `stream`.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16.
+ * staging is a DEVICE buffer of at least fa_forward_host_staging_bytes(...) bytes, 1024-byte
+ * aligned, owned by the caller.  The results are in o_host / lse_host once the stream is idle.
+ */
+int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
+                    float* lse_host, int B, int Hq, int Hkv, int Sq, int Skv, int d, int causal,
+                    float scale, int dtype, void* staging, size_t staging_bytes, void* stream);
+
+size_t fa_forward_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int d);
+
+/*
+ * Reads and clears the device-side status word of the current device.  Synchronises the
+ * device.  Returns FA_OK, FA_ERR_TIMEOUT if a bounded wait expired since the last call
+ * (detail[0] = where, detail[1] = block index, if detail != NULL), or FA_ERR_CUDA.
+ */
+int fa_device_status(unsigned int detail[2]);
+
+const char* fa_strerror(int code);
+int fa_version(void);         /* major * 10000 + minor * 100 + patch */
+int fa_last_cuda_error(void); /* cudaError_t of the last failed CUDA call on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FA_H_ */

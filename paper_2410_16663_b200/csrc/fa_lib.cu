@@ -1,0 +1,383 @@
+// Host side of the C ABI declared in include/fa.h: argument validation, TMA tensor-map
+// encoding, launch configuration.  No device memory is allocated here; every buffer is the
+// caller's.  All kernels live in the headers included below (one translation unit).
+#include "../../include/fa.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "decode.cuh"
+#include "prefill_simple.cuh"
+
+namespace {
+
+thread_local int t_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+    t_last_cuda_error = static_cast<int>(e);
+    return FA_ERR_CUDA;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup, so that the library
+// loads (and can report FA_ERR_DEVICE) on machines without a driver.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Tensor map over a [B, S, H, 128] 16-bit tensor with element strides (sb, ss, sh); a box is
+// box_rows sequence positions x 64 elements of d for one (batch, head), 128-byte swizzled.
+int encode_map(CUtensorMap* tm, const void* base, int B, int S, int H, int64_t sb, int64_t ss, int64_t sh,
+               int box_rows, bool bf16) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return FA_ERR_DEVICE;
+    cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)ss * 2, (cuuint64_t)sb * 2};
+    // a dimension of extent 1 never advances; give it a harmless legal stride
+    if (H == 1) strides[0] = 256;
+    if (S == 1) strides[1] = strides[0] * (cuuint64_t)H;
+    if (B == 1) strides[2] = strides[1] * (cuuint64_t)S;
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
+                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        t_last_cuda_error = static_cast<int>(r);
+        return FA_ERR_CUDA;
+    }
+    return FA_OK;
+}
+
+int check_device() {
+    static thread_local int cached_dev = -1, cached_rc = FA_OK;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev == cached_dev) return cached_rc;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    cached_dev = dev;
+    cached_rc = (major == 10) ? FA_OK : FA_ERR_DEVICE;
+    return cached_rc;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+void default_strides(int64_t s[3], int S, int H) {
+    if (s[0] == 0 && s[1] == 0 && s[2] == 0) {
+        s[2] = 128;
+        s[1] = (int64_t)H * 128;
+        s[0] = (int64_t)S * H * 128;
+    }
+}
+
+bool strides_ok(const int64_t s[3], int B, int S, int H) {
+    for (int i = 0; i < 3; ++i) {
+        if (s[i] < 0 || (s[i] & 7)) return false;
+        if (s[i] >= (1ll << 38)) return false;
+    }
+    if (H > 1 && s[2] < 128) return false;
+    if (S > 1 && s[1] < 128) return false;
+    if (B > 1 && s[0] < 128) return false;
+    return true;
+}
+
+template <typename K>
+int set_smem(K kernel, int bytes) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+constexpr int kSimpleSmem = 1024 + 6 * fa::kTileBytes;
+
+template <typename T, bool kPInTmem>
+int launch_simple(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const fa::FwdParams& fp,
+                  cudaStream_t st) {
+    auto kern = fa::fa_fwd_simple_kernel<T, kPInTmem>;
+    int rc = set_smem(kern, kSimpleSmem);
+    if (rc) return rc;
+    dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
+    kern<<<grid, 128, kSimpleSmem, st>>>(tq, tk, tv, fp);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+int forward_impl(const fa_params& in, cudaStream_t st) {
+    fa_params p = in;
+    // ---- validation (no CUDA call before it passes)
+    if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
+    if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
+    if (p.d != 128) return FA_ERR_UNSUPPORTED;
+    if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
+    if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
+    if (p.causal && p.Sq > p.Skv) return FA_ERR_UNSUPPORTED;
+    if (p.Hq > 65535 || p.B > 65535) return FA_ERR_UNSUPPORTED;
+    if (p.B == 0 || p.Sq == 0) return FA_OK;
+    if (!p.q || !p.o) return FA_ERR_NULL;
+    if (p.Skv > 0 && (!p.k || !p.v)) return FA_ERR_NULL;
+    default_strides(p.q_stride, p.Sq, p.Hq);
+    default_strides(p.k_stride, p.Skv, p.Hkv);
+    default_strides(p.v_stride, p.Skv, p.Hkv);
+    default_strides(p.o_stride, p.Sq, p.Hq);
+    if (!strides_ok(p.q_stride, p.B, p.Sq, p.Hq) || !strides_ok(p.k_stride, p.B, p.Skv, p.Hkv) ||
+        !strides_ok(p.v_stride, p.B, p.Skv, p.Hkv) || !strides_ok(p.o_stride, p.B, p.Sq, p.Hq))
+        return FA_ERR_SHAPE;
+    if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.o)) return FA_ERR_ALIGN;
+    if (p.lse && (reinterpret_cast<uintptr_t>(p.lse) & 3u)) return FA_ERR_ALIGN;
+
+    int rc = check_device();
+    if (rc) return rc;
+
+    fa::FwdParams fp;
+    fp.o = p.o;
+    fp.lse = p.lse;
+    fp.B = p.B; fp.Hq = p.Hq; fp.Hkv = p.Hkv; fp.Sq = p.Sq; fp.Skv = p.Skv;
+    fp.causal = p.causal ? 1 : 0;
+    fp.scale_log2 = p.scale * 1.4426950408889634f;
+    fp.o_sb = p.o_stride[0]; fp.o_ss = p.o_stride[1]; fp.o_sh = p.o_stride[2];
+    fp.o_fp32 = (p.o_dtype == FA_DTYPE_FP32) ? 1 : 0;
+    fp.n_qtiles = (p.Sq + fa::kTile - 1) / fa::kTile;
+    const bool bf16 = p.dtype == FA_DTYPE_BF16;
+
+    if (p.Skv == 0) {
+        const long long rows = (long long)p.B * p.Sq * p.Hq;
+        const int blocks = (int)((rows + 127) / 128 < 4096 ? (rows + 127) / 128 : 4096);
+        if (bf16) fa::fa_fill_empty_kernel<__nv_bfloat16><<<blocks, 128, 0, st>>>(fp);
+        else fa::fa_fill_empty_kernel<__half><<<blocks, 128, 0, st>>>(fp);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
+
+    CUtensorMap tq, tk, tv;
+    rc = encode_map(&tq, p.q, p.B, p.Sq, p.Hq, p.q_stride[0], p.q_stride[1], p.q_stride[2], 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tk, p.k, p.B, p.Skv, p.Hkv, p.k_stride[0], p.k_stride[1], p.k_stride[2], 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16);
+    if (rc) return rc;
+
+    switch (p.variant) {
+        case 0:
+        case 1:  // simple kernel, P handed over through tensor memory
+            return bf16 ? launch_simple<__nv_bfloat16, true>(tq, tk, tv, fp, st)
+                        : launch_simple<__half, true>(tq, tk, tv, fp, st);
+        case 2:  // simple kernel, P handed over through shared memory
+            return bf16 ? launch_simple<__nv_bfloat16, false>(tq, tk, tv, fp, st)
+                        : launch_simple<__half, false>(tq, tk, tv, fp, st);
+        default:
+            return FA_ERR_UNSUPPORTED;
+    }
+}
+
+int forward_plain(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                  int Sq, int Skv, int d, int causal, float scale, int dtype, void* stream) {
+    fa_params p;
+    memset(&p, 0, sizeof p);
+    p.q = q; p.k = k; p.v = v; p.o = o; p.lse = lse;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv; p.d = d;
+    p.causal = causal; p.scale = scale; p.dtype = dtype; p.o_dtype = dtype;
+    return forward_impl(p, static_cast<cudaStream_t>(stream));
+}
+
+// ---- decode helpers
+int decode_chunk(int B, int Hkv, int Smax) {
+    // Largest chunk that still leaves several waves of work items for 148 SMs; multiples of the tile.
+    const long long target = 4ll * 148;
+    int chunk = 2048;
+    while (chunk > 256 && (long long)B * Hkv * ((Smax + chunk - 1) / chunk) < target) chunk >>= 1;
+    return chunk;
+}
+
+template <typename T, int G>
+int launch_decode_split(const CUtensorMap& tk, const CUtensorMap& tv, const fa::DecodeParams& dp, int items,
+                        cudaStream_t st) {
+    constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
+    auto kern = fa::fa_decode_split_kernel<T, G>;
+    int rc = set_smem(kern, smem);
+    if (rc) return rc;
+    dim3 grid(dp.n_chunks, items, dp.B);
+    kern<<<grid, fa::kDecThreads, smem, st>>>(tk, tv, dp);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int fa_forward(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+               int Skv, int d, int causal, float scale, void* stream) {
+    return forward_plain(q, k, v, o, lse, B, Hq, Hkv, Sq, Skv, d, causal, scale, FA_DTYPE_FP16, stream);
+}
+
+int fa_forward_bf16(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
+                    int Sq, int Skv, int d, int causal, float scale, void* stream) {
+    return forward_plain(q, k, v, o, lse, B, Hq, Hkv, Sq, Skv, d, causal, scale, FA_DTYPE_BF16, stream);
+}
+
+int fa_forward_ex(const fa_params* p, void* stream) {
+    if (!p) return FA_ERR_NULL;
+    return forward_impl(*p, static_cast<cudaStream_t>(stream));
+}
+
+size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Skv_max <= 0 || d != 128) return 0;
+    const int chunk = decode_chunk(B, Hkv, Skv_max);
+    const size_t nc = (size_t)((Skv_max + chunk - 1) / chunk);
+    return (size_t)B * Hq * nc * (128 + 1) * sizeof(float);
+}
+
+int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+              int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
+              void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
+    if (B > 65535 || Hq > 65535) return FA_ERR_UNSUPPORTED;
+    if (B == 0) return FA_OK;
+    if (!q || !o || !seqlens_k) return FA_ERR_NULL;
+    if (Skv_max > 0 && (!k_cache || !v_cache)) return FA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(workspace))
+        return FA_ERR_ALIGN;
+    const size_t need = fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return FA_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    fa::DecodeParams dp;
+    dp.q = q;
+    dp.seqlens = seqlens_k;
+    dp.B = B; dp.Hq = Hq; dp.Hkv = Hkv; dp.Smax = Skv_max;
+    dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max) : 256;
+    dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
+    dp.o_part = static_cast<float*>(workspace);
+    dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
+    dp.scale_log2 = scale * 1.4426950408889634f;
+    const int g = Hq / Hkv;
+
+    if (Skv_max > 0) {
+        CUtensorMap tk, tv;
+        rc = encode_map(&tk, k_cache, B, Skv_max, Hkv, (int64_t)Skv_max * Hkv * 128, (int64_t)Hkv * 128, 128,
+                        fa::kDecTile, false);
+        if (rc) return rc;
+        rc = encode_map(&tv, v_cache, B, Skv_max, Hkv, (int64_t)Skv_max * Hkv * 128, (int64_t)Hkv * 128, 128,
+                        fa::kDecTile, false);
+        if (rc) return rc;
+        switch (g) {
+            case 1: dp.heads_per_item = 1; rc = launch_decode_split<__half, 1>(tk, tv, dp, Hq, st); break;
+            case 2: dp.heads_per_item = 2; rc = launch_decode_split<__half, 2>(tk, tv, dp, Hkv, st); break;
+            case 4: dp.heads_per_item = 4; rc = launch_decode_split<__half, 4>(tk, tv, dp, Hkv, st); break;
+            case 8: dp.heads_per_item = 8; rc = launch_decode_split<__half, 8>(tk, tv, dp, Hkv, st); break;
+            default:  // other group sizes: one query head per item (the kv head is re-read per head)
+                dp.heads_per_item = 1; rc = launch_decode_split<__half, 1>(tk, tv, dp, Hq, st); break;
+        }
+        if (rc) return rc;
+    }
+    fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+size_t fa_forward_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int d) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv < 0 || d != 128) return 0;
+    auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    const size_t qo = up((size_t)B * Sq * Hq * 128 * 2);
+    const size_t kv = up((size_t)B * Skv * Hkv * 128 * 2);
+    const size_t l = up((size_t)B * Hq * Sq * 4);
+    return 2 * qo + 2 * kv + l;
+}
+
+int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host, float* lse_host,
+                    int B, int Hq, int Hkv, int Sq, int Skv, int d, int causal, float scale, int dtype,
+                    void* staging, size_t staging_bytes, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Sq < 0 || Skv < 0 || d <= 0) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (B == 0 || Sq == 0) return FA_OK;
+    if (!q_host || !o_host || (Skv > 0 && (!k_host || !v_host))) return FA_ERR_NULL;
+    const size_t need = fa_forward_host_staging_bytes(B, Hq, Hkv, Sq, Skv, d);
+    if (!staging || staging_bytes < need) return FA_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(staging) & 1023u) return FA_ERR_ALIGN;
+    auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    const size_t qo_b = (size_t)B * Sq * Hq * 128 * 2, kv_b = (size_t)B * Skv * Hkv * 128 * 2;
+    const size_t l_b = (size_t)B * Hq * Sq * 4;
+    char* base = static_cast<char*>(staging);
+    char* dq = base;
+    char* dk = dq + up(qo_b);
+    char* dv = dk + up(kv_b);
+    char* dout = dv + up(kv_b);
+    char* dl = dout + up(qo_b);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dq, q_host, qo_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    if (kv_b) {
+        if ((e = cudaMemcpyAsync(dk, k_host, kv_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(dv, v_host, kv_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    }
+    int rc = forward_plain(dq, dk, dv, dout, reinterpret_cast<float*>(dl), B, Hq, Hkv, Sq, Skv, d, causal, scale,
+                           dtype, stream);
+    if (rc) return rc;
+    if ((e = cudaMemcpyAsync(o_host, dout, qo_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if (lse_host)
+        if ((e = cudaMemcpyAsync(lse_host, dl, l_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    return FA_OK;
+}
+
+int fa_device_status(unsigned int detail[2]) {
+    unsigned int h[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaMemcpyFromSymbol(h, fa::g_status, sizeof h);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (h[0] == 0) return FA_OK;
+    if (detail) {
+        detail[0] = h[1];
+        detail[1] = h[2];
+    }
+    unsigned int z[4] = {0, 0, 0, 0};
+    e = cudaMemcpyToSymbol(fa::g_status, z, sizeof z);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return FA_ERR_TIMEOUT;
+}
+
+const char* fa_strerror(int code) {
+    switch (code) {
+        case FA_OK: return "ok";
+        case FA_ERR_NULL: return "a required pointer is NULL";
+        case FA_ERR_SHAPE: return "invalid shape or stride";
+        case FA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case FA_ERR_ALIGN: return "pointer not sufficiently aligned";
+        case FA_ERR_WORKSPACE: return "workspace missing or too small";
+        case FA_ERR_DEVICE: return "device is not compute capability 10.x or no driver";
+        case FA_ERR_CUDA: return "CUDA call failed (see fa_last_cuda_error)";
+        case FA_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown error code";
+    }
+}
+
+int fa_version(void) { return 100; }
+
+int fa_last_cuda_error(void) { return t_last_cuda_error; }
+
+}  // extern "C"

@@ -1,0 +1,336 @@
+// Prefill forward, straightforward variant: one CTA of 128 threads per (batch, head, 128-row
+// query tile), one thread per query row.  Thread 0 additionally issues the TMA loads and the
+// tcgen05 MMAs.  K/V tiles go through a two-slot shared-memory ring; S = Q K^T and O += P V
+// both accumulate in tensor memory; P is handed to the second MMA either through tensor
+// memory (packed 16-bit, over the columns S occupied) or through a swizzled shared-memory
+// tile.  Every step of the four-stage block loop (Q*K^T, Exp, Exp*V, rowmax/rowsum update)
+// runs strictly one after the other, so this kernel is the reference point the pipelined
+// kernel is measured against, and the one kept for A/B checks.
+#pragma once
+
+#include <type_traits>
+
+#include "sm100_ptx.cuh"
+
+namespace fa {
+
+struct FwdParams {
+    void* o;
+    float* lse;
+    int B, Hq, Hkv, Sq, Skv;
+    int causal;
+    float scale_log2;  // scale * log2(e)
+    long long o_sb, o_ss, o_sh;  // element strides of o
+    int o_fp32;
+    int n_qtiles;
+};
+
+constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim
+constexpr int kHalfBytes = 16384;   // one 128-row x 64-element 16-bit box
+constexpr int kTileBytes = 32768;   // a 128 x 128 16-bit tile = two boxes
+
+// Loads one 128x128 16-bit tile (rows s0.., all of d) as two 64-column swizzled boxes.
+__device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                          int h, int s0, int b) {
+    tma_load_4d(dst, tm, bar, 0, h, s0, b);
+    tma_load_4d(dst + kHalfBytes, tm, bar, 64, h, s0, b);
+}
+
+// Number of kv tiles a query tile starting at row q0 has to visit.
+__device__ __forceinline__ int kv_tiles_for(int q0, int q_rows, int Sq, int Skv, int causal) {
+    int n = (Skv + kTile - 1) / kTile;
+    if (causal) {
+        int last_row = min(q0 + q_rows, Sq) - 1;
+        int last_key = last_row + (Skv - Sq);  // >= 0 because Sq <= Skv
+        n = min(n, last_key / kTile + 1);
+    }
+    return n;
+}
+
+template <typename T, bool kPInTmem>
+__global__ void __launch_bounds__(128, 1)
+fa_fwd_simple_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the 128-byte swizzle
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + kTileBytes;           // 2 slots
+    const uint32_t sV = sK + 2 * kTileBytes;       // 2 slots
+    const uint32_t sP = sV + 2 * kTileBytes;       // 1 tile (only when !kPInTmem)
+    __shared__ __align__(8) uint64_t bars[8];
+    __shared__ uint32_t tmem_holder;
+    __shared__ volatile uint32_t abort_flag;
+
+    const uint32_t bar_q = smem_u32(&bars[0]);
+    const uint32_t bar_k0 = smem_u32(&bars[1]);  // +8 for slot 1
+    const uint32_t bar_v0 = smem_u32(&bars[3]);
+    const uint32_t bar_s = smem_u32(&bars[5]);
+    const uint32_t bar_o = smem_u32(&bars[6]);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int qt = p.n_qtiles - 1 - blockIdx.x;  // long (late) tiles first
+    const int h = blockIdx.y;
+    const int b = blockIdx.z;
+    const int hk = h / (p.Hq / p.Hkv);
+    const int q0 = qt * kTile;
+    const int off = p.Skv - p.Sq;
+    const int n_tiles = kv_tiles_for(q0, kTile, p.Sq, p.Skv, p.causal);
+
+    if (tid == 0) {
+        for (int i = 0; i < 7; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&tmem_holder), 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t tS = tmem_base + lane_sel;        // columns [0,128): S, then P packed in [0,64)
+    const uint32_t tO = tmem_base + lane_sel + 128;  // columns [128,256): O
+
+    constexpr uint32_t idesc_qk = instr_desc_f16(std::is_same<T, __nv_bfloat16>::value, 128, 128, false, false);
+    constexpr uint32_t idesc_pv = instr_desc_f16(std::is_same<T, __nv_bfloat16>::value, 128, 128, false, true);
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_q, kTileBytes);
+        load_tile(sQ, &tm_q, bar_q, h, q0, b);
+        for (int j = 0; j < 2 && j < n_tiles; ++j) {
+            mbar_expect_tx(bar_k0 + 8 * j, kTileBytes);
+            load_tile(sK + j * kTileBytes, &tm_k, bar_k0 + 8 * j, hk, j * kTile, b);
+            mbar_expect_tx(bar_v0 + 8 * j, kTileBytes);
+            load_tile(sV + j * kTileBytes, &tm_v, bar_v0 + 8 * j, hk, j * kTile, b);
+        }
+    }
+    __syncwarp();
+
+    const int row = q0 + tid;          // this thread's query row
+    float m_run = -INFINITY;           // running row max, in raw score units
+    float l_run = 0.f;                 // running row sum
+    bool ok = true;
+
+    for (int j = 0; j < n_tiles && ok; ++j) {
+        const int slot = j & 1;
+        const uint32_t ring_parity = (j >> 1) & 1;
+        // ---- S = Q K_j^T
+        if (tid == 0) {
+            if (j == 0) ok = mbar_wait(bar_q, 0, &abort_flag, 1);
+            ok = ok && mbar_wait(bar_k0 + 8 * slot, ring_parity, &abort_flag, 2);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                    mma_ss(tmem_base, smem_desc_sw128(sQ + koff, 16, 1024),
+                           smem_desc_sw128(sK + slot * kTileBytes + koff, 16, 1024), idesc_qk,
+                           ks > 0);
+                }
+                mma_commit(bar_s);
+            }
+        }
+        __syncwarp();
+        if (!mbar_wait(bar_s, j & 1, &abort_flag, 3)) { ok = false; break; }
+        tc_fence_after();
+
+        // ---- load this row of S
+        float s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tS + c * 32, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
+        }
+        // ---- mask: only tiles the diagonal or the end of the keys cross
+        const int kv0 = j * kTile;
+        const bool need_mask = (p.causal && kv0 + kTile - 1 > q0 + off) || (kv0 + kTile > p.Skv);
+        if (need_mask) {
+            int lim = p.Skv - kv0;                                // columns >= lim are past the keys
+            if (p.causal) lim = min(lim, row + off - kv0 + 1);    // columns >= lim are above the diagonal
+#pragma unroll
+            for (int i = 0; i < 128; ++i)
+                if (i >= lim) s[i] = -INFINITY;
+        }
+        // ---- online softmax update (Appendix A: rowmax / rowsum)
+        float m_tile = s[0];
+#pragma unroll
+        for (int i = 1; i < 128; ++i) m_tile = fmaxf(m_tile, s[i]);
+        const float m_new = fmaxf(m_run, m_tile);
+        // rows past Sq in a ragged last tile may see nothing; keep them finite
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - m_use) * p.scale_log2);
+        const float neg_ms = -m_use * p.scale_log2;
+        float l_tile = 0.f;
+        if (need_mask) {
+            // masked entries become exact zeros whatever the scale (0 * -inf would be NaN)
+            int lim = p.Skv - kv0;
+            if (p.causal) lim = min(lim, row + off - kv0 + 1);
+#pragma unroll
+            for (int i = 0; i < 128; ++i) {
+                s[i] = (i < lim) ? fast_exp2(fmaf(s[i], p.scale_log2, neg_ms)) : 0.f;
+                l_tile += s[i];
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 128; ++i) {
+                s[i] = fast_exp2(fmaf(s[i], p.scale_log2, neg_ms));
+                l_tile += s[i];
+            }
+        }
+        l_run = l_run * alpha + l_tile;
+        m_run = m_new;
+
+        // ---- O <- alpha * O once the previous P V has landed; refill the slot it freed
+        if (j > 0) {
+            if (!mbar_wait(bar_o, (j - 1) & 1, &abort_flag, 4)) { ok = false; break; }
+            tc_fence_after();
+            if (tid == 0 && j + 1 < n_tiles) {
+                const int ns = (j + 1) & 1;
+                mbar_expect_tx(bar_k0 + 8 * ns, kTileBytes);
+                load_tile(sK + ns * kTileBytes, &tm_k, bar_k0 + 8 * ns, hk, (j + 1) * kTile, b);
+                mbar_expect_tx(bar_v0 + 8 * ns, kTileBytes);
+                load_tile(sV + ns * kTileBytes, &tm_v, bar_v0 + 8 * ns, hk, (j + 1) * kTile, b);
+            }
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(tO + c * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                tmem_st_x32(tO + c * 32, r);
+            }
+        }
+        // ---- hand P to the second MMA
+        if constexpr (kPInTmem) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t r[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = pack2<T>(s[c * 64 + 2 * i], s[c * 64 + 2 * i + 1]);
+                tmem_st_x32(tS + c * 32, r);
+            }
+        } else {
+            // row `tid` of the swizzled tile: 16-byte chunk c of a 128-byte row sits at c ^ (row & 7)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const uint32_t row_base = sP + half * kHalfBytes + tid * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const int e = half * 64 + c * 8;
+                    uint32_t w0 = pack2<T>(s[e], s[e + 1]), w1 = pack2<T>(s[e + 2], s[e + 3]);
+                    uint32_t w2 = pack2<T>(s[e + 4], s[e + 5]), w3 = pack2<T>(s[e + 6], s[e + 7]);
+                    const uint32_t addr = row_base + ((c ^ (tid & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0),
+                                 "r"(w1), "r"(w2), "r"(w3)
+                                 : "memory");
+                }
+            }
+            fence_proxy_async_smem();
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncthreads();
+        // ---- O += P V_j
+        if (tid == 0) {
+            ok = mbar_wait(bar_v0 + 8 * slot, ring_parity, &abort_flag, 5);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    // 16 kv rows per step: 2048 bytes down the swizzled V tile (MN-major B)
+                    const uint64_t bdesc =
+                        smem_desc_sw128(sV + slot * kTileBytes + ks * 2048, kHalfBytes, 1024);
+                    if constexpr (kPInTmem) {
+                        mma_ts(tmem_base + 128, tmem_base + ks * 8, bdesc, idesc_pv, (j > 0) || (ks > 0));
+                    } else {
+                        const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                        mma_ss(tmem_base + 128, smem_desc_sw128(sP + koff, 16, 1024), bdesc, idesc_pv,
+                               (j > 0) || (ks > 0));
+                    }
+                }
+                mma_commit(bar_o);
+            }
+        }
+        __syncwarp();
+    }
+
+    // ---- epilogue: O / l, LSE = m*scale + ln l
+    if (ok && n_tiles > 0) ok = mbar_wait(bar_o, (n_tiles - 1) & 1, &abort_flag, 6);
+    if (ok && n_tiles > 0) {
+        tc_fence_after();
+        const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+        const bool live = row < p.Sq;
+        const long long obase = (long long)b * p.o_sb + (long long)row * p.o_ss + (long long)h * p.o_sh;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tO + c * 32, r);
+            tmem_wait_ld();
+            if (live) {
+                if (p.o_fp32) {
+                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
+                                             __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
+                } else {
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.o) + obase + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 w;
+                        w.x = pack2<T>(__uint_as_float(r[8 * i]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
+                        w.y = pack2<T>(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
+                        w.z = pack2<T>(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
+                        w.w = pack2<T>(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                        dst[i] = w;
+                    }
+                }
+            }
+        }
+        if (live && p.lse != nullptr) {
+            const float lse = (l_run > 0.f) ? (m_run * p.scale_log2 + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            p.lse[((long long)b * p.Hq + h) * p.Sq + row] = lse;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
+// O = 0, LSE = -inf for a problem without keys.
+template <typename T>
+__global__ void fa_fill_empty_kernel(const FwdParams p) {
+    const long long n = (long long)p.B * p.Sq * p.Hq;
+    for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < n;
+         r += (long long)gridDim.x * blockDim.x) {
+        const int h = r % p.Hq;
+        const long long bi = r / p.Hq;
+        const int i = bi % p.Sq;
+        const int b = bi / p.Sq;
+        const long long obase = (long long)b * p.o_sb + (long long)i * p.o_ss + (long long)h * p.o_sh;
+        for (int t = 0; t < kTile; ++t) {
+            if (p.o_fp32) static_cast<float*>(p.o)[obase + t] = 0.f;
+            else static_cast<T*>(p.o)[obase + t] = T(0.f);
+        }
+        if (p.lse) p.lse[((long long)b * p.Hq + h) * p.Sq + i] = -INFINITY;
+    }
+}
+
+}  // namespace fa
