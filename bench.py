@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the attention hot path on B200: one JSON line on stdout.
+
+A step is one pass of the whole path over one batch of synthetic input:
+  1. causal prefill, Llama-7B shape (B=4, Hq=Hkv=32, S=2048, d=128, fp16)  -> fa_forward
+  2. split-KV decode, B=64, Hq=32, Hkv=32, Skv ~ U[1K,32K], fp16 cache     -> fa_decode
+  3. the same decode with Hkv=8 (grouped-query variant)                   -> fa_decode
+Each part is timed with CUDA events on the launching stream inside the step.  `value` is the
+prefill throughput in TFLOPS (causal FLOPs credited as 2*B*Hq*Sq*Skv*d); the decode parts
+report cache bytes per second.  Inputs are resident in HBM before the timed region; the `e2e`
+object repeats the measurement through the host-buffer entry point with the copies timed.
+
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2410_16663_b200 import inputs as synth
+
+METRIC = "causal fp16 attention fwd TFLOPS + % of tensor peak; decode KV HBM GB/s"
+NOMINAL_TENSOR_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        pk["source"] = "measured"
+        return pk
+    pk = dict(FALLBACK_PEAKS)
+    pk["source"] = "fallback"
+    return pk
+
+
+# --------------------------------------------------------------------------- clock sampling
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {}
+        for n in dir(nv):
+            if n.startswith("nvmlClocksThrottleReason") or n.startswith("nvmlClocksEventReason"):
+                val = getattr(nv, n)
+                if isinstance(val, int) and val not in (0,):
+                    names[val] = n.replace("nvmlClocksThrottleReason", "").replace("nvmlClocksEventReason", "")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit and bit & (bit - 1) == 0 and name not in ("GpuIdle", "All"):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- workload
+def visible_device_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def decode_cache_bytes(cfg, seqlens) -> float:
+    """Algorithmic HBM bytes of one decode pass: every valid K and V row once, plus q, o."""
+    kv = float(seqlens.sum().item()) * cfg.Hkv * cfg.d * 2 * 2
+    return kv + 2.0 * cfg.B * cfg.Hq * cfg.d * 2
+
+
+def run_product(args, rank, world, local_rank):
+    from paper_2410_16663_b200 import binding as fa  # raises if the CUDA library is missing
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback exists)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+
+    pc = synth.C2
+    dcs = [synth.C5_MHA, synth.C5_GQA]
+    if args.small:  # debugging aid: same path, small shapes (not a reportable number)
+        pc = synth.PrefillConfig("C2-small", 1, 8, 8, 1024, 1024, seed=5)
+        dcs = [synth.DecodeConfig("C5-small", 8, 8, 8, 4096, 512, 4096, seed=6),
+               synth.DecodeConfig("C5-small-gqa", 8, 8, 2, 4096, 512, 4096, seed=7)]
+
+    q, k, v = synth.prefill_inputs(pc, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(pc.B, pc.Hq, pc.Sq, dtype=torch.float32, device=dev)
+    dec = []
+    for dc in dcs:
+        dq, dk, dv, sl = synth.decode_inputs(dc, device=dev, poison=True)
+        do = torch.empty_like(dq)
+        dl = torch.empty(dc.B, dc.Hq, dtype=torch.float32, device=dev)
+        ws = torch.empty(max(16, fa.fa_decode_workspace_bytes(dc.B, dc.Hq, dc.Hkv, dc.Smax, dc.d)),
+                         dtype=torch.uint8, device=dev)
+        dec.append(dict(cfg=dc, q=dq, k=dk, v=dv, sl_host=sl, sl=sl.to(dev), o=do, lse=dl, ws=ws,
+                        bytes=decode_cache_bytes(dc, sl)))
+
+    def step(ev=None):
+        if ev: ev[0].record()
+        fa.fa_forward(q, k, v, o, lse, pc.causal, pc.scale)
+        if ev: ev[1].record()
+        for i, d in enumerate(dec):
+            fa.fa_decode(d["q"], d["k"], d["v"], d["o"], d["lse"], d["sl"], d["cfg"].scale, d["ws"])
+            if ev: ev[2 + i].record()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    sampler = ClockSampler(visible_device_index(local_rank))
+    nparts = 1 + len(dec)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(nparts + 1)] for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    sampler.start()
+    t_all0 = torch.cuda.Event(enable_timing=True)
+    t_all1 = torch.cuda.Event(enable_timing=True)
+    t_all0.record()
+    for s in range(args.steps):
+        step(events[s])
+    t_all1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = t_all0.elapsed_time(t_all1)
+    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) / args.steps for i in range(nparts)]
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+
+    # ---- max over ranks (device-timed), whole-job aggregate
+    ms_step = total_ms / args.steps
+    times = torch.tensor([ms_step] + part_ms, dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+        dist.barrier()
+    ms_step, part_ms = float(times[0]), [float(x) for x in times[1:]]
+
+    tflops = world * pc.flops() / (part_ms[0] * 1e-3) / 1e12
+    out = {
+        "metric": METRIC, "value": round(tflops, 2), "unit": "TFLOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+        "data": "synthetic",
+        "config": {"workload": f"{pc.name}: causal prefill B={pc.B} Hq=Hkv={pc.Hq} Sq=Skv={pc.Sq} d=128 fp16"
+                               f" + decode {dcs[0].name} and {dcs[1].name} (B={dcs[0].B}, Hq={dcs[0].Hq},"
+                               f" Hkv={dcs[0].Hkv}/{dcs[1].Hkv}, Skv~U[{dcs[0].len_lo},{dcs[0].len_hi}])",
+                   "parallelism": f"replicas x{world} (batch/head sharding, no collective)",
+                   "l2": "inputs larger than L2 (prefill 256 MiB per step; the decode passes between "
+                         "prefill launches stream tens of GiB)",
+                   "flop_convention": "causal 2*B*Hq*Sq*Skv*d"},
+        "prefill": {"ms": round(part_ms[0], 4), "tflops": round(tflops, 2),
+                    "frac_nominal_tensor": round(tflops / world / NOMINAL_TENSOR_TFLOPS, 4),
+                    "frac_measured_tensor": round(tflops / world / peaks["bf16_tflops"], 4)},
+        "gpu_launches": args.steps * (1 + 2 * len(dec)),
+        "clocks": clocks,
+    }
+    for i, d in enumerate(dec):
+        gbs = world * d["bytes"] / (part_ms[1 + i] * 1e-3) / 1e9
+        out["decode_" + ("mha" if i == 0 else "gqa")] = {
+            "ms": round(part_ms[1 + i], 4), "gbs": round(gbs, 1), "kv_bytes": d["bytes"],
+            "frac_nominal_hbm": round(gbs / world / NOMINAL_HBM_GBS, 4),
+            "frac_measured_hbm": round(gbs / world / peaks["hbm_gbs"], 4)}
+    # roofline of the kernel behind `value` (prefill: a dense contraction -> tensor peak, burst
+    # figure because one launch lasts a fraction of a millisecond) and of the decode scan (HBM)
+    out["roofline"] = {"kernel": "fa_fwd (prefill)", "bound": "tensor", "achieved": round(tflops / world, 2),
+                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                       "frac": round(tflops / world / peaks["bf16_tflops"], 4),
+                       "peak_source": peaks["source"] + " (bf16 GEMM burst; fp16 has the same nominal rate)",
+                       "traffic": None}
+    g0 = out["decode_mha"]["gbs"] / world
+    out["roofline_decode"] = {"kernel": "fa_decode_split (decode, Hkv=32)", "bound": "hbm",
+                              "achieved": round(g0, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": round(g0 / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],
+                              "traffic": None}
+
+    if rank == 0:
+        out["e2e"] = run_e2e(args, fa, pc, dec, dev)
+        out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
+        print(json.dumps(out), flush=True)
+
+
+def run_e2e(args, fa, pc, dec, dev):
+    """Same metric through the host-buffer entry point: inputs start in pinned host memory, the
+    result is read back to the host, copies inside the timed region."""
+    qh, kh, vh = [t.pin_memory() for t in synth.prefill_inputs(pc, device="cpu")]
+    oh = torch.empty_like(qh).pin_memory()
+    lh = torch.empty(pc.B, pc.Hq, pc.Sq, dtype=torch.float32).pin_memory()
+    nbytes = fa.fa_forward_host_staging_bytes(pc.B, pc.Hq, pc.Hkv, pc.Sq, pc.Skv, pc.d)
+    staging = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+    off = (-staging.data_ptr()) % 1024
+    staging = staging[off:off + nbytes]
+    steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        fa.fa_forward_host(qh, kh, vh, oh, lh, pc.causal, pc.scale, staging)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fa.fa_forward_host(qh, kh, vh, oh, lh, pc.causal, pc.scale, staging)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    h2d = qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2
+    d2h = oh.numel() * 2 + lh.numel() * 4
+    res = {"value": round(pc.flops() / (ms * 1e-3) / 1e12, 3), "unit": "TFLOPS", "ms": round(ms, 4),
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
+           "entry": "fa_forward_host (pinned host q,k,v -> device, forward, o,lse -> host)"}
+    # decode end to end: the KV cache is device-resident state by definition; the step's inputs
+    # are the new queries and lengths, its result the attention rows
+    d = dec[0]
+    qh2 = d["q"].cpu().pin_memory()
+    slh = d["sl_host"].pin_memory()
+    oh2 = torch.empty_like(qh2).pin_memory()
+    for it in range(steps + 3):
+        if it == 3:
+            torch.cuda.synchronize()
+            e0.record()
+        d["q"].copy_(qh2, non_blocking=True)
+        d["sl"].copy_(slh, non_blocking=True)
+        fa.fa_decode(d["q"], d["k"], d["v"], d["o"], d["lse"], d["sl"], d["cfg"].scale, d["ws"])
+        oh2.copy_(d["o"], non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    ms2 = e0.elapsed_time(e1) / steps
+    res["decode_mha"] = {"gbs": round(d["bytes"] / (ms2 * 1e-3) / 1e9, 1), "ms": round(ms2, 4),
+                         "h2d_bytes_per_step": qh2.numel() * 2 + slh.numel() * 4,
+                         "d2h_bytes_per_step": oh2.numel() * 2,
+                         "note": "KV cache resident on the device (it is the decode stage's state)"}
+    return res
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_rows(pc, n_rows, seed):
+    g = torch.Generator().manual_seed(seed)
+    b = torch.randint(0, pc.B, (n_rows,), generator=g)
+    h = torch.randint(0, pc.Hq, (n_rows,), generator=g)
+    i = torch.randint(0, pc.Sq, (n_rows,), generator=g)
+    return torch.stack([b, h, i], dim=1).to(torch.int32).numpy()
+
+
+def rows_flops(pc, rows) -> float:
+    """Credited FLOPs of the sampled rows: 4*d per visible key (QK^T and PV)."""
+    off = pc.Skv - pc.Sq
+    vis = [(min(pc.Skv, int(r[2]) + off + 1) if pc.causal else pc.Skv) for r in rows]
+    return 4.0 * pc.d * float(sum(vis))
+
+
+def time_oracle(pc, q, k, v, n_rows, seed):
+    import oracle
+    rows = oracle_sample_rows(pc, n_rows, seed)
+    t0 = time.perf_counter()
+    oracle.attention_rows(q, k, v, pc.causal, pc.scale, rows)
+    dt = time.perf_counter() - t0
+    return dt, rows_flops(pc, rows)
+
+
+def run_cpu_baseline(pc, budget_s=12.0):
+    import oracle
+    q, k, v = synth.prefill_inputs(pc, device="cpu")
+    dt, fl = time_oracle(pc, q, k, v, 256, 11)           # calibration
+    n = int(max(256, min(2_000_000, 256 * budget_s / max(dt, 1e-3))))
+    dt, fl = time_oracle(pc, q, k, v, n, 12)
+    return {"value": round(fl / dt / 1e12, 6), "unit": "TFLOPS", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": round(dt, 2),
+            "sample": f"{n} uniformly sampled (b,h,i) rows of {pc.name} (row-sampled fp64 oracle, "
+                      f"credited 4*d FLOPs per visible key)"}
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle as it stands, on the host cores, rank 0 only."""
+    if rank != 0:
+        return
+    import oracle
+    pc = synth.C2
+    q, k, v = synth.prefill_inputs(pc, device="cpu")
+    dt, _ = time_oracle(pc, q, k, v, 128, 21)
+    per_step_s = min(8.0, 120.0 / max(1, args.steps + args.warmup))
+    n = int(max(64, 128 * per_step_s / max(dt, 1e-3)))
+    for s in range(args.warmup):
+        time_oracle(pc, q, k, v, n, 100 + s)
+    tot_t, tot_f = 0.0, 0.0
+    for s in range(args.steps):
+        dt, fl = time_oracle(pc, q, k, v, n, 200 + s)
+        tot_t += dt
+        tot_f += fl
+    val = tot_f / tot_t / 1e12
+    sample = f"{n} sampled rows of {pc.name} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(val, 6), "unit": "TFLOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(tot_t / max(1, args.steps) * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{pc.name}: causal prefill B={pc.B} Hq=Hkv={pc.Hq} Sq=Skv={pc.Sq} d=128 fp16 "
+                               f"(bounded row sample per step)"},
+        "cpu_baseline": {"value": round(val, 6), "unit": "TFLOPS", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(val, 6), "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="product", choices=["product", "reference"])
+    ap.add_argument("--small", action="store_true", help="small shapes, for debugging only")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_product(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,138 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def fa():
+    from paper_2410_16663_b200 import build
+    build.build()
+    from paper_2410_16663_b200 import binding
+    return binding
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "fa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fa_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(fa):
+    names = header_functions()
+    assert "fa_forward" in names and "fa_decode" in names and len(names) >= 10
+    for n in names:
+        assert hasattr(fa.lib, n), f"{n} declared in include/fa.h but not exported"
+    assert sorted(fa.EXPORTS) == sorted(n for n in names)
+
+
+def test_version_and_strerror(fa):
+    assert fa.fa_version() >= 100
+    for code in range(0, -9, -1):
+        assert fa.fa_strerror(code) and "unknown" not in fa.fa_strerror(code)
+    assert "unknown" in fa.fa_strerror(-99)
+
+
+def _t(*shape, dtype=torch.float16):
+    return torch.zeros(*shape, dtype=dtype)
+
+
+def test_forward_validation_happens_before_any_cuda_call(fa):
+    q, k = _t(1, 4, 4, 128), _t(1, 4, 2, 128)
+    o = _t(1, 4, 4, 128)
+    L = fa.lib
+    P = lambda t: t.data_ptr()
+    # no-ops
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 0, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_OK
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 0, 4, 128, 1, 0.1, None) == fa.FA_OK
+    # shapes
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 3, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_SHAPE
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, -1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_SHAPE
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 0, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_SHAPE
+    # unsupported
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 64, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 5, 4, 128, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, -1.0, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, float("nan"), None) == fa.FA_ERR_UNSUPPORTED
+    # null / alignment
+    assert L.fa_forward(None, P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_NULL
+    assert L.fa_forward(P(q), None, P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_NULL
+    assert L.fa_forward(P(q), P(k), P(k), None, None, 1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_NULL
+    assert L.fa_forward(P(q) + 2, P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_ALIGN
+    assert L.fa_forward_bf16(P(q), P(k), P(k), P(o) + 8, None, 1, 4, 2, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_ALIGN
+    assert L.fa_forward_ex(None, None) == fa.FA_ERR_NULL
+
+
+def test_forward_ex_rejects_bad_strides_and_types(fa):
+    q = _t(1, 4, 4, 128)
+    p = fa.fa_params()
+    p.q = p.k = p.v = p.o = q.data_ptr()
+    p.B, p.Hq, p.Hkv, p.Sq, p.Skv, p.d = 1, 4, 4, 4, 4, 128
+    p.scale, p.dtype, p.o_dtype = 0.1, fa.FA_DTYPE_FP16, fa.FA_DTYPE_FP16
+    p.q_stride[0], p.q_stride[1], p.q_stride[2] = 2048, 512, 100   # head stride not a multiple of 8
+    assert fa.lib.fa_forward_ex(ctypes.byref(p), None) == fa.FA_ERR_SHAPE
+    p.q_stride[2] = 128
+    p.dtype = 7
+    assert fa.lib.fa_forward_ex(ctypes.byref(p), None) == fa.FA_ERR_UNSUPPORTED
+    p.dtype, p.o_dtype = fa.FA_DTYPE_FP16, fa.FA_DTYPE_BF16
+    assert fa.lib.fa_forward_ex(ctypes.byref(p), None) == fa.FA_ERR_UNSUPPORTED
+    p.o_dtype, p.variant = fa.FA_DTYPE_FP16, 0
+
+
+def test_decode_validation_and_workspace_size(fa):
+    L = fa.lib
+    q, kc, o = _t(2, 1, 8, 128), _t(2, 256, 2, 128), _t(2, 1, 8, 128)
+    sl = torch.zeros(2, dtype=torch.int32)
+    ws = torch.zeros(1 << 16, dtype=torch.uint8)
+    P = lambda t: t.data_ptr()
+    need = fa.fa_decode_workspace_bytes(2, 8, 2, 256, 128)
+    assert need == 2 * 8 * 1 * 129 * 4
+    assert fa.fa_decode_workspace_bytes(2, 8, 2, 256, 64) == 0
+    # large problems use 2048-key chunks
+    assert fa.fa_decode_workspace_bytes(64, 32, 32, 32768, 128) == 64 * 32 * 16 * 129 * 4
+    args = lambda **kw: None
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 2, 8, 3, 256, 128, 0.1, P(ws), need, None) == fa.FA_ERR_SHAPE
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 2, 8, 2, 256, 96, 0.1, P(ws), need, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, None, 2, 8, 2, 256, 128, 0.1, P(ws), need, None) == fa.FA_ERR_NULL
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 2, 8, 2, 256, 128, 0.1, P(ws), need - 1, None) == fa.FA_ERR_WORKSPACE
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 2, 8, 2, 256, 128, 0.1, None, 0, None) == fa.FA_ERR_WORKSPACE
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 2, 8, 2, 256, 128, 0.1, P(ws) + 4, need, None) == fa.FA_ERR_ALIGN
+    assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 0, 8, 2, 256, 128, 0.1, P(ws), need, None) == fa.FA_OK
+
+
+def test_host_entry_validation(fa):
+    L = fa.lib
+    q = _t(1, 4, 4, 128)
+    P = lambda t: t.data_ptr()
+    need = fa.fa_forward_host_staging_bytes(1, 4, 4, 4, 4, 128)
+    assert need >= 4 * (4 * 4 * 128 * 2)
+    assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_WORKSPACE
+    assert L.fa_forward_host(None, P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_NULL
+    assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 5, None, 0, None) == fa.FA_ERR_UNSUPPORTED
+
+
+def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):
+    # the binding has no fallback: a missing library is an ImportError at import time
+    import importlib.util
+    src = os.path.join(ROOT, "paper_2410_16663_b200", "binding.py")
+    dst = tmp_path / "binding_copy.py"
+    dst.write_text(open(src).read())
+    spec = importlib.util.spec_from_file_location("binding_copy", str(dst))
+    mod = importlib.util.module_from_spec(spec)
+    with pytest.raises(ImportError):
+        spec.loader.exec_module(mod)
+
+
+def test_product_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2410_16663_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "import oracle" not in text and "oracle/" not in text, f

@@ -1,0 +1,305 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI, on seeded inputs.
+
+Small and medium problems are compared element by element against the full oracle; the
+benchmark-size configurations are compared on sampled rows the oracle computes one by one.
+Tolerances: max|dO| <= 2e-3 and max|dLSE| <= 1e-3 (fp16/bf16 inputs, fp32 accumulation).
+With bf16 inputs two format roundings are allowed on top, each bounded exactly from the oracle
+(see tests/util.py): 2^-9 * sum_j P_ij |V_j| for the bf16 probabilities fed to the second MMA,
+and 2^-8 |O| for a stored bf16 output; the fp32-output mode is gated without the latter."""
+import math
+
+import pytest
+import torch
+
+import oracle
+from paper_2410_16663_b200 import inputs as synth
+from tests.util import (TOL_O, TOL_LSE, assert_close_to_oracle, guard_alloc, oracle_rows_for, rel_l2_rows)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def fa():
+    from paper_2410_16663_b200 import binding
+    return binding
+
+
+def check_status(fa):
+    rc, where, blk = fa.fa_device_status()
+    assert rc == 0, f"device status {rc} at {where} block {blk}"
+
+
+def run_forward(fa, q, k, v, causal, scale, o_dtype=None, variant=0):
+    B, Sq, Hq, d = q.shape
+    o, chk_o = guard_alloc((B, Sq, Hq, d), o_dtype or q.dtype, DEV)
+    lse, chk_l = guard_alloc((B, Hq, Sq), torch.float32, DEV)
+    fa.fa_forward_ex(q, k, v, o, lse, causal, scale, variant=variant)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o()
+    chk_l()
+    return o, lse
+
+
+def full_case(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed, variant=0, scale=None):
+    cfg = synth.PrefillConfig("t", B, Hq, Hkv, Sq, Skv, dtype=dtype, causal=causal, seed=seed)
+    q, k, v = synth.prefill_inputs(cfg, "cpu")
+    scale = cfg.scale if scale is None else scale
+    o_ref, l_ref = oracle.attention_full(q, k, v, causal, scale)
+    absv = oracle.attention_full(q, k, v.abs(), causal, scale)[0] if dtype == "bf16" else None
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    what = f"B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {dtype} variant{variant}"
+    o, lse = run_forward(fa, qd, kd, vd, causal, scale, variant=variant)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=what)
+    if dtype == "bf16":  # gate on the accumulator, without the rounding of the stored output
+        o32, lse32 = run_forward(fa, qd, kd, vd, causal, scale, o_dtype=torch.float32, variant=variant)
+        assert_close_to_oracle(o32, lse32, o_ref, l_ref, p_absv=absv, what=what + " fp32-out")
+    return o, lse
+
+
+# ------------------------------------------------------------------ C1: the small benchmark config
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_c1_full_tensor(fa, variant):
+    c = synth.C1
+    q, k, v = synth.prefill_inputs(c, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, c.causal, c.scale)
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), c.causal, c.scale, variant=variant)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what="C1")
+    assert rel_l2_rows(o, o_ref) < 3e-3
+
+
+def test_c1_plain_entry_points_and_determinism(fa):
+    c = synth.C1
+    q, k, v = (t.to(DEV) for t in synth.prefill_inputs(c, "cpu"))
+    outs = []
+    for _ in range(2):
+        o = torch.empty_like(q)
+        lse = torch.empty(c.B, c.Hq, c.Sq, dtype=torch.float32, device=DEV)
+        fa.fa_forward(q, k, v, o, lse, c.causal, c.scale)
+        torch.cuda.synchronize()
+        outs.append((o, lse))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    o_ex, lse_ex = run_forward(fa, q, k, v, c.causal, c.scale)
+    assert torch.equal(outs[0][0], o_ex) and torch.equal(outs[0][1], lse_ex)
+    # lse may be NULL
+    o2 = torch.empty_like(q)
+    fa.fa_forward(q, k, v, o2, None, c.causal, c.scale)
+    torch.cuda.synchronize()
+    assert torch.equal(o2, outs[0][0])
+    check_status(fa)
+
+
+# ------------------------------------------------------------------ shape grid, full oracle
+GRID = [  # (Sq, Skv)
+    (1, 1), (2, 2), (17, 17), (127, 127), (128, 128), (129, 129), (255, 255), (256, 256), (257, 257),
+    (384, 384), (1000, 1000), (1, 129), (17, 1000), (128, 384), (100, 257), (257, 1000),
+]
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", GRID)
+def test_shape_grid_fp16(fa, sq, skv, causal):
+    full_case(fa, 1, 2, 2, sq, skv, causal, "fp16", seed=sq * 1000 + skv)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", [(1, 1), (129, 129), (257, 1000), (384, 384), (1000, 1000)])
+def test_shape_grid_bf16(fa, sq, skv, causal):
+    full_case(fa, 1, 2, 1, sq, skv, causal, "bf16", seed=sq * 1000 + skv + 1)
+
+
+@pytest.mark.parametrize("hq,hkv", [(1, 1), (4, 1), (8, 2), (8, 8), (6, 3)])
+def test_head_grouping(fa, hq, hkv):
+    full_case(fa, 2, hq, hkv, 200, 333, True, "fp16", seed=hq * 10 + hkv)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+def test_alternate_kernels_on_ragged_shapes(fa, variant):
+    full_case(fa, 2, 4, 2, 257, 1000, True, "fp16", seed=77, variant=variant)
+    full_case(fa, 1, 2, 2, 129, 385, False, "bf16", seed=78, variant=variant)
+
+
+def test_scale_zero_and_large_scale(fa):
+    full_case(fa, 1, 2, 2, 130, 260, True, "fp16", seed=5, scale=0.0)
+    full_case(fa, 1, 2, 2, 130, 260, False, "fp16", seed=6, scale=1.0)  # peaked softmax
+
+
+def test_bhsd_strided_layout(fa):
+    cfg = synth.PrefillConfig("t", 2, 4, 2, 300, 300, dtype="fp16", causal=True, seed=9)
+    q, k, v = synth.prefill_inputs(cfg, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
+    # store as [B,H,S,d] and pass [B,S,H,d] views
+    qd = q.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
+    kd = k.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
+    vd = v.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
+    o = torch.empty(2, 4, 300, 128, dtype=torch.float16, device=DEV).permute(0, 2, 1, 3)
+    lse = torch.empty(2, 4, 300, dtype=torch.float32, device=DEV)
+    fa.fa_forward_ex(qd, kd, vd, o, lse, True, cfg.scale)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what="BHSD views")
+
+
+def test_degenerate_sizes(fa):
+    q = torch.randn(2, 5, 2, 128, device=DEV).half()
+    kv0 = torch.empty(2, 0, 2, 128, dtype=torch.float16, device=DEV)
+    o, lse = run_forward(fa, q, kv0, kv0, False, 0.1)       # no keys: O = 0, LSE = -inf
+    assert float(o.abs().max()) == 0.0 and torch.isneginf(lse).all()
+    # B = 0 and Sq = 0 are no-ops that must not touch the outputs
+    o = torch.full((2, 5, 2, 128), 7.0, dtype=torch.float16, device=DEV)
+    k = torch.randn(2, 9, 2, 128, device=DEV).half()
+    assert fa.lib.fa_forward(q.data_ptr(), k.data_ptr(), k.data_ptr(), o.data_ptr(), None, 0, 2, 2, 5, 9, 128,
+                             0, 0.1, None) == 0
+    assert fa.lib.fa_forward(q.data_ptr(), k.data_ptr(), k.data_ptr(), o.data_ptr(), None, 2, 2, 2, 0, 9, 128,
+                             0, 0.1, None) == 0
+    torch.cuda.synchronize()
+    assert float((o - 7.0).abs().max()) == 0.0
+    check_status(fa)
+
+
+def test_closed_form_identical_keys_on_gpu(fa):
+    # all keys equal: O is the running mean of V, LSE = scale*q.k + ln(n)
+    B, H, S = 1, 2, 300
+    g = torch.Generator().manual_seed(3)
+    q = torch.randn(B, S, H, 128, generator=g).half()
+    v = torch.randn(B, S, H, 128, generator=g).half()
+    k = torch.randn(B, 1, H, 128, generator=g).half().expand(B, S, H, 128).contiguous()
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), True, 0.05)
+    want = v.double().cumsum(dim=1) / torch.arange(1, S + 1, dtype=torch.float64).view(1, S, 1, 1)
+    assert float((o.double().cpu() - want).abs().max()) <= TOL_O
+    s = 0.05 * (q.double() * k.double()).sum(-1).permute(0, 2, 1)
+    want_l = s + torch.log(torch.arange(1, S + 1, dtype=torch.float64)).view(1, 1, S)
+    assert float((lse.double().cpu() - want_l).abs().max()) <= TOL_LSE
+
+
+# ------------------------------------------------------------------ benchmark-size configs, sampled rows
+def sampled_case(fa, cfg, n_random, pairs=None):
+    q, k, v = synth.prefill_inputs(cfg, DEV)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=DEV)
+    fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)    # the launch configuration bench.py times
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    rows = synth.sample_rows(cfg, n_random, seed=cfg.seed + 99, pairs=pairs)
+    bf16 = cfg.dtype == "bf16"
+    res = oracle_rows_for(q, k, v, rows, cfg.causal, cfg.scale, with_absv=bf16)
+    o_ref, l_ref, absv = res if bf16 else (res[0], res[1], None)
+    idx = torch.tensor(rows, device=DEV)
+    o_s = o[idx[:, 0], idx[:, 2], idx[:, 1]]
+    l_s = lse[idx[:, 0], idx[:, 1], idx[:, 2]]
+    assert_close_to_oracle(o_s, l_s, o_ref, l_ref, stored_bf16=bf16, p_absv=absv, what=cfg.name)
+    if bf16:
+        # gate on the accumulator through the fp32-output mode
+        o32 = torch.empty(cfg.B, cfg.Sq, cfg.Hq, cfg.d, dtype=torch.float32, device=DEV)
+        fa.fa_forward_ex(q, k, v, o32, lse, cfg.causal, cfg.scale)
+        torch.cuda.synchronize()
+        check_status(fa)
+        assert_close_to_oracle(o32[idx[:, 0], idx[:, 2], idx[:, 1]], lse[idx[:, 0], idx[:, 1], idx[:, 2]],
+                               o_ref, l_ref, p_absv=absv, what=cfg.name + " fp32-out")
+    return len(rows)
+
+
+def test_c2_llama7b_prefill_sampled(fa):
+    assert sampled_case(fa, synth.C2, 48) >= 256
+
+
+@pytest.mark.parametrize("s", [8192, 32768])
+def test_c3_long_context_sampled(fa, s):
+    assert sampled_case(fa, synth.C3[s], 48) >= 256
+
+
+@pytest.mark.parametrize("s", [131072, 262144])
+def test_c3_very_long_context_sampled(fa, s):
+    cfg = synth.C3[s]
+    assert sampled_case(fa, cfg, 20, pairs=[(0, 0), (0, 13), (0, 31)]) >= 64
+
+
+def test_c4_gqa_sampled(fa):
+    assert sampled_case(fa, synth.C4, 48) >= 256
+    assert sampled_case(fa, synth.C4_NC, 48) >= 256
+
+
+# ------------------------------------------------------------------ decode
+def run_decode(fa, q, k, v, seqlens_dev, scale):
+    B, _, Hq, d = q.shape
+    Smax, Hkv = k.shape[1], k.shape[2]
+    o, chk_o = guard_alloc((B, 1, Hq, d), torch.float16, DEV)
+    lse, chk_l = guard_alloc((B, Hq), torch.float32, DEV)
+    nbytes = fa.fa_decode_workspace_bytes(B, Hq, Hkv, Smax, d)
+    ws, chk_w = guard_alloc((max(nbytes // 4, 4),), torch.float32, DEV)
+    fa.fa_decode(q, k, v, o, lse, seqlens_dev, scale, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    return o, lse
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (8, 2), (8, 1), (6, 2), (16, 1)])
+def test_decode_small_full(fa, hq, hkv):
+    cfg = synth.DecodeConfig("t", 5, hq, hkv, 1500, 1, 1500, seed=hq * 31 + hkv)
+    q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=True)
+    sl[0], sl[1], sl[2] = 1500, 0, 1          # full, empty, single key
+    for b in range(cfg.B):                     # re-poison after editing the lengths
+        n = int(sl[b])
+        k[b, n:] = float("nan"); v[b, n:] = float("nan")
+        if n and torch.isnan(k[b, :n].float()).any():
+            g = torch.Generator().manual_seed(b)
+            k[b, :n] = torch.randn(n, hkv, 128, generator=g).half()
+            v[b, :n] = torch.randn(n, hkv, 128, generator=g).half()
+    o_ref, l_ref = oracle.decode(q, k, v, sl, cfg.scale)
+    o, lse = run_decode(fa, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), cfg.scale)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what=f"decode {hq}/{hkv}")
+    assert float(o[1].abs().max()) == 0.0 and torch.isneginf(lse[1]).all()
+
+
+def test_decode_chunked_lengths_and_clamping(fa):
+    # lengths on both sides of chunk and tile boundaries; a length beyond Smax is clamped
+    cfg = synth.DecodeConfig("t", 8, 8, 8, 4096, 1, 4096, seed=321)
+    q, k, v, _ = synth.decode_inputs(cfg, "cpu", poison=False)
+    sl = torch.tensor([127, 128, 129, 255, 256, 257, 4096, 99999], dtype=torch.int32)
+    o_ref, l_ref = oracle.decode(q, k, v, sl.clamp(max=4096), cfg.scale)
+    o, lse = run_decode(fa, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), cfg.scale)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what="decode boundaries")
+    o2, lse2 = run_decode(fa, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), cfg.scale)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)      # bit-reproducible
+
+
+@pytest.mark.parametrize("cfg", [synth.C5_MHA, synth.C5_GQA], ids=["mha", "gqa"])
+def test_c5_decode_full_size_sampled(fa, cfg):
+    q, k, v, sl = synth.decode_inputs(cfg, DEV, poison=True)
+    o, lse = run_decode(fa, q, k, v, sl.to(DEV), cfg.scale)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    g = cfg.Hq // cfg.Hkv
+    gen = torch.Generator().manual_seed(cfg.seed + 5)
+    order = torch.argsort(sl)
+    seqs = {int(order[0]), int(order[-1]), 0, cfg.B - 1}
+    seqs.update(int(x) for x in torch.randint(0, cfg.B, (6,), generator=gen))
+    for b in sorted(seqs):
+        n = int(sl[b])
+        heads = {0, g - 1, cfg.Hq - 1, int(torch.randint(0, cfg.Hq, (1,), generator=gen))}
+        for h in sorted(heads):
+            hk = h // g
+            qs = q[b:b + 1, :, h:h + 1].cpu()
+            ks = k[b:b + 1, :n, hk:hk + 1].contiguous().cpu()
+            vs = v[b:b + 1, :n, hk:hk + 1].contiguous().cpu()
+            o_ref, l_ref = oracle.decode(qs, ks, vs, [n], cfg.scale)
+            assert_close_to_oracle(o[b, 0, h].view(1, 1, -1), lse[b, h].view(1, 1), o_ref, l_ref,
+                                   what=f"{cfg.name} b{b} h{h} n{n}")
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+def test_forward_host_entry(fa):
+    c = synth.C1
+    q, k, v = (t.pin_memory() for t in synth.prefill_inputs(c, "cpu"))
+    o = torch.empty_like(q).pin_memory()
+    lse = torch.empty(c.B, c.Hq, c.Sq, dtype=torch.float32).pin_memory()
+    n = fa.fa_forward_host_staging_bytes(c.B, c.Hq, c.Hkv, c.Sq, c.Skv, c.d)
+    st = torch.empty(n + 1024, dtype=torch.uint8, device=DEV)
+    off = (-st.data_ptr()) % 1024
+    fa.fa_forward_host(q, k, v, o, lse, c.causal, c.scale, st[off:off + n])
+    torch.cuda.synchronize()
+    check_status(fa)
+    o_ref, l_ref = oracle.attention_full(q, k, v, c.causal, c.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what="host entry")

@@ -1,0 +1,91 @@
+"""Shared helpers for the parity tests: run the CUDA library on seeded inputs and compare with
+the CPU oracle element by element."""
+import math
+
+import torch
+
+import oracle
+
+TOL_O = 2e-3      # max |dO| for fp16/bf16 inputs with fp32 accumulation
+TOL_LSE = 1e-3    # max |dLSE|
+BF16_ULP = 2.0 ** -8  # half-ulp relative spacing of bfloat16 rounding of the stored output
+
+
+def guard_alloc(shape, dtype, device, pad=1024):
+    """A tensor inside a larger allocation whose margins hold NaN; returns (view, check)."""
+    n = 1
+    for s in shape:
+        n *= s
+    flat = torch.full((n + 2 * pad,), float("nan"), dtype=dtype, device=device)
+    view = flat[pad:pad + n].view(*shape)
+
+    def check():
+        assert torch.isnan(flat[:pad]).all() and torch.isnan(flat[pad + n:]).all(), "guard band overwritten"
+
+    return view, check
+
+
+def assert_close_to_oracle(o_gpu, lse_gpu, o_ref, lse_ref, stored_bf16=False, p_absv=None, what=""):
+    """o_ref/lse_ref are fp64 oracle results with the same shapes as the GPU tensors.
+
+    The gate is max|dO| <= 2e-3.  Two roundings that the 16-bit formats impose are allowed on
+    top of it, each with its exact bound computed from the oracle:
+      * p_absv (bf16 inputs): the second MMA takes P in the inputs' 16-bit type, so with bf16
+        each probability carries a relative rounding of up to 2^-9, which moves O_i by at most
+        2^-9 * sum_j P_ij |V_j|; p_absv is that softmax-weighted mean of |V| from the oracle.
+      * stored_bf16: the stored bf16 output is rounded by up to 2^-8 |O|.
+    """
+    o = o_gpu.detach().double().cpu()
+    l = lse_gpu.detach().double().cpu()
+    assert torch.isfinite(o).all(), f"{what}: non-finite O"
+    diff = (o - o_ref).abs()
+    allow = torch.zeros_like(diff)
+    if p_absv is not None:
+        allow = allow + (2.0 ** -9) * p_absv
+    if stored_bf16:
+        allow = allow + BF16_ULP * o_ref.abs()
+    excess = diff - allow
+    assert float(excess.max()) <= TOL_O, f"{what}: max(|dO| - allowance) = {float(excess.max()):.3e}"
+    both_ninf = torch.isneginf(l) & torch.isneginf(lse_ref)
+    dl = torch.where(both_ninf, torch.zeros_like(l), (l - lse_ref).abs())
+    assert not torch.isnan(dl).any(), f"{what}: NaN in LSE comparison"
+    assert float(dl.max()) <= TOL_LSE, f"{what}: max|dLSE| = {float(dl.max()):.3e}"
+    return float(diff.max()), float(dl.max())
+
+
+def rel_l2_rows(o_gpu, o_ref):
+    o = o_gpu.detach().double().cpu()
+    num = (o - o_ref).norm(dim=-1)
+    den = o_ref.norm(dim=-1).clamp_min(1e-30)
+    return float((num / den).max())
+
+
+def oracle_rows_for(q, k, v, rows, causal, scale, with_absv=False):
+    """Row-sampled oracle on device tensors: copies only the (b, kv-head) slices the rows need.
+    With with_absv also returns sum_j P_ij |V_j| for the same rows (see assert_close_to_oracle)."""
+    B, Sq, Hq, d = q.shape
+    Hkv = k.shape[2]
+    g = Hq // Hkv
+    out_o = torch.zeros(len(rows), d, dtype=torch.float64)
+    out_l = torch.zeros(len(rows), dtype=torch.float64)
+    out_a = torch.zeros(len(rows), d, dtype=torch.float64) if with_absv else None
+    groups = {}
+    for n, (b, h, i) in enumerate(rows):
+        groups.setdefault((b, h), []).append((n, i))
+    for (b, h), items in groups.items():
+        hk = h // g
+        qs = q[b:b + 1, :, h:h + 1].contiguous().cpu()
+        ks = k[b:b + 1, :, hk:hk + 1].contiguous().cpu()
+        vs = v[b:b + 1, :, hk:hk + 1].contiguous().cpu()
+        r = [(0, 0, i) for (_, i) in items]
+        o, l = oracle.attention_rows(qs, ks, vs, causal, scale, r)
+        if with_absv:
+            a, _ = oracle.attention_rows(qs, ks, vs.abs(), causal, scale, r)
+        for j, (n, _) in enumerate(items):
+            out_o[n] = o[j]
+            out_l[n] = l[j]
+            if with_absv:
+                out_a[n] = a[j]
+    if with_absv:
+        return out_o, out_l, out_a
+    return out_o, out_l
