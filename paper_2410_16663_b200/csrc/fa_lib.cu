@@ -10,6 +10,7 @@
 #include <string.h>
 
 #include "decode.cuh"
+#include "prefill_pipelined.cuh"
 #include "prefill_simple.cuh"
 
 namespace {
@@ -176,7 +177,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (rc) return rc;
 
     switch (p.variant) {
-        case 0:
+        case 0:  // pipelined, warp-specialised kernel
+            return bf16 ? fa::launch_pipelined<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
+                        : fa::launch_pipelined<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
         case 1:  // simple kernel, P handed over through tensor memory
             return bf16 ? launch_simple<__nv_bfloat16, true>(tq, tk, tv, fp, st)
                         : launch_simple<__half, true>(tq, tk, tv, fp, st);

@@ -202,12 +202,12 @@ def sampled_case(fa, cfg, n_random, pairs=None):
 
 
 def test_c2_llama7b_prefill_sampled(fa):
-    assert sampled_case(fa, synth.C2, 48) >= 256
+    assert sampled_case(fa, synth.C2, 80) >= 256
 
 
 @pytest.mark.parametrize("s", [8192, 32768])
 def test_c3_long_context_sampled(fa, s):
-    assert sampled_case(fa, synth.C3[s], 48) >= 256
+    assert sampled_case(fa, synth.C3[s], 80) >= 256
 
 
 @pytest.mark.parametrize("s", [131072, 262144])
@@ -217,8 +217,8 @@ def test_c3_very_long_context_sampled(fa, s):
 
 
 def test_c4_gqa_sampled(fa):
-    assert sampled_case(fa, synth.C4, 48) >= 256
-    assert sampled_case(fa, synth.C4_NC, 48) >= 256
+    assert sampled_case(fa, synth.C4, 64) >= 256
+    assert sampled_case(fa, synth.C4_NC, 64) >= 256
 
 
 # ------------------------------------------------------------------ decode
