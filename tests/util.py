@@ -25,7 +25,8 @@ def guard_alloc(shape, dtype, device, pad=1024):
     return view, check
 
 
-def assert_close_to_oracle(o_gpu, lse_gpu, o_ref, lse_ref, stored_bf16=False, p_absv=None, what=""):
+def assert_close_to_oracle(o_gpu, lse_gpu, o_ref, lse_ref, stored_bf16=False, p_absv=None, what="",
+                           stored_fp16_ulp=False):
     """o_ref/lse_ref are fp64 oracle results with the same shapes as the GPU tensors.
 
     The gate is max|dO| <= 2e-3.  Two roundings that the 16-bit formats impose are allowed on
@@ -34,6 +35,9 @@ def assert_close_to_oracle(o_gpu, lse_gpu, o_ref, lse_ref, stored_bf16=False, p_
         each probability carries a relative rounding of up to 2^-9, which moves O_i by at most
         2^-9 * sum_j P_ij |V_j|; p_absv is that softmax-weighted mean of |V| from the oracle.
       * stored_bf16: the stored bf16 output is rounded by up to 2^-8 |O|.
+      * stored_fp16_ulp: only for the peaked-softmax stress case, where |O| reaches 4 and the
+        fp16 output rounding alone (2^-11 |O|) reaches the gate; the benchmark configurations
+        are gated without it.
     """
     o = o_gpu.detach().double().cpu()
     l = lse_gpu.detach().double().cpu()
@@ -44,6 +48,8 @@ def assert_close_to_oracle(o_gpu, lse_gpu, o_ref, lse_ref, stored_bf16=False, p_
         allow = allow + (2.0 ** -9) * p_absv
     if stored_bf16:
         allow = allow + BF16_ULP * o_ref.abs()
+    if stored_fp16_ulp:
+        allow = allow + (2.0 ** -11) * o_ref.abs()
     excess = diff - allow
     assert float(excess.max()) <= TOL_O, f"{what}: max(|dO| - allowance) = {float(excess.max()):.3e}"
     both_ninf = torch.isneginf(l) & torch.isneginf(lse_ref)
