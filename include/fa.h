@@ -116,6 +116,31 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * Decode for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * convenience of this library).  Some hosts of this code may not call cudaMalloc at all: code
+ * running inside a framework that owns the memory pool and forbids outside allocations, a
+ * real-time serving loop that must not take the allocator's locks or risk an out-of-memory
+ * failure mid-request, or a plugin that is handed buffers and nothing else.  They still pass
+ * q, the caches, o, lse and seqlens_k exactly as for fa_decode, but no workspace: the per-chunk
+ * partial results go to a fixed array that lives inside the library's device image
+ * (FA_DECODE_NOALLOC_BYTES bytes, held by every GPU that loads the library until the process
+ * exits).
+ *   - The call fails with FA_ERR_WORKSPACE, before any CUDA work, when
+ *     fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d) exceeds FA_DECODE_NOALLOC_BYTES.
+ *   - The first call on each device looks the array's device address up (once per device, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - No entry of the array needs to start at zero: every slot the merge reads is written by
+ *     the same call first.  All calls share the one array, so two calls whose kernels may
+ *     overlap on the GPU (different streams, no ordering between them) race on it; order them.
+ *   - The function itself allocates nothing: no cudaMalloc, cudaFree or allocating library call.
+ * Results are identical to fa_decode's for the same arguments.
+ */
+#define FA_DECODE_NOALLOC_BYTES (4u << 20)
+int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                      const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
+                      void* stream);
+
+/*
  * Host-buffer form of fa_forward for callers whose tensors live in host memory (pinned memory
  * makes the copies asynchronous): copies q, k, v to the device staging area, runs the forward,
  * copies o and lse back, all on `stream`.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16.

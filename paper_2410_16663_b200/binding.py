@@ -45,6 +45,8 @@ lib.fa_decode.restype = _i
 lib.fa_decode.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_workspace_bytes.restype = _sz
 lib.fa_decode_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
+lib.fa_decode_noalloc.restype = _i
+lib.fa_decode_noalloc.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _p]
 lib.fa_forward_host.restype = _i
 lib.fa_forward_host.argtypes = [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p, _sz, _p]
 lib.fa_forward_host_staging_bytes.restype = _sz
@@ -56,7 +58,10 @@ lib.fa_strerror.argtypes = [_i]
 lib.fa_version.restype = _i
 lib.fa_last_cuda_error.restype = _i
 
+FA_DECODE_NOALLOC_BYTES = 4 << 20
+
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
+           "fa_decode_noalloc",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -137,6 +142,18 @@ def fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace,
     rc = lib.fa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq,
                        Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode", raise_on_error)
+
+
+def fa_decode_noalloc(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, raise_on_error: bool = True) -> int:
+    """``fa_decode_noalloc``: decode for callers that may not allocate device memory.  Same
+    arguments as ``fa_decode`` minus the workspace; the partial results live in a fixed
+    ``FA_DECODE_NOALLOC_BYTES`` array inside the library, shared by all calls (do not overlap
+    two calls on the GPU).  Problems whose partials do not fit are refused with FA_ERR_WORKSPACE."""
+    B, _, Hq, d = q.shape
+    _, Smax, Hkv, _ = k_cache.shape
+    rc = lib.fa_decode_noalloc(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B,
+                               Hq, Hkv, Smax, d, float(scale), _stream())
+    return _check(rc, "fa_decode_noalloc", raise_on_error)
 
 
 def fa_forward_host_staging_bytes(B, Hq, Hkv, Sq, Skv, d) -> int:

@@ -302,6 +302,42 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
+// ---- decode without a caller workspace -------------------------------------------------------
+// Scratch for the per-chunk partials of fa_decode_noalloc.  It is part of the device image, so
+// every GPU that loads the library holds it until exit.  In host code the name below is only a
+// host-side stand-in for the device array; the device address is looked up once per device.
+static __device__ __align__(256) unsigned char g_decode_scratch[FA_DECODE_NOALLOC_BYTES];
+
+int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                      const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
+                      void* stream) {
+    // sizes first: nothing CUDA-related happens for a problem the fixed scratch cannot hold
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d) > (size_t)FA_DECODE_NOALLOC_BYTES)
+        return FA_ERR_WORKSPACE;
+    if (B == 0) return FA_OK;
+    constexpr int kMaxDevices = 64;
+    static void* scratch_of_device[kMaxDevices] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return FA_ERR_DEVICE;
+    void* scratch = __atomic_load_n(&scratch_of_device[dev], __ATOMIC_ACQUIRE);
+    if (!scratch) {
+        // set-up, once per device, with that device current (it is: we just asked which one)
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_decode_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!ptr) return FA_ERR_DEVICE;
+        __atomic_store_n(&scratch_of_device[dev], ptr, __ATOMIC_RELEASE);  // same value from any thread
+        scratch = ptr;
+    }
+    return fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, scratch,
+                     (size_t)FA_DECODE_NOALLOC_BYTES, stream);
+}
+
 size_t fa_forward_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int d) {
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv < 0 || d != 128) return 0;
     auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
