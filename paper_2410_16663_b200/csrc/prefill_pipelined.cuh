@@ -68,15 +68,22 @@ template <typename T, bool kMasked>
 __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, uint32_t tO, float scale_log2,
                                              int lim, bool first, float& m_ref, float& l_run) {
     // row max over the visible columns
-    float mx = -INFINITY;
+    float mx;
+    if (kMasked) {
+        mx = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 128; ++i) {
-        const float v = __uint_as_float(s[i]);
-        if (kMasked) {
-            if (i < lim) mx = fmaxf(mx, v);
-        } else {
-            mx = fmaxf(mx, v);
+        for (int i = 0; i < 128; ++i)
+            if (i < lim) mx = fmaxf(mx, __uint_as_float(s[i]));
+    } else {
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 8) {
+            m0 = max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+            m1 = max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+            m2 = max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+            m3 = max3(m3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
         }
+        mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     }
     // lazy reference update: move the reference max only when the row max outgrew it by more
     // than the threshold; O and l then carry the same (stale) reference, so O / l is exact
@@ -102,30 +109,53 @@ __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, ui
     l_run *= alpha;
     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
     const float neg_ms = -m_use * scale_log2;
-    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+    if (kMasked) {
+        float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
+        for (int c = 0; c < 4; ++c) {
+            uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            const int e = c * 32 + i;
-            float p0 = fast_exp2(fmaf(__uint_as_float(s[e]), scale_log2, neg_ms));
-            float p1 = fast_exp2(fmaf(__uint_as_float(s[e + 1]), scale_log2, neg_ms));
-            float p2 = fast_exp2(fmaf(__uint_as_float(s[e + 2]), scale_log2, neg_ms));
-            float p3 = fast_exp2(fmaf(__uint_as_float(s[e + 3]), scale_log2, neg_ms));
-            if (kMasked) {  // exact zeros whatever the scale
-                p0 = (e < lim) ? p0 : 0.f;
+            for (int i = 0; i < 32; i += 2) {
+                const int e = c * 32 + i;
+                float p0 = fast_exp2(fmaf(__uint_as_float(s[e]), scale_log2, neg_ms));
+                float p1 = fast_exp2(fmaf(__uint_as_float(s[e + 1]), scale_log2, neg_ms));
+                p0 = (e < lim) ? p0 : 0.f;  // exact zeros whatever the scale
                 p1 = (e + 1 < lim) ? p1 : 0.f;
-                p2 = (e + 2 < lim) ? p2 : 0.f;
-                p3 = (e + 3 < lim) ? p3 : 0.f;
+                l0 += p0;
+                l1 += p1;
+                pk[i / 2] = pack2<T>(p0, p1);
             }
-            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-            pk[i / 2] = pack2<T>(p0, p1);
-            pk[i / 2 + 1] = pack2<T>(p2, p3);
+            tmem_st_x16(tS + c * 16, pk);
         }
-        tmem_st_x16(tS + c * 16, pk);
+        l_run += l0 + l1;
+    } else {
+        // packed f32x2 arithmetic: one FMA and one add per pair of columns
+        const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
+        uint64_t la = f2_pack(0.f, 0.f), lb = la;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                const int e = c * 32 + i;
+                const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), sc2, nm2);
+                const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[e + 2]), __uint_as_float(s[e + 3])), sc2, nm2);
+                float x0, x1, x2, x3;
+                f2_unpack(x01, x0, x1);
+                f2_unpack(x23, x2, x3);
+                const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                la = f2_add(la, f2_pack(p0, p1));
+                lb = f2_add(lb, f2_pack(p2, p3));
+                pk[i / 2] = pack2<T>(p0, p1);
+                pk[i / 2 + 1] = pack2<T>(p2, p3);
+            }
+            tmem_st_x16(tS + c * 16, pk);
+        }
+        float a0, a1, b0, b1;
+        f2_unpack(la, a0, a1);
+        f2_unpack(lb, b0, b1);
+        l_run += (a0 + a1) + (b0 + b1);
     }
-    l_run += (l0 + l1) + (l2 + l3);
 }
 
 template <typename T>
@@ -175,6 +205,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
     if (warp < 8) {
         // ================================================================ softmax + epilogue
+        setmaxnreg_inc<224>();  // a whole row of S lives in registers
         const int t = warp >> 2;                    // query tile of this warpgroup
         const int r_in_tile = tid & 127;
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -259,7 +290,10 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             // p_full arrival, i.e. after these reads of O
             tc_fence_before();
         }
-    } else if (warp == 8) {
+    } else {
+        setmaxnreg_dec<56>();
+    }
+    if (warp == 8) {
         // ================================================================ MMA issue
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc_f16(kBf16, 128, 128, false, false);
