@@ -54,11 +54,11 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int idx, int n_q
     // a second tile that starts past the last row still runs (on zero-filled rows, never
     // stored) so that both roles always have work in every item
     const int n_hi = (q_lo + kTile < p.Sq) ? kv_tiles_for(q_lo + kTile, kTile, p.Sq, p.Skv, p.causal) : n_lo;
-    const int r_lo = lead ? 1 : 0;  // role that takes the lower (shorter) tile
-    it.q0[r_lo] = q_lo;
-    it.n[r_lo] = n_lo;
-    it.q0[1 - r_lo] = q_lo + kTile;
-    it.n[1 - r_lo] = n_hi;
+    const bool swap = lead != 0;  // role 0 takes the upper (longer) tile when it is a step ahead
+    it.q0[0] = swap ? q_lo + kTile : q_lo;
+    it.n[0] = swap ? n_hi : n_lo;
+    it.q0[1] = swap ? q_lo : q_lo + kTile;
+    it.n[1] = swap ? n_lo : n_hi;
     lead += lead ? -(n_hi - n_lo) : (n_hi - n_lo);
     return it;
 }
@@ -158,6 +158,177 @@ __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, ui
     }
 }
 
+// ---- barrier addresses (shared by all roles): byte offsets from the first barrier
+__device__ __forceinline__ uint32_t bar_q_full(uint32_t b0, int t) { return b0 + 8 * t; }
+__device__ __forceinline__ uint32_t bar_q_empty(uint32_t b0, int t) { return b0 + 8 * (2 + t); }
+__device__ __forceinline__ uint32_t bar_kv_full(uint32_t b0, uint32_t s) { return b0 + 8 * (4 + s); }
+__device__ __forceinline__ uint32_t bar_kv_empty(uint32_t b0, uint32_t s) { return b0 + 8 * (4 + kStages + s); }
+__device__ __forceinline__ uint32_t bar_s_full(uint32_t b0, int t) { return b0 + 8 * (4 + 2 * kStages + t); }
+__device__ __forceinline__ uint32_t bar_p_full(uint32_t b0, int t) { return b0 + 8 * (6 + 2 * kStages + t); }
+__device__ __forceinline__ uint32_t bar_o_final(uint32_t b0, int t) { return b0 + 8 * (8 + 2 * kStages + t); }
+__device__ __forceinline__ uint32_t bar_turn(uint32_t b0, int t) { return b0 + 8 * (10 + 2 * kStages + t); }
+constexpr int kNumBars = 12 + 2 * kStages;
+
+// High word shared by every shared-memory operand descriptor used here: SBO = 1024 bytes,
+// version 1, 128-byte swizzle.  The low word carries the address and the leading offset, so a
+// k-step only adds a constant to it.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3ffffu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+
+// The single thread that issues every tcgen05.mma of the CTA.  It keeps one cursor per tile
+// role; a round is: wait for the role's P, issue its O += P V, then issue S for the role's
+// next step (possibly of the next item).  All state lives in registers.
+template <typename T>
+struct MmaIssuer {
+    uint32_t bar0, sQ, sKV, tmem;
+    volatile uint32_t* abort_flag;
+
+    struct Cursor {
+        int idx, ord, lead;   // work item, its ordinal in this CTA's sequence, role-assignment replay
+        int j, n, n_other;    // step, steps of this role's tile, steps of the other role's tile
+        uint32_t slot, par;   // ring slot / parity of this step's K entry (V is the next entry)
+        bool valid;
+    };
+    static constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    static constexpr uint32_t kIdescQK = instr_desc_f16(kBf16, 128, 128, false, false);
+    static constexpr uint32_t kIdescPV = instr_desc_f16(kBf16, 128, 128, false, true);
+
+    __device__ __forceinline__ static void ring_add(uint32_t& slot, uint32_t& par, uint32_t k) {
+        slot += k;  // k < kStages
+        if (slot >= kStages) {
+            slot -= kStages;
+            par ^= 1;
+        }
+    }
+    template <int t>
+    __device__ __forceinline__ void load_item(Cursor& c, const FwdParams& p, int total_items, int n_qpairs) {
+        c.valid = c.idx < total_items;
+        if (c.valid) {
+            const Item it = decode_item(p, c.idx, n_qpairs, c.lead);
+            c.n = it.n[t];
+            c.n_other = it.n[1 - t];
+            c.j = 0;
+        }
+    }
+    // S = Q K^T for the step the cursor points at (operands already waited for)
+    template <int t>
+    __device__ __forceinline__ void mma_s(const Cursor& c) {
+        const uint32_t a_lo = desc_lo(sQ + t * kTileBytes, 16);
+        const uint32_t b_lo = desc_lo(sKV + c.slot * kTileBytes, 16);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t koff = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+            mma_ss_lo(tmem + t * 128, a_lo + koff, b_lo + koff, kIdescQK, ks > 0 ? 1u : 0u);
+        }
+        mma_commit(bar_s_full(bar0, t));
+    }
+    // Commits that only free resources; they go after the turn has been handed over.
+    // A ring slot is free once both roles' MMAs on it are done: each reader commits one arrival,
+    // and the only reader of an entry the other role never visits commits both.
+    template <int t>
+    __device__ __forceinline__ void release_s(const Cursor& c) {
+        mma_commit(bar_kv_empty(bar0, c.slot));
+        if (c.j >= c.n_other) mma_commit(bar_kv_empty(bar0, c.slot));
+        if (c.j == c.n - 1) mma_commit(bar_q_empty(bar0, t));  // Q of this item is no longer needed
+    }
+    template <int t>
+    __device__ __forceinline__ bool wait_s_operands(const Cursor& c) {
+        if (c.j == 0 && !mbar_wait(bar_q_full(bar0, t), c.ord & 1, abort_flag, 30 + t)) return false;
+        return mbar_wait(bar_kv_full(bar0, c.slot), c.par, abort_flag, 32 + t);
+    }
+    // One round of a role: O += P V for the current step, then S for the next step (possibly of
+    // the next item).  Everything that can be waited for in advance is waited for before the
+    // role takes its turn on the tensor core; the turn passes to the other role right after the
+    // MMAs and the S commit, so the two roles' MMA batches alternate back to back while each
+    // role's bookkeeping overlaps the other's batch.
+    template <int t>
+    __device__ __forceinline__ bool round(Cursor& c, uint32_t& ph_p, uint32_t& turn_k, const FwdParams& p,
+                                          int total_items, int n_qpairs) {
+        uint32_t v_slot = c.slot, v_par = c.par;
+        ring_add(v_slot, v_par, 1);
+        if (!mbar_wait(bar_kv_full(bar0, v_slot), v_par, abort_flag, 34 + t)) return false;
+        Cursor nx = c;  // the role's next step
+        ring_add(nx.slot, nx.par, 2);
+        if (++nx.j == nx.n) {  // next item: skip the entries only the other role reads
+            if (nx.n_other > nx.n) ring_add(nx.slot, nx.par, 2);
+            nx.idx += gridDim.x;
+            nx.ord += 1;
+            load_item<t>(nx, p, total_items, n_qpairs);
+        }
+        if (nx.valid && !wait_s_operands<t>(nx)) return false;
+        if (!mbar_wait(bar_p_full(bar0, t), ph_p, abort_flag, 36 + t)) return false;
+        ph_p ^= 1;
+        if (!mbar_wait(bar_turn(bar0, t), (turn_k & 1) ^ (t == 0 ? 1u : 0u), abort_flag, 38 + t)) return false;
+        ++turn_k;
+        tc_fence_after();
+        const uint32_t b_lo = desc_lo(sKV + v_slot * kTileBytes, kHalfBytes);  // V: N-major, 16 kv rows per step
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+            mma_ts_lo(tmem + 256 + t * 128, tmem + t * 128 + ks * 8, b_lo + ks * (2048 >> 4), kIdescPV,
+                      (ks > 0) ? 1u : (c.j > 0 ? 1u : 0u));
+        if (nx.valid) mma_s<t>(nx);
+        mbar_arrive(bar_turn(bar0, 1 - t));
+        // bookkeeping, off the other role's critical path
+        mma_commit(bar_kv_empty(bar0, v_slot));
+        if (c.j >= c.n_other) mma_commit(bar_kv_empty(bar0, v_slot));
+        if (c.j == c.n - 1) mma_commit(bar_o_final(bar0, t));
+        if (nx.valid) release_s<t>(nx);
+        c = nx;
+        return true;
+    }
+    // One issuing thread per role (they sit in different warps).  MMAs of one thread execute in
+    // issue order, which is all the P/S aliasing needs; the two roles share the K/V ring and
+    // the turn tokens.  Role 0 never has more rounds than role 1 and at most one fewer, so one
+    // empty turn at its end keeps the token moving for role 1's last round.
+    template <int t>
+    __device__ __forceinline__ void run(const FwdParams& p, int total_items, int n_qpairs) {
+        Cursor c;
+        c.idx = blockIdx.x;
+        c.ord = 0;
+        c.lead = 0;
+        c.slot = 0;
+        c.par = 0;
+        load_item<t>(c, p, total_items, n_qpairs);
+        uint32_t ph = 0, turn_k = 0;
+        bool ok = true;
+        if (c.valid) {
+            ok = wait_s_operands<t>(c);
+            if (ok) {
+                tc_fence_after();
+                mma_s<t>(c);
+                release_s<t>(c);
+            }
+        }
+        while (ok && c.valid) ok = round<t>(c, ph, turn_k, p, total_items, n_qpairs);
+        if (t == 0 && ok) {
+            if (mbar_wait(bar_turn(bar0, 0), (turn_k & 1) ^ 1u, abort_flag, 40)) mbar_arrive(bar_turn(bar0, 1));
+        }
+    }
+};
+
 template <typename T>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -167,7 +338,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;                      // 2 tiles
     const uint32_t sKV = smem_base + 2 * kTileBytes;    // kStages tiles
-    __shared__ __align__(8) uint64_t bars[4 + 2 * kStages + 6];
+    __shared__ __align__(8) uint64_t bars[kNumBars];
     __shared__ uint32_t tmem_holder;
     __shared__ volatile uint32_t abort_flag;
 
@@ -185,9 +356,11 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const int lane = tid & 31;
 
     if (tid == 0) {
-        for (int i = 0; i < 4 + 2 * kStages + 6; ++i) {
+        for (int i = 0; i < kNumBars; ++i) {
             const bool is_p_full = (i == 6 + 2 * kStages) || (i == 7 + 2 * kStages);
-            mbar_init(bar0 + 8 * i, is_p_full ? 4 : 1);  // p_full: one arrival per softmax warp
+            const bool is_kv_empty = (i >= 4 + kStages) && (i < 4 + 2 * kStages);
+            // p_full: one arrival per softmax warp; kv_empty: one per reading role
+            mbar_init(bar0 + 8 * i, is_p_full ? 4 : (is_kv_empty ? 2 : 1));
         }
         abort_flag = 0;
         fence_mbar_init();
@@ -201,7 +374,6 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = tmem_holder;
     const int off = p.Skv - p.Sq;
-    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
 
     if (warp < 8) {
         // ================================================================ softmax + epilogue
@@ -293,95 +465,17 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     } else {
         setmaxnreg_dec<56>();
     }
-    if (warp == 8) {
-        // ================================================================ MMA issue
+    if (warp == 8 || warp == 10) {
+        // ================================================================ MMA issue (role 0 / 1)
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc_f16(kBf16, 128, 128, false, false);
-            constexpr uint32_t idesc_pv = instr_desc_f16(kBf16, 128, 128, false, true);
-            struct Cursor {
-                int idx;       // work item index (global)
-                int ord;       // ordinal of the item in this CTA's sequence
-                int lead;      // this cursor's replay of the role assignment
-                int j, n;      // step within the item, steps of this role's tile
-                int n_other;   // steps of the other role's tile in the same item
-                uint32_t base; // ring index of the item's K_0
-                bool valid;
-            } cur[2];
-            bool ok = true;
-            auto load_item = [&](Cursor& c, int t) {
-                c.valid = c.idx < total_items;
-                if (c.valid) {
-                    const Item it = decode_item(p, c.idx, n_qpairs, c.lead);
-                    c.n = it.n[t];
-                    c.n_other = it.n[1 - t];
-                    c.j = 0;
-                }
-            };
-            for (int t = 0; t < 2; ++t) {
-                cur[t].idx = blockIdx.x;
-                cur[t].ord = 0;
-                cur[t].lead = 0;
-                cur[t].base = 0;
-                load_item(cur[t], t);
-            }
-            uint32_t ph_p[2] = {0, 0};
-            auto issue_s = [&](int t) {
-                Cursor& c = cur[t];
-                if (c.j == 0) ok = ok && mbar_wait(q_full(t), c.ord & 1, &abort_flag, 30 + t);
-                const uint32_t g = c.base + 2 * c.j;
-                const uint32_t slot = g % kStages;
-                ok = ok && mbar_wait(kv_full(slot), (g / kStages) & 1, &abort_flag, 32 + t);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t a0 = sQ + t * kTileBytes, b0 = sKV + slot * kTileBytes;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    mma_ss(tmem_base + t * 128, smem_desc_sw128(a0 + koff, 16, 1024),
-                           smem_desc_sw128(b0 + koff, 16, 1024), idesc_qk, ks > 0);
-                }
-                mma_commit(s_full(t));
-                // role 1 trails role 0 in ring order, so it is the last reader of every entry it
-                // reads; role 0 frees the entries role 1 never reads
-                if (t == 1 || c.j >= c.n_other) mma_commit(kv_empty(slot));
-                if (c.j == c.n - 1) mma_commit(q_empty(t));     // Q_t of this item is no longer needed
-            };
-            auto issue_pv = [&](int t) {
-                Cursor& c = cur[t];
-                const uint32_t g = c.base + 2 * c.j + 1;
-                const uint32_t slot = g % kStages;
-                ok = ok && mbar_wait(kv_full(slot), (g / kStages) & 1, &abort_flag, 34 + t);
-                if (!ok) return;
-                tc_fence_after();
-                const uint32_t b0 = sKV + slot * kTileBytes;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8,
-                           smem_desc_sw128(b0 + ks * 2048, kHalfBytes, 1024), idesc_pv, (c.j > 0) || (ks > 0));
-                if (t == 1 || c.j >= c.n_other) mma_commit(kv_empty(slot));
-                if (c.j == c.n - 1) mma_commit(o_final(t));
-            };
-            if (cur[0].valid) issue_s(0);
-            if (cur[1].valid) issue_s(1);
-            while (ok && (cur[0].valid || cur[1].valid)) {
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    Cursor& c = cur[t];
-                    if (!c.valid || !ok) continue;
-                    ok = mbar_wait(p_full(t), ph_p[t], &abort_flag, 36 + t);
-                    if (!ok) break;
-                    ph_p[t] ^= 1;
-                    issue_pv(t);
-                    // advance this tile to its next step, possibly in the next item
-                    if (++c.j == c.n) {
-                        c.base += 2 * max(c.n, c.n_other);
-                        c.idx += gridDim.x;
-                        c.ord += 1;
-                        load_item(c, t);
-                    }
-                    if (c.valid && ok) issue_s(t);
-                }
-            }
+            MmaIssuer<T> mi;
+            mi.bar0 = bar0;
+            mi.sQ = sQ;
+            mi.sKV = sKV;
+            mi.tmem = tmem_base;
+            mi.abort_flag = &abort_flag;
+            if (warp == 8) mi.template run<0>(p, total_items, n_qpairs);
+            else mi.template run<1>(p, total_items, n_qpairs);
         }
         __syncwarp();
     } else if (warp == 9) {
