@@ -28,6 +28,18 @@ namespace fa {
 constexpr int kStages = 5;                  // K/V ring slots of one 128x128 16-bit tile each
 constexpr int kPipeThreads = 384;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
+#ifndef FA_POLY_PAIRS
+#define FA_POLY_PAIRS 0
+#endif
+constexpr int kPolyPairs = FA_POLY_PAIRS;   // of every 4 column pairs, how many take the polynomial exp2
+
+// Work item taken by this CTA in its k-th round.  Items are listed longest first; rounds
+// alternate direction across the CTAs (boustrophedon) so that every CTA gets nearly the same
+// total length.  Returns a value >= total_items when the CTA has no k-th item.
+__device__ __forceinline__ int item_of_round(int k, int total_items) {
+    const int g = gridDim.x, b = blockIdx.x;
+    return k * g + ((k & 1) ? (g - 1 - b) : b);
+}
 
 struct Item {
     int b, h, hk;
@@ -129,25 +141,37 @@ __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, ui
         }
         l_run += l0 + l1;
     } else {
-        // packed f32x2 arithmetic: one FMA and one add per pair of columns
+        // packed f32x2 arithmetic: one FMA and one add per pair of columns.  Of every four pairs,
+        // kPolyPairs take the polynomial exp2 on the FMA pipe and the rest the special-function
+        // unit, so that neither pipe alone bounds the softmax.
         const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
         uint64_t la = f2_pack(0.f, 0.f), lb = la;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
+            for (int i = 0; i < 32; i += 8) {
                 const int e = c * 32 + i;
-                const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), sc2, nm2);
-                const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[e + 2]), __uint_as_float(s[e + 3])), sc2, nm2);
-                float x0, x1, x2, x3;
-                f2_unpack(x01, x0, x1);
-                f2_unpack(x23, x2, x3);
-                const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
-                la = f2_add(la, f2_pack(p0, p1));
-                lb = f2_add(lb, f2_pack(p2, p3));
-                pk[i / 2] = pack2<T>(p0, p1);
-                pk[i / 2 + 1] = pack2<T>(p2, p3);
+                float pv[8];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint64_t x01 =
+                        f2_fma(f2_pack(__uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1])), sc2, nm2);
+                    float x0, x1;
+                    f2_unpack(x01, x0, x1);
+                    if (q < kPolyPairs) {
+                        exp2_poly_pair(fmaxf(x0, -125.f), fmaxf(x1, -125.f), pv[2 * q], pv[2 * q + 1]);
+                    } else {
+                        pv[2 * q] = fast_exp2(x0);
+                        pv[2 * q + 1] = fast_exp2(x1);
+                    }
+                }
+                la = f2_add(la, f2_pack(pv[0], pv[1]));
+                lb = f2_add(lb, f2_pack(pv[2], pv[3]));
+                la = f2_add(la, f2_pack(pv[4], pv[5]));
+                lb = f2_add(lb, f2_pack(pv[6], pv[7]));
+#pragma unroll
+                for (int q = 0; q < 4; ++q) pk[i / 2 + q] = pack2<T>(pv[2 * q], pv[2 * q + 1]);
             }
             tmem_st_x16(tS + c * 16, pk);
         }
@@ -274,8 +298,8 @@ struct MmaIssuer {
         ring_add(nx.slot, nx.par, 2);
         if (++nx.j == nx.n) {  // next item: skip the entries only the other role reads
             if (nx.n_other > nx.n) ring_add(nx.slot, nx.par, 2);
-            nx.idx += gridDim.x;
             nx.ord += 1;
+            nx.idx = item_of_round(nx.ord, total_items);
             load_item<t>(nx, p, total_items, n_qpairs);
         }
         if (nx.valid && !wait_s_operands<t>(nx)) return false;
@@ -306,7 +330,7 @@ struct MmaIssuer {
     template <int t>
     __device__ __forceinline__ void run(const FwdParams& p, int total_items, int n_qpairs) {
         Cursor c;
-        c.idx = blockIdx.x;
+        c.idx = item_of_round(0, total_items);
         c.ord = 0;
         c.lead = 0;
         c.slot = 0;
@@ -386,7 +410,9 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         uint32_t ph_s = 0, ph_o = 0;
         bool ok = true;
         int lead = 0;
-        for (int idx = blockIdx.x; idx < total_items && ok; idx += gridDim.x) {
+        for (int k = 0; ok; ++k) {
+            const int idx = item_of_round(k, total_items);
+            if (idx >= total_items) break;
             const Item it = decode_item(p, idx, n_qpairs, lead);
             const int n = it.n[t];
             const int q0 = it.q0[t];
@@ -487,7 +513,9 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             uint32_t g = 0;
             int ord = 0, lead = 0;
             bool ok = true;
-            for (int idx = blockIdx.x; idx < total_items && ok; idx += gridDim.x, ++ord) {
+            for (;; ++ord) {
+                const int idx = item_of_round(ord, total_items);
+                if (idx >= total_items || !ok) break;
                 const Item it = decode_item(p, idx, n_qpairs, lead);
                 const int n_kv = max(it.n[0], it.n[1]);
                 const uint32_t q_par = (ord & 1) ^ 1;  // passes at once the first time
