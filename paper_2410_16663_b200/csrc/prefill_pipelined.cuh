@@ -1,19 +1,25 @@
 // Prefill forward, pipelined variant (the default kernel).
 //
 // A persistent CTA (one per SM, 384 threads) walks a static list of work items, longest
-// first.  An item is a pair of adjacent 128-row query tiles of one (batch, head); K/V tiles
-// of 128 keys stream through a 5-slot TMA ring shared by both query tiles.  Roles:
-//   warpgroup 0 / 1 : softmax for query tile 0 / 1, one thread per row.  Reads S from tensor
+// first, in boustrophedon order over the CTAs.  An item is a pair of adjacent 128-row query
+// tiles of one (batch, head); K/V tiles of 128 keys stream through a 5-slot TMA ring shared by
+// both query tiles.  The two tiles are handled by two "tile roles":
+//   warpgroup 0 / 1 : softmax of role 0 / 1, one thread per query row.  Reads S from tensor
 //                     memory, keeps the running rowmax / rowsum, writes P (16-bit, packed)
 //                     back over the columns S occupied, rescales O when the row max grew by
 //                     more than 2^8, and at the end of an item normalises and stores O, LSE.
-//   warp 8          : one thread issues every tcgen05.mma: S_t = Q_t K_j^T (operands in shared
-//                     memory) and O_t += P_t V_j (P from tensor memory, V N-major from shared
-//                     memory).  The S MMA for a tile's next step is issued right behind the
-//                     PV MMA of its current step, so the tensor core works on one query tile
-//                     while the other tile's softmax runs (the Cube/Vector overlap of
-//                     Section 4.1 on this hardware), also across item boundaries.
+//   warp 8 / 10     : one thread each issues the tcgen05.mma of role 0 / 1: S = Q K_j^T
+//                     (operands in shared memory) and O += P V_j (P from tensor memory, V
+//                     N-major from shared memory).  A role's round is "wait for P, issue P V,
+//                     issue S of the role's next step", so the tensor core works on one role
+//                     while the other role's softmax runs (the Cube/Vector overlap of
+//                     Section 4.1 on this hardware), also across item boundaries.  The two
+//                     threads pass a turn token so that their MMA batches alternate back to
+//                     back while each thread's waits and commits overlap the other's batch.
 //   warp 9          : one thread issues every TMA load.
+// Under the causal mask the upper tile of a pair visits one kv tile more than the lower one;
+// the roles swap which tile they take whenever role 0 is a step ahead, so both carry the same
+// load and role 0 is never behind role 1 in the ring.
 // Tensor memory: columns [0,128) S_0/P_0, [128,256) S_1/P_1, [256,384) O_0, [384,512) O_1.
 // Synchronisation is mbarrier-only; every wait is bounded (see mbar_wait).
 #pragma once
@@ -27,6 +33,12 @@ namespace fa {
 
 constexpr int kStages = 5;                  // K/V ring slots of one 128x128 16-bit tile each
 constexpr int kPipeThreads = 384;
+// Register reallocation (setmaxnreg moves registers between warpgroups of the CTA only; an
+// increase that the other warpgroups' decrease does not cover would wait forever).
+constexpr int kPipeLaunchRegs = (65536 / kPipeThreads) & ~7;  // 168
+constexpr int kPipeSoftmaxRegs = 224, kPipeOtherRegs = 56;
+static_assert(256 * (kPipeSoftmaxRegs - kPipeLaunchRegs) <= 128 * (kPipeLaunchRegs - kPipeOtherRegs),
+              "setmaxnreg.inc would wait for registers nobody releases");
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
 #ifndef FA_POLY_PAIRS
 #define FA_POLY_PAIRS 0
@@ -353,6 +365,47 @@ struct MmaIssuer {
     }
 };
 
+// The single thread that issues every TMA load of the CTA: per item Q of role 0, K_0, Q of
+// role 1, V_0, K_1, V_1, ... through the K/V ring.
+__device__ __forceinline__ void run_loader(uint32_t bar0, uint32_t sQ, uint32_t sKV, const CUtensorMap* tm_q,
+                                           const CUtensorMap* tm_k, const CUtensorMap* tm_v, const FwdParams& p,
+                                           int total_items, int n_qpairs, volatile uint32_t* abort_flag) {
+        tma_prefetch_desc(tm_q);
+        tma_prefetch_desc(tm_k);
+        tma_prefetch_desc(tm_v);
+        uint32_t g = 0;
+        int ord = 0, lead = 0;
+        bool ok = true;
+        for (;; ++ord) {
+            const int idx = item_of_round(ord, total_items);
+            if (idx >= total_items || !ok) break;
+            const Item it = decode_item(p, idx, n_qpairs, lead);
+            const int n_kv = max(it.n[0], it.n[1]);
+            const uint32_t q_par = (ord & 1) ^ 1;  // passes at once the first time
+            ok = mbar_wait(bar_q_empty(bar0, 0), q_par, abort_flag, 50);
+            if (!ok) break;
+            mbar_expect_tx(bar_q_full(bar0, 0), kTileBytes);
+            load_tile(sQ, tm_q, bar_q_full(bar0, 0), it.h, it.q0[0], it.b);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                for (int kv = 0; kv < 2 && ok; ++kv, ++g) {
+                    const uint32_t slot = g % kStages;
+                    ok = mbar_wait(bar_kv_empty(bar0, slot), ((g / kStages) & 1) ^ 1, abort_flag, 52 + kv);
+                    if (!ok) break;
+                    mbar_expect_tx(bar_kv_full(bar0, slot), kTileBytes);
+                    load_tile(sKV + slot * kTileBytes, kv ? tm_v : tm_k, bar_kv_full(bar0, slot), it.hk, j * kTile, it.b);
+                    if (j == 0 && kv == 0) {
+                        // Q of role 1 goes after K_0 so that role 0 can start the item while
+                        // role 1 still finishes the previous one
+                        ok = mbar_wait(bar_q_empty(bar0, 1), q_par, abort_flag, 51);
+                        if (!ok) break;
+                        mbar_expect_tx(bar_q_full(bar0, 1), kTileBytes);
+                        load_tile(sQ + kTileBytes, tm_q, bar_q_full(bar0, 1), it.h, it.q0[1], it.b);
+                    }
+                }
+            }
+        }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -401,7 +454,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
     if (warp < 8) {
         // ================================================================ softmax + epilogue
-        setmaxnreg_inc<224>();  // a whole row of S lives in registers
+        setmaxnreg_inc<kPipeSoftmaxRegs>();  // a whole row of S lives in registers
         const int t = warp >> 2;                    // query tile of this warpgroup
         const int r_in_tile = tid & 127;
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -489,7 +542,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             tc_fence_before();
         }
     } else {
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<kPipeOtherRegs>();
     }
     if (warp == 8 || warp == 10) {
         // ================================================================ MMA issue (role 0 / 1)
@@ -506,42 +559,7 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         __syncwarp();
     } else if (warp == 9) {
         // ================================================================ TMA loads
-        if (lane == 0) {
-            tma_prefetch_desc(&tm_q);
-            tma_prefetch_desc(&tm_k);
-            tma_prefetch_desc(&tm_v);
-            uint32_t g = 0;
-            int ord = 0, lead = 0;
-            bool ok = true;
-            for (;; ++ord) {
-                const int idx = item_of_round(ord, total_items);
-                if (idx >= total_items || !ok) break;
-                const Item it = decode_item(p, idx, n_qpairs, lead);
-                const int n_kv = max(it.n[0], it.n[1]);
-                const uint32_t q_par = (ord & 1) ^ 1;  // passes at once the first time
-                ok = mbar_wait(q_empty(0), q_par, &abort_flag, 50);
-                if (!ok) break;
-                mbar_expect_tx(q_full(0), kTileBytes);
-                load_tile(sQ, &tm_q, q_full(0), it.h, it.q0[0], it.b);
-                for (int j = 0; j < n_kv && ok; ++j) {
-                    for (int kv = 0; kv < 2 && ok; ++kv, ++g) {
-                        const uint32_t slot = g % kStages;
-                        ok = mbar_wait(kv_empty(slot), ((g / kStages) & 1) ^ 1, &abort_flag, 52 + kv);
-                        if (!ok) break;
-                        mbar_expect_tx(kv_full(slot), kTileBytes);
-                        load_tile(sKV + slot * kTileBytes, kv ? &tm_v : &tm_k, kv_full(slot), it.hk, j * kTile, it.b);
-                        if (j == 0 && kv == 0) {
-                            // Q of role 1 goes after K_0 so that role 0 can start the item while
-                            // role 1 still finishes the previous one
-                            ok = mbar_wait(q_empty(1), q_par, &abort_flag, 51);
-                            if (!ok) break;
-                            mbar_expect_tx(q_full(1), kTileBytes);
-                            load_tile(sQ + kTileBytes, &tm_q, q_full(1), it.h, it.q0[1], it.b);
-                        }
-                    }
-                }
-            }
-        }
+        if (lane == 0) run_loader(bar0, sQ, sKV, &tm_q, &tm_k, &tm_v, p, total_items, n_qpairs, &abort_flag);
         __syncwarp();
     }
 
