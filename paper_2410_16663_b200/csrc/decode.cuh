@@ -1,9 +1,9 @@
 // Decode-stage attention (one query row per sequence over the cached K and V), split along
 // the cache: each CTA streams one chunk of one (sequence, kv head) through a TMA-fed
-// shared-memory ring and keeps running (rowmax, rowsum, O) for the G query heads that share
+// shared-memory ring and keeps running (rowmax, rowsum, O) for the query heads that share
 // the kv head; a second kernel merges the per-chunk partial results.  The work is a single
-// pass over the cache, so the kernel is written for HBM bandwidth: arithmetic is plain fp32
-// FMA, every cache byte is read exactly once and nothing but the partials is written.
+// pass over the cache, so the kernel is written for HBM bandwidth: every cache byte is read
+// exactly once and nothing but the partials is written.
 #pragma once
 
 #include "sm100_ptx.cuh"
@@ -14,7 +14,6 @@ constexpr int kDecTile = 128;                 // keys per shared-memory tile
 constexpr int kDecStages = 3;                 // ring depth (K and V tiles each 32 KiB)
 constexpr int kDecTileBytes = 32768;
 constexpr int kDecHalfBytes = 16384;
-constexpr int kDecThreads = 128;
 
 struct DecodeParams {
     const void* q;        // [B,1,Hq,128] 16-bit
@@ -24,236 +23,270 @@ struct DecodeParams {
     int B, Hq, Hkv, Smax;
     int chunk;            // keys per chunk (multiple of kDecTile)
     int n_chunks;         // ceil(Smax / chunk)
-    int heads_per_item;   // G when query heads of a group are processed together, else 1
     float scale_log2;
 };
 
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+// ---------------------------------------------------------------------------------------
+// Split kernel.  A CTA takes one chunk of one (sequence, kv head) and up to 16 of the query
+// heads that share the kv head (all of them when Hq / Hkv <= 16).  The query rows are padded
+// to the 16 rows of a warp-level mma.sync (m16n8k16, fp32 accumulate): the scan is bound by
+// the cache stream, and the warp-level tensor path keeps the arithmetic per cache byte far
+// below what the FMA pipe would need, for one query head as well as for sixteen.  Each of the
+// four consumer warps owns keys [32w, 32w+32) of every 128-key tile and keeps its own running
+// (rowmax, rowsum, O) for them, so consumer warps never synchronise with each other until the
+// final merge; a fifth warp issues the TMA loads into a 3-slot ring of K and V tiles.
+// Cache rows past the sequence may hold NaN: their scores are masked and their V rows are
+// zeroed in shared memory before the second MMA touches them.
+constexpr int kDecMmaThreads = 160;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                  : "r"(addr));
-    return v;
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <typename T>
-__device__ __forceinline__ float2 unpack2(uint32_t w);
-template <>
-__device__ __forceinline__ float2 unpack2<__half>(uint32_t w) {
-    return __half22float2(*reinterpret_cast<__half2*>(&w));
-}
-template <>
-__device__ __forceinline__ float2 unpack2<__nv_bfloat16>(uint32_t w) {
-    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-
-// grid: (n_chunks, items_per_batch, B) where items_per_batch = Hkv (grouped) or Hq (G == 1 fallback)
-template <typename T, int G>
-__global__ void __launch_bounds__(kDecThreads, 1)
-fa_decode_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                       const DecodeParams p) {
+// grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
+__global__ void __launch_bounds__(kDecMmaThreads, 1)
+fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                           const DecodeParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sK = smem_base;                                   // kDecStages tiles
-    const uint32_t sV = smem_base + kDecStages * kDecTileBytes;      // kDecStages tiles
-    __shared__ __align__(16) float q_s[G][128];
-    __shared__ __align__(16) float p_s[G][kDecTile];
-    __shared__ float red_s[G][4];
-    __shared__ __align__(8) uint64_t bars[2 * kDecStages];
+    const uint32_t sK = smem_base;
+    const uint32_t sV = smem_base + kDecStages * kDecTileBytes;
+    __shared__ __align__(8) uint64_t bars[3 * kDecStages];  // K full, V full, slot empty
     __shared__ volatile uint32_t abort_flag;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int c = blockIdx.x;
-    const int item = blockIdx.y;
     const int b = blockIdx.z;
     const int g_all = p.Hq / p.Hkv;
-    const int h0 = (p.heads_per_item == 1) ? item : item * G;   // first query head of this item
-    const int hk = h0 / g_all;
+    const int n_sub = (g_all + 15) / 16;           // CTAs per kv head when more than 16 heads share it
+    const int hk = blockIdx.y / n_sub;
+    const int sub = blockIdx.y % n_sub;
+    const int h0 = hk * g_all + sub * 16;          // first query head of this CTA
+    const int G = min(16, g_all - sub * 16);       // its number of query heads
 
     int len = p.seqlens[b];
     len = max(0, min(len, p.Smax));
     const int k_begin = c * p.chunk;
     const int k_end = min(len, k_begin + p.chunk);
-    if (k_begin >= k_end) return;  // uniform for the CTA: nothing allocated, nothing pending
+    if (k_begin >= k_end) return;  // uniform for the CTA
     const int n_tiles = (k_end - k_begin + kDecTile - 1) / kDecTile;
 
     if (tid == 0) {
         for (int i = 0; i < 2 * kDecStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        for (int i = 0; i < kDecStages; ++i) mbar_init(smem_u32(&bars[2 * kDecStages + i]), 4);  // one arrival per consumer warp
         abort_flag = 0;
         fence_mbar_init();
     }
-    // q -> fp32 in shared memory
-    for (int i = tid; i < G * 64; i += kDecThreads) {
-        const int g = i >> 6, t2 = i & 63;
-        const uint32_t w = reinterpret_cast<const uint32_t*>(
-            static_cast<const T*>(p.q) + ((long long)b * p.Hq + h0 + g) * 128)[t2];
-        const float2 f = unpack2<T>(w);
-        q_s[g][2 * t2] = f.x;
-        q_s[g][2 * t2 + 1] = f.y;
-    }
     __syncthreads();
 
-    auto issue_tile = [&](int t) {
-        const int st = t % kDecStages;
-        const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
-        const int row0 = k_begin + t * kDecTile;
-        mbar_expect_tx(bk, kDecTileBytes);
-        tma_load_4d(sK + st * kDecTileBytes, &tm_k, bk, 0, hk, row0, b);
-        tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes, &tm_k, bk, 64, hk, row0, b);
-        mbar_expect_tx(bv, kDecTileBytes);
-        tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, b);
-        tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, b);
-    };
-    int issued = 0;
-    if (tid == 0) {
-        for (; issued < kDecStages - 1 && issued < n_tiles; ++issued) issue_tile(issued);
-    }
-
-    float m_run[G], l_loc[G], o_acc[G][8];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-        m_run[g] = -INFINITY;
-        l_loc[g] = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o_acc[g][i] = 0.f;
-    }
-    const int kg = tid >> 4, dc = tid & 15;  // P V phase: key group (key & 7 == kg) and 8-wide slice of d
-    bool ok = true;
-
-    for (int t = 0; t < n_tiles; ++t) {
-        const int st = t % kDecStages;
-        const uint32_t parity = (t / kDecStages) & 1;
-        const int valid = min(kDecTile, k_end - (k_begin + t * kDecTile));  // keys of this tile in range
-        if (!mbar_wait(smem_u32(&bars[st]), parity, &abort_flag, 20)) { ok = false; break; }
-        // ---- scores: thread `tid` owns key `tid` of the tile
-        float s[G];
+    if (warp == 4) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0) {
+            for (int t = 0; t < n_tiles; ++t) {
+                const int st = t % kDecStages;
+                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                if (!mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22)) break;
+                const int row0 = k_begin + t * kDecTile;
+                mbar_expect_tx(bk, kDecTileBytes);
+                tma_load_4d(sK + st * kDecTileBytes, &tm_k, bk, 0, hk, row0, b);
+                tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes, &tm_k, bk, 64, hk, row0, b);
+                mbar_expect_tx(bv, kDecTileBytes);
+                tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, b);
+                tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, b);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------------------------------------------------------- consumers
+        const int g = lane >> 2, t4 = lane & 3;  // fragment row (query head g and g + 8) and column pair
+        // Q as A fragments for the eight k-steps of d = 128 (rows >= G are zero)
+        uint32_t qa[8][4];
         {
-            float sa[G], sb[G];  // two partial sums per head keep the FMA chains short
+            const __half* qb = static_cast<const __half*>(p.q) + ((long long)b * p.Hq + h0) * 128;
 #pragma unroll
-            for (int g = 0; g < G; ++g) sa[g] = sb[g] = 0.f;
-            const uint32_t krow = sK + st * kDecTileBytes + tid * 128;
+            for (int ks = 0; ks < 8; ++ks) {
+                const int k0 = ks * 16 + 2 * t4;
+                qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0) : 0u;
+                qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0) : 0u;
+                qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0 + 8) : 0u;
+                qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0 + 8) : 0u;
+            }
+        }
+        float o[16][4];
 #pragma unroll
-            for (int c16 = 0; c16 < 16; ++c16) {
-                const uint4 kw = lds128(krow + (c16 >> 3) * kDecHalfBytes + (((c16 & 7) ^ (tid & 7)) << 4));
-                const float2 k0 = unpack2<T>(kw.x), k1 = unpack2<T>(kw.y), k2 = unpack2<T>(kw.z),
-                             k3 = unpack2<T>(kw.w);
+        for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;  // rows g and g + 8
+        const int key_w = warp * 32;  // this warp's keys inside a tile
+        bool ok = true;
+
+        for (int t = 0; t < n_tiles; ++t) {
+            const int st = t % kDecStages;
+            const uint32_t parity = (t / kDecStages) & 1;
+            const int valid = min(kDecTile, k_end - (k_begin + t * kDecTile)) - key_w;  // valid keys of this warp's 32
+            ok = mbar_wait(smem_u32(&bars[st]), parity, &abort_flag, 20);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            float sc[4][4];
+            if (valid > 0) {
+                // ---- S = Q K^T for this warp's four blocks of 8 keys
+                const uint32_t kt = sK + st * kDecTileBytes;
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const float4 qa = *reinterpret_cast<const float4*>(&q_s[g][c16 * 8]);
-                    const float4 qb = *reinterpret_cast<const float4*>(&q_s[g][c16 * 8 + 4]);
-                    sa[g] = fmaf(qa.x, k0.x, sa[g]);
-                    sb[g] = fmaf(qb.x, k2.x, sb[g]);
-                    sa[g] = fmaf(qa.y, k0.y, sa[g]);
-                    sb[g] = fmaf(qb.y, k2.y, sb[g]);
-                    sa[g] = fmaf(qa.z, k1.x, sa[g]);
-                    sb[g] = fmaf(qb.z, k3.x, sb[g]);
-                    sa[g] = fmaf(qa.w, k1.y, sa[g]);
-                    sb[g] = fmaf(qb.w, k3.y, sb[g]);
+                for (int nb = 0; nb < 4; ++nb) {
+                    sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+                    const int key = key_w + nb * 8 + (lane & 7);
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {  // 4 d-chunks of 8 per ldmatrix.x4 = two k-steps
+                        const int chunk = c4 * 4 + (lane >> 3);
+                        const uint32_t addr = kt + (chunk >> 3) * kDecHalfBytes + key * 128 + (((chunk & 7) ^ (key & 7)) << 4);
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4(addr, b0, b1, b2, b3);
+                        mma_16816(sc[nb], qa[2 * c4], b0, b1);
+                        mma_16816(sc[nb], qa[2 * c4 + 1], b2, b3);
+                    }
+                }
+                // ---- mask, running max, probabilities
+                float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+                for (int nb = 0; nb < 4; ++nb) {
+                    const int k0 = nb * 8 + 2 * t4;
+                    if (k0 >= valid) sc[nb][0] = sc[nb][2] = -INFINITY;
+                    if (k0 + 1 >= valid) sc[nb][1] = sc[nb][3] = -INFINITY;
+                    mx_lo = fmaxf(mx_lo, fmaxf(sc[nb][0], sc[nb][1]));
+                    mx_hi = fmaxf(mx_hi, fmaxf(sc[nb][2], sc[nb][3]));
+                }
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);  // finite: key 0 of the warp is valid
+                const float a_lo = (m_lo == -INFINITY) ? 0.f : fast_exp2((m_lo - mn_lo) * p.scale_log2);
+                const float a_hi = (m_hi == -INFINITY) ? 0.f : fast_exp2((m_hi - mn_hi) * p.scale_log2);
+                m_lo = mn_lo;
+                m_hi = mn_hi;
+                const float nm_lo = -mn_lo * p.scale_log2, nm_hi = -mn_hi * p.scale_log2;
+                float s_lo = 0.f, s_hi = 0.f;
+#pragma unroll
+                for (int nb = 0; nb < 4; ++nb) {
+                    const int k0 = nb * 8 + 2 * t4;
+                    sc[nb][0] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][0], p.scale_log2, nm_lo)) : 0.f;
+                    sc[nb][1] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][1], p.scale_log2, nm_lo)) : 0.f;
+                    sc[nb][2] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][2], p.scale_log2, nm_hi)) : 0.f;
+                    sc[nb][3] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][3], p.scale_log2, nm_hi)) : 0.f;
+                    s_lo += sc[nb][0] + sc[nb][1];
+                    s_hi += sc[nb][2] + sc[nb][3];
+                }
+                l_lo = l_lo * a_lo + s_lo;  // per-thread partial of the row sum (the quad is summed at the end)
+                l_hi = l_hi * a_hi + s_hi;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    o[i][0] *= a_lo;
+                    o[i][1] *= a_lo;
+                    o[i][2] *= a_hi;
+                    o[i][3] *= a_hi;
                 }
             }
+            ok = mbar_wait(smem_u32(&bars[kDecStages + st]), parity, &abort_flag, 21);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (valid > 0) {
+                const uint32_t vt = sV + st * kDecTileBytes;
+                if (valid < 32) {
+                    // rows past the sequence may hold NaN bits: zero them (0 * NaN would poison O)
+                    for (int i = lane; i < (32 - valid) * 16; i += 32) {
+                        const int key = key_w + valid + (i >> 4), ch = i & 15;
+                        const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                    }
+                    __syncwarp();
+                }
+                // ---- O += P V: two k-steps of 16 keys, sixteen blocks of 8 output columns
 #pragma unroll
-            for (int g = 0; g < G; ++g) s[g] = sa[g] + sb[g];
-        }
-        const bool live = tid < valid;  // keys past the sequence hold arbitrary bits
+                for (int k2 = 0; k2 < 2; ++k2) {
+                    uint32_t pa[4];
+                    {
+                        __half2 h0 = __floats2half2_rn(sc[2 * k2][0], sc[2 * k2][1]);
+                        __half2 h1 = __floats2half2_rn(sc[2 * k2][2], sc[2 * k2][3]);
+                        __half2 h2 = __floats2half2_rn(sc[2 * k2 + 1][0], sc[2 * k2 + 1][1]);
+                        __half2 h3 = __floats2half2_rn(sc[2 * k2 + 1][2], sc[2 * k2 + 1][3]);
+                        pa[0] = *reinterpret_cast<uint32_t*>(&h0);
+                        pa[1] = *reinterpret_cast<uint32_t*>(&h1);
+                        pa[2] = *reinterpret_cast<uint32_t*>(&h2);
+                        pa[3] = *reinterpret_cast<uint32_t*>(&h3);
+                    }
+                    const int key = key_w + k2 * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float wm = warp_max(live ? s[g] : -INFINITY);
-            if (lane == 0) red_s[g][warp] = wm;
-        }
-        __syncthreads();  // (A) all warps are also past the P V of the previous tile
-        if (tid == 0 && issued < n_tiles) {
-            issue_tile(issued);  // refills the slot the previous tile used
-            ++issued;
-        }
-        float alpha[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float tm = fmaxf(fmaxf(red_s[g][0], red_s[g][1]), fmaxf(red_s[g][2], red_s[g][3]));
-            const float m_new = fmaxf(m_run[g], tm);  // finite: every tile holds at least one key in range
-            alpha[g] = (m_run[g] == -INFINITY) ? 0.f : fast_exp2((m_run[g] - m_new) * p.scale_log2);
-            const float pv = live ? fast_exp2((s[g] - m_new) * p.scale_log2) : 0.f;
-            p_s[g][tid] = pv;
-            l_loc[g] = l_loc[g] * alpha[g] + pv;
-            m_run[g] = m_new;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o_acc[g][i] *= alpha[g];
-        }
-        __syncthreads();  // (B) probabilities visible
-        if (!mbar_wait(smem_u32(&bars[kDecStages + st]), parity, &abort_flag, 21)) { ok = false; break; }
-        // ---- O += P V: this thread adds keys kg, kg+8, ... for its 8 output dims
-        {
-            const uint32_t vbase = sV + st * kDecTileBytes + (dc >> 3) * kDecHalfBytes + (((dc & 7) ^ kg) << 4);
-#pragma unroll 4
-            for (int i = 0; i < 16; ++i) {
-                const int key = kg + 8 * i;
-                if (key < valid) {  // never touch rows past the sequence (0 * NaN)
-                    const uint4 vw = lds128(vbase + key * 128);
-                    const float2 v0 = unpack2<T>(vw.x), v1 = unpack2<T>(vw.y), v2 = unpack2<T>(vw.z),
-                                 v3 = unpack2<T>(vw.w);
-#pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const float pg = p_s[g][key];
-                        o_acc[g][0] = fmaf(pg, v0.x, o_acc[g][0]);
-                        o_acc[g][1] = fmaf(pg, v0.y, o_acc[g][1]);
-                        o_acc[g][2] = fmaf(pg, v1.x, o_acc[g][2]);
-                        o_acc[g][3] = fmaf(pg, v1.y, o_acc[g][3]);
-                        o_acc[g][4] = fmaf(pg, v2.x, o_acc[g][4]);
-                        o_acc[g][5] = fmaf(pg, v2.y, o_acc[g][5]);
-                        o_acc[g][6] = fmaf(pg, v3.x, o_acc[g][6]);
-                        o_acc[g][7] = fmaf(pg, v3.y, o_acc[g][7]);
+                    for (int n2 = 0; n2 < 8; ++n2) {  // two output blocks per ldmatrix.x4.trans
+                        const int ch = n2 * 2 + (lane >> 4);
+                        const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4_trans(addr, b0, b1, b2, b3);
+                        mma_16816(o[2 * n2], pa, b0, b1);
+                        mma_16816(o[2 * n2 + 1], pa, b2, b3);
                     }
                 }
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kDecStages + st]));
         }
-    }
 
-    // ---- reduce over threads and write this chunk's partial result
-    __syncthreads();
-    if (ok) {
-        // every tile that was requested has been consumed, so the ring is free: reuse its
-        // first bytes as the [8 key groups][G][128] reduction buffer
-        float* o_red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+        // ---- merge the four warps' states and write this chunk's partial result
+        // (all tiles this CTA requested have been consumed by every warp before the barrier below,
+        // so the ring can be reused as the merge buffer)
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][128]
+        float* ml = mo + 4 * 16 * 128;                                                       // [4][16][2]: m, l
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ok) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float ws = warp_sum(l_loc[g]);
-            if (lane == 0) red_s[g][warp] = ws;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o_red[(kg * G + g) * 128 + dc * 8 + i] = o_acc[g][i];
+            for (int i = 0; i < 16; ++i) {
+                const int col = i * 8 + 2 * t4;
+                *reinterpret_cast<float2*>(&mo[(warp * 16 + g) * 128 + col]) = make_float2(o[i][0], o[i][1]);
+                *reinterpret_cast<float2*>(&mo[(warp * 16 + g + 8) * 128 + col]) = make_float2(o[i][2], o[i][3]);
+            }
+            if (t4 == 0) {
+                ml[(warp * 16 + g) * 2] = m_lo;
+                ml[(warp * 16 + g) * 2 + 1] = l_lo;
+                ml[(warp * 16 + g + 8) * 2] = m_hi;
+                ml[(warp * 16 + g + 8) * 2 + 1] = l_hi;
+            }
         }
-        __syncthreads();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ok) {
+            for (int r = 0; r < G; ++r) {  // thread `tid` owns output column `tid` of every row
+                float M = -INFINITY;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float l = red_s[g][0] + red_s[g][1] + red_s[g][2] + red_s[g][3];
-            float acc = 0.f;
+                for (int w = 0; w < 4; ++w) M = fmaxf(M, ml[(w * 16 + r) * 2]);
+                float l = 0.f, acc = 0.f;
 #pragma unroll
-            for (int r = 0; r < 8; ++r) acc += o_red[(r * G + g) * 128 + tid];
-            const long long slot = ((long long)b * p.Hq + h0 + g) * p.n_chunks + c;
-            p.o_part[slot * 128 + tid] = acc / l;
-            if (tid == 0)
-                p.lse_part[slot] = (m_run[g] * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
-        }
-    } else if (tid == 0) {
-        // gave up on a wait: wait (bounded) for copies still in flight before the CTA's
-        // shared memory is released
-        for (int t = 0; t < issued; ++t) {
-            const int st = t % kDecStages;
-            const uint32_t parity = (t / kDecStages) & 1;
-            const unsigned long long t0 = globaltimer_ns();
-            while (!mbar_try_wait(smem_u32(&bars[st]), parity) && globaltimer_ns() - t0 < 100000000ull) {}
-            while (!mbar_try_wait(smem_u32(&bars[kDecStages + st]), parity) &&
-                   globaltimer_ns() - t0 < 200000000ull) {}
+                for (int w = 0; w < 4; ++w) {
+                    const float mw = ml[(w * 16 + r) * 2];
+                    const float sw = (mw == -INFINITY) ? 0.f : fast_exp2((mw - M) * p.scale_log2);
+                    l += sw * ml[(w * 16 + r) * 2 + 1];
+                    acc += sw * mo[(w * 16 + r) * 128 + tid];
+                }
+                const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;
+                p.o_part[slot * 128 + tid] = acc / l;
+                if (tid == 0) p.lse_part[slot] = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
+            }
         }
     }
 }

@@ -210,19 +210,6 @@ int decode_chunk(int B, int Hkv, int Smax) {
     return chunk;
 }
 
-template <typename T, int G>
-int launch_decode_split(const CUtensorMap& tk, const CUtensorMap& tv, const fa::DecodeParams& dp, int items,
-                        cudaStream_t st) {
-    constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
-    auto kern = fa::fa_decode_split_kernel<T, G>;
-    int rc = set_smem(kern, smem);
-    if (rc) return rc;
-    dim3 grid(dp.n_chunks, items, dp.B);
-    kern<<<grid, fa::kDecThreads, smem, st>>>(tk, tv, dp);
-    cudaError_t e = cudaGetLastError();
-    return e == cudaSuccess ? FA_OK : cuda_fail(e);
-}
-
 }  // namespace
 
 extern "C" {
@@ -287,14 +274,17 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
         rc = encode_map(&tv, v_cache, B, Skv_max, Hkv, (int64_t)Skv_max * Hkv * 128, (int64_t)Hkv * 128, 128,
                         fa::kDecTile, false);
         if (rc) return rc;
-        switch (g) {
-            case 1: dp.heads_per_item = 1; rc = launch_decode_split<__half, 1>(tk, tv, dp, Hq, st); break;
-            case 2: dp.heads_per_item = 2; rc = launch_decode_split<__half, 2>(tk, tv, dp, Hkv, st); break;
-            case 4: dp.heads_per_item = 4; rc = launch_decode_split<__half, 4>(tk, tv, dp, Hkv, st); break;
-            case 8: dp.heads_per_item = 8; rc = launch_decode_split<__half, 8>(tk, tv, dp, Hkv, st); break;
-            default:  // other group sizes: one query head per item (the kv head is re-read per head)
-                dp.heads_per_item = 1; rc = launch_decode_split<__half, 1>(tk, tv, dp, Hq, st); break;
+        constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
+        static bool attr_set = false;
+        if (!attr_set) {
+            rc = set_smem(fa::fa_decode_split_mma_kernel, smem);
+            if (rc) return rc;
+            attr_set = true;
         }
+        dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
+        fa::fa_decode_split_mma_kernel<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
+        cudaError_t e = cudaGetLastError();
+        rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
     }
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);

@@ -237,7 +237,7 @@ def run_decode(fa, q, k, v, seqlens_dev, scale):
     return o, lse
 
 
-@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (8, 2), (8, 1), (6, 2), (16, 1)])
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (8, 2), (8, 1), (6, 2), (16, 1), (17, 1), (40, 2)])
 def test_decode_small_full(fa, hq, hkv):
     cfg = synth.DecodeConfig("t", 5, hq, hkv, 1500, 1, 1500, seed=hq * 31 + hkv)
     q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=True)
