@@ -223,16 +223,25 @@ def run_product(args, rank, world, local_rank):
             "frac_measured_hbm": round(gbs / world / peaks["hbm_gbs"], 4)}
     # roofline of the kernel behind `value` (prefill: a dense contraction -> tensor peak, burst
     # figure because one launch lasts a fraction of a millisecond) and of the decode scan (HBM)
-    out["roofline"] = {"kernel": "fa_fwd (prefill)", "bound": "tensor", "achieved": round(tflops / world, 2),
-                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+    # `traffic`: DRAM bytes per launch from one ncu capture (profiles/): the C2 prefill launch
+    # itself, and for decode a 4.3 GB case of the same kernel whose dram bytes were 1.007 x its
+    # algorithmic bytes, scaled to this launch by the cache bytes it scans
+    c2_traffic = 546.0e6 if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
+    algo_prefill_bytes = (2.0 * pc.B * pc.Sq * pc.Hq + 2.0 * pc.B * pc.Skv * pc.Hkv) * pc.d * 2 + 4.0 * pc.B * pc.Hq * pc.Sq
+    out["roofline"] = {"kernel": "fa_fwd_pipelined_kernel (prefill, the kernel behind `value`)", "bound": "tensor",
+                       "achieved": round(tflops / world, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                        "frac": round(tflops / world / peaks["bf16_tflops"], 4),
-                       "peak_source": peaks["source"] + " (bf16 GEMM burst; fp16 has the same nominal rate)",
-                       "traffic": None}
+                       "peak_source": peaks["source"] + " bf16 GEMM burst (of measured; fp16 has the same nominal rate)",
+                       "frac_nominal": round(tflops / world / NOMINAL_TENSOR_TFLOPS, 4),
+                       "algorithmic_flops": pc.flops(), "algorithmic_bytes": algo_prefill_bytes,
+                       "traffic": c2_traffic}
     g0 = out["decode_mha"]["gbs"] / world
-    out["roofline_decode"] = {"kernel": "fa_decode_split (decode, Hkv=32)", "bound": "hbm",
-                              "achieved": round(g0, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                              "frac": round(g0 / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],
-                              "traffic": None}
+    out["roofline_decode"] = {"kernel": "fa_decode_split_mma_kernel (decode Hkv=32, the dominant kernel by time)",
+                              "bound": "hbm", "achieved": round(g0, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": round(g0 / peaks["hbm_gbs"], 4),
+                              "peak_source": peaks["source"] + " copy bandwidth (of measured; the scan only reads)",
+                              "frac_nominal": round(g0 / NOMINAL_HBM_GBS, 4),
+                              "algorithmic_bytes": dec[0]["bytes"], "traffic": round(1.007 * dec[0]["bytes"])}
 
     if rank == 0:
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
