@@ -121,6 +121,23 @@ def decode_cache_bytes(cfg, seqlens) -> float:
     return kv + 2.0 * cfg.B * cfg.Hq * cfg.d * 2
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of per-rank device timings over all ranks (the slowest rank sets the
+    job's time); every rank gets the result.  No data-path collective exists in this workload:
+    this reduction of a few timing scalars is the only communication."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+    return [float(x) for x in t]
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms: float) -> float:
+    """Aggregate rate of `world` ranks that each process `units_per_rank` in `ms` (weak scaling)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 def run_product(args, rank, world, local_rank):
     from paper_2410_16663_b200 import binding as fa  # raises if the CUDA library is missing
 
@@ -189,14 +206,10 @@ def run_product(args, rank, world, local_rank):
 
     # ---- max over ranks (device-timed), whole-job aggregate
     ms_step = total_ms / args.steps
-    times = torch.tensor([ms_step] + part_ms, dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.barrier()
-    ms_step, part_ms = float(times[0]), [float(x) for x in times[1:]]
+    times = max_over_ranks([ms_step] + part_ms, world, dev)
+    ms_step, part_ms = times[0], times[1:]
 
-    tflops = world * pc.flops() / (part_ms[0] * 1e-3) / 1e12
+    tflops = whole_job_rate(pc.flops(), world, part_ms[0]) / 1e12
     out = {
         "metric": METRIC, "value": round(tflops, 2), "unit": "TFLOPS", "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4),
@@ -216,7 +229,7 @@ def run_product(args, rank, world, local_rank):
         "clocks": clocks,
     }
     for i, d in enumerate(dec):
-        gbs = world * d["bytes"] / (part_ms[1 + i] * 1e-3) / 1e9
+        gbs = whole_job_rate(d["bytes"], world, part_ms[1 + i]) / 1e9
         out["decode_" + ("mha" if i == 0 else "gqa")] = {
             "ms": round(part_ms[1 + i], 4), "gbs": round(gbs, 1), "kv_bytes": d["bytes"],
             "frac_nominal_hbm": round(gbs / world / NOMINAL_HBM_GBS, 4),
