@@ -23,6 +23,7 @@ struct FwdParams {
     long long o_sb, o_ss, o_sh;  // element strides of o
     int o_fp32;
     int n_qtiles;
+    int o_align32;  // o and its strides are 32-byte aligned: rows can be written with 256-bit stores
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim
