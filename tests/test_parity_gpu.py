@@ -142,6 +142,24 @@ def test_bhsd_strided_layout(fa):
     assert_close_to_oracle(o, lse, o_ref, l_ref, what="BHSD views")
 
 
+def test_output_aligned_to_16_but_not_32_bytes(fa):
+    # rows that start on a 16-byte but not a 32-byte boundary take the 128-bit store path
+    cfg = synth.PrefillConfig("t", 1, 2, 2, 260, 260, dtype="fp16", causal=True, seed=12)
+    q, k, v = synth.prefill_inputs(cfg, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
+    n = q.numel()
+    buf = torch.full((n + 64,), float("nan"), dtype=torch.float16, device=DEV)
+    base = (-buf.data_ptr() // 2) % 16          # elements up to the next 32-byte boundary
+    o = buf[base + 8: base + 8 + n].view(1, 260, 2, 128)
+    assert o.data_ptr() % 32 == 16
+    lse = torch.empty(1, 2, 260, dtype=torch.float32, device=DEV)
+    fa.fa_forward_ex(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, True, cfg.scale)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what="16-byte aligned output")
+    assert torch.isnan(buf[:base + 8]).all() and torch.isnan(buf[base + 8 + n:]).all()
+
+
 def test_degenerate_sizes(fa):
     q = torch.randn(2, 5, 2, 128, device=DEV).half()
     kv0 = torch.empty(2, 0, 2, 128, dtype=torch.float16, device=DEV)
