@@ -153,7 +153,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.lse = p.lse;
     fp.B = p.B; fp.Hq = p.Hq; fp.Hkv = p.Hkv; fp.Sq = p.Sq; fp.Skv = p.Skv;
     fp.causal = p.causal ? 1 : 0;
-    fp.scale_log2 = p.scale * 1.4426950408889634f;
+    // strictly positive, so that a hidden score (-inf) times the scale is -inf and never NaN;
+    // for scale == 0 the substitute is far below anything fp32 scores could resolve
+    fp.scale_log2 = fmaxf(p.scale * 1.4426950408889634f, 1e-30f);
     fp.o_sb = p.o_stride[0]; fp.o_ss = p.o_stride[1]; fp.o_sh = p.o_stride[2];
     fp.o_fp32 = (p.o_dtype == FA_DTYPE_FP32) ? 1 : 0;
     fp.n_qtiles = (p.Sq + fa::kTile - 1) / fa::kTile;

@@ -486,12 +486,16 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 const int kv0 = j * kTile;
                 const bool need_mask = (p.causal && kv0 + kTile - 1 > q0 + off) || (kv0 + kTile > p.Skv);
                 if (need_mask) {
+                    // tiles crossed by the diagonal or by the end of the keys: hidden scores
+                    // become -inf (the scale is strictly positive, so they come out as exact
+                    // zeros) and the tile then takes the common path
                     int lim = p.Skv - kv0;
                     if (p.causal) lim = min(lim, row + off - kv0 + 1);
-                    softmax_step<T, true>(s, tS, tO, p.scale_log2, lim, j == 0, m_ref, l_run);
-                } else {
-                    softmax_step<T, false>(s, tS, tO, p.scale_log2, 128, j == 0, m_ref, l_run);
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i >= lim) s[i] = 0xff800000u;
                 }
+                softmax_step<T, false>(s, tS, tO, p.scale_log2, 128, j == 0, m_ref, l_run);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
