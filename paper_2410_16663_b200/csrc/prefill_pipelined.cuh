@@ -67,9 +67,15 @@ struct Item {
 // this sequence with its own copy of `lead`.
 __device__ __forceinline__ Item decode_item(const FwdParams& p, int idx, int n_qpairs, int& lead) {
     Item it;
+    // Item order.  Normally the longest (last) query tile pairs of all heads come first, which
+    // balances the CTAs best.  When one head alone has at least one round of items for every
+    // CTA (very long sequences, whose K and V per head no longer fit in L2), the list goes head
+    // by head instead: all CTAs then walk the same head's K/V at about the same pace and share
+    // it through L2 rather than each streaming its own head from HBM.
     const int bh_count = p.B * p.Hq;
-    const int qp = n_qpairs - 1 - idx / bh_count;  // long (late) query tiles first
-    const int bh = idx % bh_count;
+    const bool head_major = n_qpairs >= (int)gridDim.x;
+    const int qp = n_qpairs - 1 - (head_major ? idx % n_qpairs : idx / bh_count);  // long (late) tiles first
+    const int bh = head_major ? idx / n_qpairs : idx % bh_count;
     it.b = bh / p.Hq;
     it.h = bh % p.Hq;
     it.hk = it.h / (p.Hq / p.Hkv);
