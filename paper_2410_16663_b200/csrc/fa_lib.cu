@@ -10,6 +10,7 @@
 #include <string.h>
 
 #include "decode.cuh"
+#include "prefill_pingpong.cuh"
 #include "prefill_pipelined.cuh"
 #include "prefill_simple.cuh"
 
@@ -190,6 +191,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         case 2:  // simple kernel, P handed over through shared memory
             return bf16 ? launch_simple<__nv_bfloat16, false>(tq, tk, tv, fp, st)
                         : launch_simple<__half, false>(tq, tk, tv, fp, st);
+        case 3:  // ping-pong kernel: one query tile per CTA, two softmax warpgroups alternate over kv steps
+            return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
+                        : fa::launch_pingpong<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
         default:
             return FA_ERR_UNSUPPORTED;
     }

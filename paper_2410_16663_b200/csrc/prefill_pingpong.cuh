@@ -1,0 +1,597 @@
+// Prefill forward, ping-pong variant.
+//
+// A persistent CTA (one per SM, 384 threads) walks a static list of work items; an item is one
+// 128-row query tile of one (batch, head).  The kv steps of the CTA are numbered g = 0, 1, 2, ...
+// across items, and everything a step needs is double-buffered on the parity of g:
+//   tensor memory : O [0,128)   S_0 [128,256)  S_1 [256,384)  P_0 [384,448)  P_1 [448,512)
+//   warpgroup g&1 : softmax of step g, one thread per query row: reads S_{g&1}, keeps its part
+//                   of the row sum, writes P (16-bit, packed) to P_{g&1}.
+//   warp 8        : one thread issues S_{g&1} = Q K_g^T for every step, as soon as K_g has
+//                   landed and the softmax of step g-2 has read its scores out of the buffer.
+//   warp 10       : one thread issues O += P_{g&1} V_g for every step, as soon as P is written.
+//   warp 9 / 11   : one thread each issues the TMA loads of Q and K / of V (separate rings, as
+//                   K is consumed about two steps ahead of V).
+// Because P has columns of its own, Q K^T of step g+1 and g+2 run on the tensor core while the
+// softmax of step g is still at work: the tensor core never waits for a softmax of the same
+// tile (the Cube/Vector overlap of Section 4.1 within one query tile), and the two warpgroups
+// give the exponentials two steps of time per step of tensor work.
+//
+// The online-softmax recurrence (Appendix A) is carried from step to step through shared
+// memory: the warpgroup of step g takes the reference max left by step g-1, decides whether its
+// own row max moves it (only when it outgrew it by more than 2^8, see kRescaleThreshold),
+// publishes the result for step g+1 right away, and, in the rare case that it moved, rescales O
+// once O += P V of step g-1 has completed.  Each warpgroup keeps the row sum of its own steps;
+// the one that runs an item's last step adds the other's and writes O and LSE.
+// Synchronisation is mbarrier-only; every wait is bounded (see mbar_wait).
+#pragma once
+
+#include <type_traits>
+
+#include "prefill_pipelined.cuh"
+
+namespace fa {
+
+#ifndef FA_PP_NK
+#define FA_PP_NK 3
+#endif
+#ifndef FA_PP_NV
+#define FA_PP_NV 2
+#endif
+constexpr int kPpNK = FA_PP_NK;   // K ring slots
+constexpr int kPpNV = FA_PP_NV;   // V ring slots
+constexpr int kPpQBufs = 2;
+#ifndef FA_PP_TURNS
+#define FA_PP_TURNS 0
+#endif
+constexpr bool kPpTurns = FA_PP_TURNS != 0;
+static_assert((kPpQBufs + kPpNK + kPpNV) * kTileBytes + 3072 <= 232448, "shared memory budget");
+
+// ---- barriers: indices into one array
+namespace ppb {
+constexpr int q_full = 0;                       // [2]  TMA -> S thread
+constexpr int q_empty = 2;                      // [2]  S thread (commit) -> loader
+constexpr int k_full = 4;                       // [NK]
+constexpr int k_empty = k_full + kPpNK;         // [NK]
+constexpr int v_full = k_empty + kPpNK;         // [NV]
+constexpr int v_empty = v_full + kPpNV;         // [NV]
+constexpr int s_full = v_empty + kPpNV;         // [2]  S thread (commit) -> softmax
+constexpr int pv_done = s_full + 2;             // [2]  PV thread (commit) -> softmax
+constexpr int o_final = pv_done + 2;            // [2]  PV thread (commit) -> epilogue, by item parity
+// barriers every thread of a softmax warpgroup arrives on (count 128)
+constexpr int p_full = o_final + 2;             // [2]  softmax -> PV thread
+constexpr int m_ready = p_full + 2;             // [2]  softmax of step g -> softmax of step g+1 (reference max
+                                                //      published) and -> S thread (scores read out of S_{g&1})
+constexpr int l_pub = m_ready + 2;              // [2]  softmax of an item's last-but-one step -> of its last step
+constexpr int o_free = l_pub + 2;               // [1]  epilogue -> PV thread
+constexpr int count = o_free + 1;
+}  // namespace ppb
+
+struct PpStatic {
+    uint64_t bars[ppb::count];
+    uint32_t tmem_holder;
+    uint32_t abort_flag;
+    float m_xch[2][128];   // [warpgroup][row]: reference max after that warpgroup's latest step
+    float l_xch[2][128];   // [item parity][row]: row sum of the warpgroup that does not run the last step
+    uint8_t pad[3072 - ppb::count * 8 - 8 - 4 * 128 * 4];
+};
+static_assert(sizeof(PpStatic) == 3072, "static shared state must fill exactly 3 KiB");
+
+struct PpItem {
+    int b, h, hk, q0, n;
+};
+
+// Work item `idx`: longest (latest) query tiles of all heads first; head by head when one head
+// alone has a round of items for every CTA (see decode_item in the pipelined kernel).
+__device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
+    PpItem it;
+    const int bh_count = p.B * p.Hq;
+    const bool head_major = p.n_qtiles >= (int)gridDim.x;
+    const int qt = p.n_qtiles - 1 - (head_major ? idx % p.n_qtiles : idx / bh_count);
+    const int bh = head_major ? idx / p.n_qtiles : idx % bh_count;
+    it.b = bh / p.Hq;
+    it.h = bh % p.Hq;
+    it.hk = it.h / (p.Hq / p.Hkv);
+    it.q0 = qt * kTile;
+    it.n = kv_tiles_for(it.q0, kTile, p.Sq, p.Skv, p.causal);
+    return it;
+}
+
+// Row max of 128 raw scores.
+__device__ __forceinline__ float pp_row_max(const uint32_t (&s)[128]) {
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 128; i += 8) {
+        m0 = max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        m1 = max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        m2 = max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        m3 = max3(m3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// exp2(s * scale_log2 + neg_ms) of 32 scores -> 16 packed 16-bit pairs; adds them to (la, lb).
+template <typename T>
+__device__ __forceinline__ void pp_exp_chunk(const uint32_t (&s)[128], int c, uint64_t sc2, uint64_t nm2,
+                                             uint64_t& la, uint64_t& lb, uint32_t (&pk)[16]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        const int e = c * 32 + i;
+        float pv[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint64_t x01 =
+                f2_fma(f2_pack(__uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1])), sc2, nm2);
+            float x0, x1;
+            f2_unpack(x01, x0, x1);
+            if (q < kPolyPairs) {
+                exp2_poly_pair(fmaxf(x0, -125.f), fmaxf(x1, -125.f), pv[2 * q], pv[2 * q + 1]);
+            } else {
+                pv[2 * q] = fast_exp2(x0);
+                pv[2 * q + 1] = fast_exp2(x1);
+            }
+        }
+        la = f2_add(la, f2_pack(pv[0], pv[1]));
+        lb = f2_add(lb, f2_pack(pv[2], pv[3]));
+        la = f2_add(la, f2_pack(pv[4], pv[5]));
+        lb = f2_add(lb, f2_pack(pv[6], pv[7]));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) pk[i / 2 + q] = pack2<T>(pv[2 * q], pv[2 * q + 1]);
+    }
+}
+
+__device__ __forceinline__ uint32_t pp_bar(uint32_t bar0, int i) { return bar0 + 8 * i; }
+
+// Ring cursor: slot and phase parity of the g-th entry of a ring of N slots.
+template <int N>
+struct PpRing {
+    uint32_t slot = 0, par = 0;
+    __device__ __forceinline__ void next() {
+        if (++slot == N) {
+            slot = 0;
+            par ^= 1;
+        }
+    }
+};
+
+// The thread that issues S = Q K^T of every step.
+template <typename T>
+__device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK, uint32_t tmem, const FwdParams& p,
+                                         int total_items, volatile uint32_t* abort_flag) {
+    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, false);
+    uint32_t g = 0;
+    PpRing<kPpNK> ring;
+    for (int ord = 0;; ++ord) {
+        const int idx = item_of_round(ord, total_items);
+        if (idx >= total_items) break;
+        const PpItem it = pp_decode_item(p, idx);
+        const uint32_t qb = ord & 1;
+        if (!mbar_wait(pp_bar(bar0, ppb::q_full + qb), (ord >> 1) & 1, abort_flag, 130)) return;
+        const uint32_t a_lo = desc_lo(sQ + qb * kTileBytes, 16);
+        for (int j = 0; j < it.n; ++j, ++g, ring.next()) {
+            const uint32_t buf = g & 1;
+            if (!mbar_wait(pp_bar(bar0, ppb::k_full + ring.slot), ring.par, abort_flag, 131)) return;
+            // the softmax of step g-2 has read its scores out of this buffer (it says so together
+            // with its reference max)
+            if (g >= 2 && !mbar_wait(pp_bar(bar0, ppb::m_ready + buf), ((g >> 1) - 1) & 1, abort_flag, 132)) return;
+            tc_fence_after();
+            const uint32_t b_lo = desc_lo(sK + ring.slot * kTileBytes, 16);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t koff = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                mma_ss_lo(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
+            }
+            mma_commit(pp_bar(bar0, ppb::s_full + buf));
+            mma_commit(pp_bar(bar0, ppb::k_empty + ring.slot));
+            if (j == it.n - 1) mma_commit(pp_bar(bar0, ppb::q_empty + qb));
+        }
+    }
+}
+
+// The thread that issues O += P V of every step.
+template <typename T>
+__device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t tmem, const FwdParams& p,
+                                          int total_items, volatile uint32_t* abort_flag) {
+    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, true);
+    uint32_t g = 0;
+    PpRing<kPpNV> ring;
+    for (int ord = 0;; ++ord) {
+        const int idx = item_of_round(ord, total_items);
+        if (idx >= total_items) break;
+        const PpItem it = pp_decode_item(p, idx);
+        for (int j = 0; j < it.n; ++j, ++g, ring.next()) {
+            const uint32_t buf = g & 1;
+            if (!mbar_wait(pp_bar(bar0, ppb::v_full + ring.slot), ring.par, abort_flag, 140)) return;
+            // the previous item's epilogue has read O out of tensor memory
+            if (j == 0 && ord > 0 && !mbar_wait(pp_bar(bar0, ppb::o_free), (ord - 1) & 1, abort_flag, 141)) return;
+            if (!mbar_wait(pp_bar(bar0, ppb::p_full + buf), (g >> 1) & 1, abort_flag, 142)) return;
+            tc_fence_after();
+            const uint32_t b_lo = desc_lo(sV + ring.slot * kTileBytes, kHalfBytes);  // V: N-major, 16 kv rows per step
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                mma_ts_lo(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (2048 >> 4), idesc,
+                          (ks > 0) ? 1u : (j > 0 ? 1u : 0u));
+            mma_commit(pp_bar(bar0, ppb::pv_done + buf));
+            mma_commit(pp_bar(bar0, ppb::v_empty + ring.slot));
+            if (j == it.n - 1) mma_commit(pp_bar(bar0, ppb::o_final + (ord & 1)));
+        }
+    }
+}
+
+// The thread that loads Q of every item and K of every step.
+__device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint32_t sK, const CUtensorMap* tm_q,
+                                               const CUtensorMap* tm_k, const FwdParams& p, int total_items,
+                                               volatile uint32_t* abort_flag) {
+    tma_prefetch_desc(tm_q);
+    tma_prefetch_desc(tm_k);
+    PpRing<kPpNK> ring;
+    for (int ord = 0;; ++ord) {
+        const int idx = item_of_round(ord, total_items);
+        if (idx >= total_items) break;
+        const PpItem it = pp_decode_item(p, idx);
+        const uint32_t qb = ord & 1;
+        // passes at once the first time each buffer is used
+        if (!mbar_wait(pp_bar(bar0, ppb::q_empty + qb), ((ord >> 1) & 1) ^ 1, abort_flag, 150)) return;
+        mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
+        load_tile(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h, it.q0, it.b);
+        for (int j = 0; j < it.n; ++j, ring.next()) {
+            if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
+            mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
+            load_tile(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, j * kTile, it.b);
+        }
+    }
+}
+
+// The thread that loads V of every step.
+__device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const CUtensorMap* tm_v, const FwdParams& p,
+                                              int total_items, volatile uint32_t* abort_flag) {
+    tma_prefetch_desc(tm_v);
+    PpRing<kPpNV> ring;
+    for (int ord = 0;; ++ord) {
+        const int idx = item_of_round(ord, total_items);
+        if (idx >= total_items) break;
+        const PpItem it = pp_decode_item(p, idx);
+        for (int j = 0; j < it.n; ++j, ring.next()) {
+            if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
+            mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
+            load_tile(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, j * kTile, it.b);
+        }
+    }
+}
+
+// Warp-wide wait: every lane waits, and the warp leaves together if any lane gave up (the
+// tensor-memory instructions that follow need the whole warp).
+__device__ __forceinline__ bool pp_warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                             unsigned int where) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, where);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// One thread of a softmax warpgroup: its state across the steps of an item, and the step.
+template <typename T>
+struct PpSoftmax {
+    // fixed for the kernel
+    uint32_t bar0;
+    volatile uint32_t* abort_flag;
+    float* m_mine;          // this row's slot in the reference-max exchange, written by this warpgroup
+    const float* m_other;   // the same row's slot written by the other warpgroup
+    int w;                  // warpgroup: runs the steps with g & 1 == w
+    uint32_t tO, tS, tP;    // this warp's lane quarter of O, S_w, P_w in tensor memory
+    float scale_log2;
+    int causal, Skv, off;
+    // per item
+    int row;                // query row of this thread
+    float l_part;           // row sum over this warpgroup's steps, relative to m_loc
+    float m_loc;            // reference max after this warpgroup's latest step
+    float m_before;         // reference max that step received from the step before it
+
+    // Step g of the CTA = step j of the item.  kMasked: the tile is crossed by the diagonal or by
+    // the end of the keys.  Returns false when a wait gave up.
+    template <bool kMasked>
+    __device__ __forceinline__ bool step(uint32_t (&s)[128], uint32_t g, int j) {
+        if (!pp_warp_wait(pp_bar(bar0, ppb::s_full + w), (g >> 1) & 1, abort_flag, 110 + w)) return false;
+        tc_fence_after();
+        tmem_ld_x32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+        tmem_ld_x32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+        tmem_ld_x32(tS + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
+        tmem_ld_x32(tS + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+        tmem_wait_ld();
+        tc_fence_before();  // for the arrival below that hands the S buffer back
+        // probe early, look at the answer after the row max
+        const bool m_there = g > 0 && mbar_test(pp_bar(bar0, ppb::m_ready + (1 - w)), ((g - 1) >> 1) & 1);
+        if (kMasked) {
+            // hidden scores become -inf (the scale is strictly positive, so they come out as exact zeros)
+            const int kv0 = j * kTile;
+            int lim = Skv - kv0;
+            if (causal) lim = min(lim, row + off - kv0 + 1);
+#pragma unroll
+            for (int i = 0; i < 128; ++i)
+                if (i >= lim) s[i] = 0xff800000u;
+        }
+        const float mx = pp_row_max(s);
+        // reference max left by step g-1 (of the other warpgroup); an item starts afresh
+        float m_prev = -INFINITY;
+        if (g > 0) {
+            if (!__all_sync(0xffffffffu, m_there) &&
+                !pp_warp_wait(pp_bar(bar0, ppb::m_ready + (1 - w)), ((g - 1) >> 1) & 1, abort_flag, 112 + w))
+                return false;
+            if (j > 0) m_prev = *m_other;
+        }
+        m_before = m_prev;
+        // lazy reference update: the reference moves only when the row max outgrew it by more than
+        // the threshold (always on the first visible score; never on -inf)
+        const bool grow = (mx - m_prev) * scale_log2 > kRescaleThreshold;
+        const float m_new = grow ? mx : m_prev;
+        *m_mine = m_new;
+        // one arrival per thread: publishes its reference max and, the scores being in registers,
+        // lets Q K^T of step g+2 overwrite the S buffer
+        mbar_arrive(pp_bar(bar0, ppb::m_ready + w));
+        if (m_loc != m_new) {  // this warpgroup's row sum follows the reference
+            if (l_part > 0.f) l_part *= fast_exp2((m_loc - m_new) * scale_log2);
+            m_loc = m_new;
+        }
+        const float neg_ms = -((m_new == -INFINITY) ? 0.f : m_new) * scale_log2;
+        const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
+        uint64_t la = f2_pack(0.f, 0.f), lb = la;
+        if (kPpTurns && g >= 1) {
+            // the two warpgroups take turns at the exponentials
+            if (!pp_warp_wait(pp_bar(bar0, ppb::p_full + (1 - w)), ((g - 1) >> 1) & 1, abort_flag, 122 + w)) return false;
+        }
+        {
+            uint32_t pk[16];
+            const bool p_free = g < 2 || mbar_test(pp_bar(bar0, ppb::pv_done + w), ((g >> 1) - 1) & 1);
+            pp_exp_chunk<T>(s, 0, sc2, nm2, la, lb, pk);
+            if (g >= 2) {
+                // O += P V of step g-2 has read this P buffer
+                if (!__all_sync(0xffffffffu, p_free) &&
+                    !pp_warp_wait(pp_bar(bar0, ppb::pv_done + w), ((g >> 1) - 1) & 1, abort_flag, 116 + w))
+                    return false;
+                tc_fence_after();
+            }
+            if (__builtin_expect(j > 0 && __any_sync(0xffffffffu, grow), 0)) {
+                // rare: the reference moved.  O holds the P V sums up to step g-1 once that step's
+                // MMAs have completed (those of step g-2 have, see above, so the parity wait on the
+                // other buffer's barrier is one phase at most behind).
+                if (!pp_warp_wait(pp_bar(bar0, ppb::pv_done + (1 - w)), ((g - 1) >> 1) & 1, abort_flag, 114 + w)) return false;
+                tc_fence_after();
+                const float alpha = grow ? ((m_prev == -INFINITY) ? 0.f : fast_exp2((m_prev - mx) * scale_log2)) : 1.f;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t o[16];
+                    tmem_ld_x16(tO + c * 16, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_x16(tO + c * 16, o);
+                }
+            }
+            tmem_st_x16(tP, pk);
+        }
+#pragma unroll
+        for (int c = 1; c < 4; ++c) {
+            uint32_t pk[16];
+            pp_exp_chunk<T>(s, c, sc2, nm2, la, lb, pk);
+            tmem_st_x16(tP + c * 16, pk);
+        }
+        {
+            float a0, a1, b0, b1;
+            f2_unpack(la, a0, a1);
+            f2_unpack(lb, b0, b1);
+            l_part += (a0 + a1) + (b0 + b1);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(pp_bar(bar0, ppb::p_full + w));
+        return true;
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kPipeThreads, 1)
+fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, const FwdParams p, const int total_items) {
+    // Shared memory is used to the last byte: 3 KiB of static state (sized so that the dynamic
+    // part that follows it starts on a 1024-byte boundary, which the 128-byte swizzle needs)
+    // plus seven 32 KiB tiles.  The alignment is checked rather than assumed.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(1024) PpStatic ss;
+    const uint32_t smem_base = smem_u32(smem_raw);
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + kPpQBufs * kTileBytes;
+    const uint32_t sV = sK + kPpNK * kTileBytes;
+    const uint32_t bar0 = smem_u32(&ss.bars[0]);
+    volatile uint32_t* abort_flag = &ss.abort_flag;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    if (smem_base & 1023u) {  // uniform for the CTA: nothing has been set up yet
+        if (tid == 0) record_timeout(900);
+        return;
+    }
+    if (tid == 0) {
+        for (int i = 0; i < ppb::count; ++i) {
+            mbar_init(pp_bar(bar0, i), i >= ppb::p_full ? 128 : 1);
+        }
+        ss.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(smem_u32(&ss.tmem_holder), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ss.tmem_holder;
+    const int off = p.Skv - p.Sq;
+
+    if (warp < 8) {
+        // ================================================================ softmax + epilogue
+        setmaxnreg_inc<kPipeSoftmaxRegs>();  // a whole row of S lives in registers
+        const int w = warp >> 2;             // this warpgroup runs the steps with g & 1 == w
+        const int r = tid & 127;
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tO = tmem_base + lane_sel;
+        const uint32_t tS = tmem_base + lane_sel + 128 + 128 * w;
+        const uint32_t tP = tmem_base + lane_sel + 384 + 64 * w;
+        const float scale_log2 = p.scale_log2;
+        PpSoftmax<T> sm;
+        sm.bar0 = bar0;
+        sm.abort_flag = abort_flag;
+        sm.m_mine = &ss.m_xch[w][r];
+        sm.m_other = &ss.m_xch[1 - w][r];
+        sm.w = w;
+        sm.tO = tO;
+        sm.tS = tS;
+        sm.tP = tP;
+        sm.scale_log2 = scale_log2;
+        sm.causal = p.causal;
+        sm.Skv = p.Skv;
+        sm.off = off;
+        uint32_t g = 0;        // step counter of the CTA
+        uint32_t items2 = 0;   // items with at least two steps seen so far
+        bool ok = true;
+        for (int ord = 0; ok; ++ord) {
+            const int idx = item_of_round(ord, total_items);
+            if (idx >= total_items) break;
+            const PpItem it = pp_decode_item(p, idx);
+            const int n = it.n;
+            const int row = it.q0 + r;
+            sm.row = row;
+            sm.l_part = 0.f;
+            sm.m_loc = -INFINITY;
+            sm.m_before = -INFINITY;
+            uint32_t s[128];             // this thread's row of S, later of O
+            const uint32_t xb = items2 & 1, xpar = (items2 >> 1) & 1;  // row-sum exchange buffer / phase
+            // kv tiles every row of the query tile sees in full: they come first and take the
+            // loop without mask code; the few tiles crossed by the diagonal or by the end of the
+            // keys follow
+            int n_full = p.Skv / kTile;
+            if (p.causal) n_full = min(n_full, max(0, (it.q0 + off + 1) / kTile));
+            n_full = min(n_full, n);
+            // this warpgroup's steps of the item: those with an absolute step number of its parity
+            const uint32_t g_item = g;
+            int j = (int)((g_item ^ (uint32_t)w) & 1u);
+            for (; j < n_full && ok; j += 2) {
+                ok = sm.template step<false>(s, g_item + (uint32_t)j, j);
+                if (ok && j == n - 2) {
+                    // the other warpgroup runs the last step and the epilogue: hand it this row sum
+                    // (it is relative to the reference this step left, which that step receives)
+                    ss.l_xch[xb][r] = sm.l_part;
+                    mbar_arrive(pp_bar(bar0, ppb::l_pub + xb));
+                }
+            }
+            for (; j < n && ok; j += 2) {
+                ok = sm.template step<true>(s, g_item + (uint32_t)j, j);
+                if (ok && j == n - 2) {
+                    ss.l_xch[xb][r] = sm.l_part;
+                    mbar_arrive(pp_bar(bar0, ppb::l_pub + xb));
+                }
+            }
+            const float l_part = sm.l_part, m_loc = sm.m_loc, m_before = sm.m_before;
+            if (ok && ((g_item + (uint32_t)n - 1u) & 1u) == (uint32_t)w) {
+                // ---- epilogue of the item, by the warpgroup that ran its last step
+                float l_run = l_part;
+                if (n >= 2) {
+                    ok = pp_warp_wait(pp_bar(bar0, ppb::l_pub + xb), xpar, abort_flag, 118 + w);
+                    if (!ok) break;
+                    const float l_other = ss.l_xch[xb][r];
+                    // the other warpgroup's sum is relative to the reference this one's last step received
+                    if (l_other > 0.f) l_run += l_other * fast_exp2((m_before - m_loc) * scale_log2);
+                }
+                ok = pp_warp_wait(pp_bar(bar0, ppb::o_final + (ord & 1)), (ord >> 1) & 1, abort_flag, 120 + w);
+                if (!ok) break;
+                tc_fence_after();
+                tmem_ld_x32(tO, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                tmem_ld_x32(tO + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                tmem_ld_x32(tO + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
+                tmem_ld_x32(tO + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+                tmem_wait_ld();
+                // O is in registers: the next item's first P V may overwrite it
+                tc_fence_before();
+                mbar_arrive(pp_bar(bar0, ppb::o_free));
+                const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+                if (row < p.Sq) {
+                    const long long obase =
+                        (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
+                    if (p.o_fp32) {
+                        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            dst[i] = make_float4(__uint_as_float(s[4 * i]) * inv_l, __uint_as_float(s[4 * i + 1]) * inv_l,
+                                                 __uint_as_float(s[4 * i + 2]) * inv_l,
+                                                 __uint_as_float(s[4 * i + 3]) * inv_l);
+                    } else {
+                        T* dst = static_cast<T*>(p.o) + obase;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t v[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                v[i] = pack2<T>(__uint_as_float(s[c * 16 + 2 * i]) * inv_l,
+                                                __uint_as_float(s[c * 16 + 2 * i + 1]) * inv_l);
+                            if (p.o_align32) {
+                                // 32-byte stores: every instruction writes whole 32-byte sectors
+                                st_global_v8(dst + c * 16, v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]);
+                            } else {
+                                reinterpret_cast<uint4*>(dst + c * 16)[0] = make_uint4(v[0], v[1], v[2], v[3]);
+                                reinterpret_cast<uint4*>(dst + c * 16)[1] = make_uint4(v[4], v[5], v[6], v[7]);
+                            }
+                        }
+                    }
+                    if (p.lse != nullptr) {
+                        const float lse = (l_run > 0.f)
+                                              ? (m_loc * scale_log2 + log2f(l_run)) * 0.6931471805599453f
+                                              : -INFINITY;
+                        p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
+                    }
+                }
+            }
+            g = g_item + (uint32_t)n;
+            if (n >= 2) ++items2;
+        }
+    } else {
+        setmaxnreg_dec<kPipeOtherRegs>();
+        if (lane == 0) {
+            if (warp == 8) pp_run_s<T>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
+            else if (warp == 10) pp_run_pv<T>(bar0, sV, tmem_base, p, total_items, abort_flag);
+            else if (warp == 9) pp_run_load_qk(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
+            else pp_run_load_v(bar0, sV, &tm_v, p, total_items, abort_flag);
+        }
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+template <typename T>
+int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& fp,
+                    cudaStream_t st, int* cuda_err) {
+    constexpr int smem = (kPpQBufs + kPpNK + kPpNV) * kTileBytes;
+    auto kern = fa_fwd_pingpong_kernel<T>;
+    static int sm_count = 0;
+    cudaError_t e;
+    if (sm_count == 0) {
+        int dev = 0, n = 0;
+        if ((e = cudaGetDevice(&dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
+        sm_count = n;
+    }
+    const long long total = (long long)fp.n_qtiles * fp.B * fp.Hq;
+    if (total > 0x7fffffffll) return -3;
+    const int grid = (int)(total < sm_count ? total : sm_count);
+    kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, fp, (int)total);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { *cuda_err = (int)e; return -7; }
+    return 0;
+}
+
+}  // namespace fa

@@ -60,7 +60,7 @@ def full_case(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed, variant=0, scale=Non
 
 
 # ------------------------------------------------------------------ C1: the small benchmark config
-@pytest.mark.parametrize("variant", [0, 1, 2])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
 def test_c1_full_tensor(fa, variant):
     c = synth.C1
     q, k, v = synth.prefill_inputs(c, "cpu")
@@ -115,10 +115,38 @@ def test_head_grouping(fa, hq, hkv):
     full_case(fa, 2, hq, hkv, 200, 333, True, "fp16", seed=hq * 10 + hkv)
 
 
-@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("variant", [1, 2, 3])
 def test_alternate_kernels_on_ragged_shapes(fa, variant):
     full_case(fa, 2, 4, 2, 257, 1000, True, "fp16", seed=77, variant=variant)
     full_case(fa, 1, 2, 2, 129, 385, False, "bf16", seed=78, variant=variant)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", [(1, 1), (127, 127), (128, 128), (129, 129), (256, 256), (257, 257), (1000, 1000),
+                                    (1, 129), (17, 1000), (128, 384), (100, 257), (257, 1000)])
+def test_pingpong_kernel_shape_grid(fa, sq, skv, causal):
+    full_case(fa, 1, 2, 2, sq, skv, causal, "fp16", seed=sq * 1000 + skv + 7, variant=3)
+
+
+def test_pingpong_kernel_many_items_per_cta(fa):
+    # more query tiles than CTAs, of one to five kv steps each: every CTA strings several items
+    # together, odd and even step counts, through both warpgroups
+    full_case(fa, 2, 160, 8, 640, 640, True, "bf16", seed=91, variant=3)
+    full_case(fa, 3, 64, 64, 300, 300, True, "fp16", seed=92, variant=3)
+    full_case(fa, 2, 100, 20, 129, 700, False, "fp16", seed=93, variant=3)
+
+
+def test_pingpong_kernel_peaked_rows_rescale(fa):
+    # keys whose norm grows along the sequence: the running max keeps moving, O is rescaled often
+    torch.manual_seed(5)
+    B, H, S = 1, 2, 1024
+    q = torch.randn(B, S, H, 128).half()
+    k = (torch.randn(B, S, H, 128) * torch.linspace(0.2, 6.0, S).view(1, S, 1, 1)).half()
+    v = torch.randn(B, S, H, 128).half()
+    for causal in (False, True):
+        o_ref, l_ref = oracle.attention_full(q, k, v, causal, 1.0)
+        o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, 1.0, variant=3)
+        assert_close_to_oracle(o, lse, o_ref, l_ref, what=f"peaked causal={causal}", stored_fp16_ulp=True)
 
 
 def test_scale_zero_and_large_scale(fa):
