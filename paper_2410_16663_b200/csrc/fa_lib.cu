@@ -181,8 +181,13 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16);
     if (rc) return rc;
 
-    switch (p.variant) {
-        case 0:  // pipelined, warp-specialised kernel
+    // Default choice, from timings of both kernels on B200: the ping-pong kernel (one query tile
+    // per CTA, Q K^T running ahead of the softmax) wins once an item has many kv steps; the
+    // paired-tile kernel keeps a small edge on short sequences, where items change every few steps.
+    int variant = p.variant;
+    if (variant == 0) variant = (p.Skv >= 4096) ? 3 : 4;
+    switch (variant) {
+        case 4:  // pipelined kernel, two query tiles per CTA
             return bf16 ? fa::launch_pipelined<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
                         : fa::launch_pipelined<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
         case 1:  // simple kernel, P handed over through tensor memory

@@ -60,7 +60,7 @@ def full_case(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed, variant=0, scale=Non
 
 
 # ------------------------------------------------------------------ C1: the small benchmark config
-@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4])
 def test_c1_full_tensor(fa, variant):
     c = synth.C1
     q, k, v = synth.prefill_inputs(c, "cpu")
