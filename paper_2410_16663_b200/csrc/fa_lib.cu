@@ -160,6 +160,11 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.o_sb = p.o_stride[0]; fp.o_ss = p.o_stride[1]; fp.o_sh = p.o_stride[2];
     fp.o_fp32 = (p.o_dtype == FA_DTYPE_FP32) ? 1 : 0;
     fp.n_qtiles = (p.Sq + fa::kTile - 1) / fa::kTile;
+    fp.by_bh.set(p.B * p.Hq);
+    fp.by_hq.set(p.Hq);
+    fp.by_group.set(p.Hq / p.Hkv);
+    fp.by_qtiles.set(fp.n_qtiles > 0 ? fp.n_qtiles : 1);
+    fp.by_qpairs.set(fp.n_qtiles > 0 ? (fp.n_qtiles + 1) / 2 : 1);
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
     const bool bf16 = p.dtype == FA_DTYPE_BF16;

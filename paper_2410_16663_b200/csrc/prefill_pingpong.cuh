@@ -84,13 +84,14 @@ struct PpItem {
 // alone has a round of items for every CTA (see decode_item in the pipelined kernel).
 __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
     PpItem it;
-    const int bh_count = p.B * p.Hq;
     const bool head_major = p.n_qtiles >= (int)gridDim.x;
-    const int qt = p.n_qtiles - 1 - (head_major ? idx % p.n_qtiles : idx / bh_count);
-    const int bh = head_major ? idx / p.n_qtiles : idx % bh_count;
-    it.b = bh / p.Hq;
-    it.h = bh % p.Hq;
-    it.hk = it.h / (p.Hq / p.Hkv);
+    int major, minor;  // idx = major * (inner count) + minor
+    if (head_major) p.by_qtiles.divmod(idx, major, minor);
+    else p.by_bh.divmod(idx, major, minor);
+    const int qt = p.n_qtiles - 1 - (head_major ? minor : major);
+    const int bh = head_major ? major : minor;
+    p.by_hq.divmod(bh, it.b, it.h);
+    it.hk = p.by_group.div(it.h);
     it.q0 = qt * kTile;
     it.n = kv_tiles_for(it.q0, kTile, p.Sq, p.Skv, p.causal);
     return it;

@@ -72,13 +72,14 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int idx, int n_q
     // CTA (very long sequences, whose K and V per head no longer fit in L2), the list goes head
     // by head instead: all CTAs then walk the same head's K/V at about the same pace and share
     // it through L2 rather than each streaming its own head from HBM.
-    const int bh_count = p.B * p.Hq;
     const bool head_major = n_qpairs >= (int)gridDim.x;
-    const int qp = n_qpairs - 1 - (head_major ? idx % n_qpairs : idx / bh_count);  // long (late) tiles first
-    const int bh = head_major ? idx / n_qpairs : idx % bh_count;
-    it.b = bh / p.Hq;
-    it.h = bh % p.Hq;
-    it.hk = it.h / (p.Hq / p.Hkv);
+    int major, minor;  // idx = major * (inner count) + minor
+    if (head_major) p.by_qpairs.divmod(idx, major, minor);
+    else p.by_bh.divmod(idx, major, minor);
+    const int qp = n_qpairs - 1 - (head_major ? minor : major);  // long (late) tiles first
+    const int bh = head_major ? major : minor;
+    p.by_hq.divmod(bh, it.b, it.h);
+    it.hk = p.by_group.div(it.h);
     const int q_lo = qp * 2 * kTile;
     const int n_lo = kv_tiles_for(q_lo, kTile, p.Sq, p.Skv, p.causal);
     // a second tile that starts past the last row still runs (on zero-filled rows, never

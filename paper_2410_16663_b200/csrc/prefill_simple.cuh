@@ -14,6 +14,28 @@
 
 namespace fa {
 
+// Division of a non-negative 32-bit integer by a divisor fixed at launch time, as a multiply and
+// a shift: the persistent kernels turn a work item's index into (batch, head, tile) with it.
+// With s = ceil(log2 d) and M = floor(2^(31+s) / d) + 1, floor(n * M / 2^(31+s)) = floor(n / d)
+// for every 0 <= n < 2^31 (the excess of M over 2^(31+s)/d adds less than 1/d to the quotient).
+struct FastDiv {
+    uint32_t mul, shift, d;
+    __host__ void set(int divisor) {
+        d = static_cast<uint32_t>(divisor);
+        uint32_t s = 0;
+        while ((1ull << s) < d) ++s;
+        shift = 31 + s;
+        mul = static_cast<uint32_t>((1ull << shift) / d + 1);
+    }
+    __device__ __forceinline__ int div(int n) const {
+        return static_cast<int>((static_cast<unsigned long long>(static_cast<uint32_t>(n)) * mul) >> shift);
+    }
+    __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
+        q = div(n);
+        r = n - q * static_cast<int>(d);
+    }
+};
+
 struct FwdParams {
     void* o;
     float* lse;
@@ -24,6 +46,7 @@ struct FwdParams {
     int o_fp32;
     int n_qtiles;
     int o_align32;  // o and its strides are 32-byte aligned: rows can be written with 256-bit stores
+    FastDiv by_bh, by_hq, by_group, by_qtiles, by_qpairs;  // B*Hq, Hq, Hq/Hkv, n_qtiles, ceil(n_qtiles/2)
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim
