@@ -514,9 +514,20 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 tc_fence_before();
                 mbar_arrive(pp_bar(bar0, ppb::o_free));
                 const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-                if (row < p.Sq) {
-                    const long long obase =
-                        (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
+                const long long obase = (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
+                if (row < p.Sq && p.lse != nullptr) {
+                    const float lse = (l_run > 0.f) ? (m_loc * scale_log2 + log2f(l_run)) * 0.6931471805599453f
+                                                    : -INFINITY;
+                    p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
+                }
+                if (!p.o_fp32 && p.o_align32) {
+                    // 16-bit output, rows 32-byte aligned: whole-line stores through a lane exchange
+                    uint32_t wv[64];
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        wv[i] = pack2<T>(__uint_as_float(s[2 * i]) * inv_l, __uint_as_float(s[2 * i + 1]) * inv_l);
+                    store_rows_coalesced<T>(static_cast<T*>(p.o) + obase, p.o_ss, p.Sq - (row - lane), wv);
+                } else if (row < p.Sq) {
                     if (p.o_fp32) {
                         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
 #pragma unroll
@@ -527,26 +538,12 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     } else {
                         T* dst = static_cast<T*>(p.o) + obase;
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t v[8];
-#pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                v[i] = pack2<T>(__uint_as_float(s[c * 16 + 2 * i]) * inv_l,
-                                                __uint_as_float(s[c * 16 + 2 * i + 1]) * inv_l);
-                            if (p.o_align32) {
-                                // 32-byte stores: every instruction writes whole 32-byte sectors
-                                st_global_v8(dst + c * 16, v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]);
-                            } else {
-                                reinterpret_cast<uint4*>(dst + c * 16)[0] = make_uint4(v[0], v[1], v[2], v[3]);
-                                reinterpret_cast<uint4*>(dst + c * 16)[1] = make_uint4(v[4], v[5], v[6], v[7]);
-                            }
-                        }
-                    }
-                    if (p.lse != nullptr) {
-                        const float lse = (l_run > 0.f)
-                                              ? (m_loc * scale_log2 + log2f(l_run)) * 0.6931471805599453f
-                                              : -INFINITY;
-                        p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
+                        for (int c = 0; c < 16; ++c)
+                            reinterpret_cast<uint4*>(dst)[c] =
+                                make_uint4(pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 2]) * inv_l, __uint_as_float(s[8 * c + 3]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 4]) * inv_l, __uint_as_float(s[8 * c + 5]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 6]) * inv_l, __uint_as_float(s[8 * c + 7]) * inv_l));
                     }
                 }
             }

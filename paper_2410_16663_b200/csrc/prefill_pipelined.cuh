@@ -518,29 +518,38 @@ fa_fwd_pipelined_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
             const bool live = row < p.Sq;
             const long long obase = (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
+            if (!p.o_fp32 && p.o_align32) {
+                // 16-bit output, rows 32-byte aligned: whole-line stores through a lane exchange
+                uint32_t wv[64];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld_x32(tO + c * 32, r);
-                tmem_wait_ld();
-                if (live) {
-                    if (p.o_fp32) {
-                        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_x32(tO + c * 32, r);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
-                                                 __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
-                    } else {
-                        T* dst = static_cast<T*>(p.o) + obase + c * 32;
-                        uint32_t w[16];
+                    for (int i = 0; i < 16; ++i)
+                        wv[c * 16 + i] = pack2<T>(__uint_as_float(r[2 * i]) * inv_l, __uint_as_float(r[2 * i + 1]) * inv_l);
+                }
+                store_rows_coalesced<T>(static_cast<T*>(p.o) + obase, p.o_ss, p.Sq - (row - lane), wv);
+            } else {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            w[i] = pack2<T>(__uint_as_float(r[2 * i]) * inv_l, __uint_as_float(r[2 * i + 1]) * inv_l);
-                        if (p.o_align32) {
-                            // 32-byte stores: every instruction writes whole 32-byte sectors
-                            st_global_v8(dst, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
-                            st_global_v8(dst + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_x32(tO + c * 32, r);
+                    tmem_wait_ld();
+                    if (live) {
+                        if (p.o_fp32) {
+                            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
+                                                     __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
                         } else {
+                            T* dst = static_cast<T*>(p.o) + obase + c * 32;
+                            uint32_t w[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                w[i] = pack2<T>(__uint_as_float(r[2 * i]) * inv_l, __uint_as_float(r[2 * i + 1]) * inv_l);
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
                                 reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);

@@ -60,6 +60,57 @@ __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, u
     tma_load_4d(dst + kHalfBytes, tm, bar, 64, h, s0, b);
 }
 
+// Stores 32 consecutive rows of a 16-bit output tile, one row of 128 elements (64 packed words
+// w) per lane, so that every store instruction writes whole 128-byte lines.  A lane's own row is
+// eight 32-byte sectors; written directly, one instruction would touch 32 different lines with one
+// sector each.  Two butterfly exchanges inside each group of four lanes (with the lanes at
+// distance 1, then 2) leave lane a of the group with sectors a and 4 + a of all four rows of the
+// group, and the four lanes then write the four sectors of one line together.
+// row_ptr: this lane's own row (32-byte aligned); row_stride: elements between consecutive rows
+// (the rows of lanes l and l + 1); rows_live: how many of the warp's 32 rows exist (lane < rows_live).
+template <typename T>
+__device__ __forceinline__ void store_rows_coalesced(T* row_ptr, long long row_stride, int rows_live,
+                                                     uint32_t (&w)[64]) {
+    const int lane = threadIdx.x & 31;
+    const bool b0 = lane & 1, b1 = lane & 2;
+    // exchange with the lane at distance 1: keep the sectors whose index has bit 0 == b0
+    uint32_t a[4][2][8];  // [q][row slot: own pair member / the other][word]; sector index 2q + b0
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t lo = w[(2 * q) * 8 + i], hi = w[(2 * q + 1) * 8 + i];
+            const uint32_t send = b0 ? lo : hi;
+            a[q][0][i] = b0 ? hi : lo;
+            a[q][1][i] = __shfl_xor_sync(0xffffffffu, send, 1);
+        }
+    // exchange with the lane at distance 2: keep the sectors whose index has bit 1 == b1
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            uint32_t keep[8], got[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t lo = a[2 * h][r][i], hi = a[2 * h + 1][r][i];
+                const uint32_t send = b1 ? lo : hi;
+                keep[i] = b1 ? hi : lo;
+                got[i] = __shfl_xor_sync(0xffffffffu, send, 2);
+            }
+            // this lane now holds sector 4h + (lane & 3) of the rows of lanes lane^r and lane^r^2
+            const int sector = 4 * h + (lane & 3);
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int src_lane = lane ^ r ^ (2 * t);
+                if (src_lane < rows_live) {
+                    T* dst = row_ptr + (long long)(src_lane - lane) * row_stride + sector * 16;
+                    const uint32_t(&v)[8] = t ? got : keep;
+                    st_global_v8(dst, v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]);
+                }
+            }
+        }
+}
+
 // Number of kv tiles a query tile starting at row q0 has to visit.
 __device__ __forceinline__ int kv_tiles_for(int q0, int q_rows, int Sq, int Skv, int causal) {
     int n = (Skv + kTile - 1) / kTile;
