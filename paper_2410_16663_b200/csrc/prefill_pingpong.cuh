@@ -226,6 +226,7 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
                                                volatile uint32_t* abort_flag) {
     tma_prefetch_desc(tm_q);
     tma_prefetch_desc(tm_k);
+    const uint64_t pol_q = l2_policy_evict_first(), pol_kv = l2_policy_evict_last();
     PpRing<kPpNK> ring;
     for (int ord = 0;; ++ord) {
         const int idx = item_of_round(ord, total_items);
@@ -235,11 +236,11 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         // passes at once the first time each buffer is used
         if (!mbar_wait(pp_bar(bar0, ppb::q_empty + qb), ((ord >> 1) & 1) ^ 1, abort_flag, 150)) return;
         mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
-        load_tile(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h, it.q0, it.b);
+        load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h, it.q0, it.b, pol_q);
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
-            load_tile(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, j * kTile, it.b);
+            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, j * kTile, it.b, pol_kv);
         }
     }
 }
@@ -248,6 +249,7 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
 __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const CUtensorMap* tm_v, const FwdParams& p,
                                               int total_items, volatile uint32_t* abort_flag) {
     tma_prefetch_desc(tm_v);
+    const uint64_t pol_kv = l2_policy_evict_last();
     PpRing<kPpNV> ring;
     for (int ord = 0;; ++ord) {
         const int idx = item_of_round(ord, total_items);
@@ -256,7 +258,7 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
-            load_tile(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, j * kTile, it.b);
+            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, j * kTile, it.b, pol_kv);
         }
     }
 }

@@ -380,6 +380,7 @@ __device__ __forceinline__ void run_loader(uint32_t bar0, uint32_t sQ, uint32_t 
         tma_prefetch_desc(tm_q);
         tma_prefetch_desc(tm_k);
         tma_prefetch_desc(tm_v);
+        const uint64_t pol_q = l2_policy_evict_first(), pol_kv = l2_policy_evict_last();
         uint32_t g = 0;
         int ord = 0, lead = 0;
         bool ok = true;
@@ -392,21 +393,21 @@ __device__ __forceinline__ void run_loader(uint32_t bar0, uint32_t sQ, uint32_t 
             ok = mbar_wait(bar_q_empty(bar0, 0), q_par, abort_flag, 50);
             if (!ok) break;
             mbar_expect_tx(bar_q_full(bar0, 0), kTileBytes);
-            load_tile(sQ, tm_q, bar_q_full(bar0, 0), it.h, it.q0[0], it.b);
+            load_tile_hint(sQ, tm_q, bar_q_full(bar0, 0), it.h, it.q0[0], it.b, pol_q);
             for (int j = 0; j < n_kv && ok; ++j) {
                 for (int kv = 0; kv < 2 && ok; ++kv, ++g) {
                     const uint32_t slot = g % kStages;
                     ok = mbar_wait(bar_kv_empty(bar0, slot), ((g / kStages) & 1) ^ 1, abort_flag, 52 + kv);
                     if (!ok) break;
                     mbar_expect_tx(bar_kv_full(bar0, slot), kTileBytes);
-                    load_tile(sKV + slot * kTileBytes, kv ? tm_v : tm_k, bar_kv_full(bar0, slot), it.hk, j * kTile, it.b);
+                    load_tile_hint(sKV + slot * kTileBytes, kv ? tm_v : tm_k, bar_kv_full(bar0, slot), it.hk, j * kTile, it.b, pol_kv);
                     if (j == 0 && kv == 0) {
                         // Q of role 1 goes after K_0 so that role 0 can start the item while
                         // role 1 still finishes the previous one
                         ok = mbar_wait(bar_q_empty(bar0, 1), q_par, abort_flag, 51);
                         if (!ok) break;
                         mbar_expect_tx(bar_q_full(bar0, 1), kTileBytes);
-                        load_tile(sQ + kTileBytes, tm_q, bar_q_full(bar0, 1), it.h, it.q0[1], it.b);
+                        load_tile_hint(sQ + kTileBytes, tm_q, bar_q_full(bar0, 1), it.h, it.q0[1], it.b, pol_q);
                     }
                 }
             }

@@ -60,6 +60,21 @@ __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, u
     tma_load_4d(dst + kHalfBytes, tm, bar, 64, h, s0, b);
 }
 
+#ifndef FA_L2_HINTS
+#define FA_L2_HINTS 1
+#endif
+// The persistent kernels' loads carry an L2 eviction policy: Q is read once (evict first), K and V
+// of a head are read again by every later query tile of that head (evict last).
+__device__ __forceinline__ void load_tile_hint(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int h, int s0, int b,
+                                               uint64_t policy) {
+#if FA_L2_HINTS
+    tma_load_4d_hint(dst, tm, bar, 0, h, s0, b, policy);
+    tma_load_4d_hint(dst + kHalfBytes, tm, bar, 64, h, s0, b, policy);
+#else
+    load_tile(dst, tm, bar, h, s0, b);
+#endif
+}
+
 // Stores 32 consecutive rows of a 16-bit output tile, one row of 128 elements (64 packed words
 // w) per lane, so that every store instruction writes whole 128-byte lines.  A lane's own row is
 // eight 32-byte sectors; written directly, one instruction would touch 32 different lines with one
@@ -73,6 +88,9 @@ __device__ __forceinline__ void store_rows_coalesced(T* row_ptr, long long row_s
                                                      uint32_t (&w)[64]) {
     const int lane = threadIdx.x & 31;
     const bool b0 = lane & 1, b1 = lane & 2;
+#if FA_L2_HINTS
+    const uint64_t out_policy = l2_policy_evict_first();  // the output is not read again
+#endif
     // exchange with the lane at distance 1: keep the sectors whose index has bit 0 == b0
     uint32_t a[4][2][8];  // [q][row slot: own pair member / the other][word]; sector index 2q + b0
 #pragma unroll
@@ -105,7 +123,11 @@ __device__ __forceinline__ void store_rows_coalesced(T* row_ptr, long long row_s
                 if (src_lane < rows_live) {
                     T* dst = row_ptr + (long long)(src_lane - lane) * row_stride + sector * 16;
                     const uint32_t(&v)[8] = t ? got : keep;
+#if FA_L2_HINTS
+                    st_global_v8_hint(dst, v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], out_policy);
+#else
                     st_global_v8(dst, v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]);
+#endif
                 }
             }
         }
