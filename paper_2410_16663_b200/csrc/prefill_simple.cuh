@@ -27,10 +27,10 @@ struct FastDiv {
         shift = 31 + s;
         mul = static_cast<uint32_t>((1ull << shift) / d + 1);
     }
-    __device__ __forceinline__ int div(int n) const {
+    __host__ __device__ __forceinline__ int div(int n) const {
         return static_cast<int>((static_cast<unsigned long long>(static_cast<uint32_t>(n)) * mul) >> shift);
     }
-    __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
+    __host__ __device__ __forceinline__ void divmod(int n, int& q, int& r) const {
         q = div(n);
         r = n - q * static_cast<int>(d);
     }

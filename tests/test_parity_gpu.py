@@ -128,6 +128,15 @@ def test_pingpong_kernel_shape_grid(fa, sq, skv, causal):
     full_case(fa, 1, 2, 2, sq, skv, causal, "fp16", seed=sq * 1000 + skv + 7, variant=3)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_default_choice_of_kernel_from_4096_keys_on(fa, causal):
+    # fa_forward's own choice (the ping-pong kernel once Skv >= 4096) on a shape the full oracle
+    # finishes quickly: few query rows over many keys, rows ending inside a tile, a ragged key tail,
+    # bottom-right aligned mask
+    full_case(fa, 1, 4, 2, 130, 4200, causal, "fp16", seed=401)
+    full_case(fa, 1, 2, 2, 300, 4096, causal, "bf16", seed=402)
+
+
 def test_pingpong_kernel_many_items_per_cta(fa):
     # more query tiles than CTAs, of one to five kv steps each: every CTA strings several items
     # together, odd and even step counts, through both warpgroups
