@@ -165,6 +165,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.by_group.set(p.Hq / p.Hkv);
     fp.by_qtiles.set(fp.n_qtiles > 0 ? fp.n_qtiles : 1);
     fp.by_qpairs.set(fp.n_qtiles > 0 ? (fp.n_qtiles + 1) / 2 : 1);
+    fp.cls_log2 = 0;  // set by the ping-pong launcher
+    fp.by_class.set(1);
+    fp.by_lastcls.set(1);
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
     const bool bf16 = p.dtype == FA_DTYPE_BF16;
@@ -187,10 +190,10 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (rc) return rc;
 
     // Default choice, from timings of both kernels on B200: the ping-pong kernel (one query tile
-    // per CTA, Q K^T running ahead of the softmax) wins once an item has many kv steps; the
-    // paired-tile kernel keeps a small edge on short sequences, where items change every few steps.
+    // per CTA, Q K^T running ahead of the softmax) wins from 2048 keys on; the paired-tile kernel
+    // keeps an edge on shorter sequences, where items change every few steps.
     int variant = p.variant;
-    if (variant == 0) variant = (p.Skv >= 4096) ? 3 : 4;
+    if (variant == 0) variant = (p.Skv >= 2048) ? 3 : 4;
     switch (variant) {
         case 4:  // pipelined kernel, two query tiles per CTA
             return bf16 ? fa::launch_pipelined<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)

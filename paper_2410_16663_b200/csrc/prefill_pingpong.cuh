@@ -80,16 +80,26 @@ struct PpItem {
     int b, h, hk, q0, n;
 };
 
-// Work item `idx`: longest (latest) query tiles of all heads first; head by head when one head
-// alone has a round of items for every CTA (see decode_item in the pipelined kernel).
+// Work item `idx`.  The query tiles of a head are taken in classes of C = 2^cls_log2 consecutive
+// tiles, the class of the last (longest) tiles first; inside a class the items go head by head,
+// a head's tiles longest first.  With the items dealt to the CTAs round by round, a round then
+// works on about gridDim.x / C heads, whose K and V stay in L2 while the C tiles of each head
+// read them, and the rounds still get shorter and shorter items, which keeps the static
+// assignment balanced (the launcher picks C from the K/V bytes of a head, see launch_pingpong).
+// C >= n_qtiles is the plain head-by-head order used for very long sequences.
 __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
     PpItem it;
-    const bool head_major = p.n_qtiles >= (int)gridDim.x;
-    int major, minor;  // idx = major * (inner count) + minor
-    if (head_major) p.by_qtiles.divmod(idx, major, minor);
-    else p.by_bh.divmod(idx, major, minor);
-    const int qt = p.n_qtiles - 1 - (head_major ? minor : major);
-    const int bh = head_major ? major : minor;
+    int c, rem;  // class, index inside the class
+    p.by_class.divmod(idx, c, rem);
+    const int first = c << p.cls_log2;  // tiles in the classes before this one
+    int bh, j;
+    if (p.n_qtiles - first >= (1 << p.cls_log2)) {
+        bh = rem >> p.cls_log2;
+        j = rem & ((1 << p.cls_log2) - 1);
+    } else {
+        p.by_lastcls.divmod(rem, bh, j);
+    }
+    const int qt = p.n_qtiles - 1 - first - j;
     p.by_hq.divmod(bh, it.b, it.h);
     it.hk = p.by_group.div(it.h);
     it.q0 = qt * kTile;
@@ -588,7 +598,35 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
     const long long total = (long long)fp.n_qtiles * fp.B * fp.Hq;
     if (total > 0x7fffffffll) return -3;
     const int grid = (int)(total < sm_count ? total : sm_count);
-    kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, fp, (int)total);
+    // Class size of the item order: large enough that the K and V of the kv heads one round of
+    // CTAs works on (about grid / (C * group) of them, Skv * 512 bytes each) fit in a fraction of
+    // L2, but at most half of a head's tiles and 16 (a class that is the whole head makes all
+    // its tiles read the same K/V lines at the same moment, which measured slower).  Under the
+    // causal mask the items of a class differ in length, which costs balance when a head has few
+    // tiles: heads with fewer than 16 keep the plain longest-first order.  When one head alone
+    // fills every CTA, a single class: the plain head-by-head order.
+    FwdParams fpc = fp;
+    int cls_log2 = 0;
+    if (fp.n_qtiles >= grid) {
+        while ((1 << cls_log2) < fp.n_qtiles) ++cls_log2;
+    } else {
+#ifdef FA_PP_CLASS_LOG2
+        cls_log2 = FA_PP_CLASS_LOG2;
+#else
+        const double head_bytes = 512.0 * fp.Skv / (fp.Hq / fp.Hkv);
+        const double budget = 32.0 * 1024 * 1024;
+        const int half = fp.n_qtiles / 2 < 16 ? fp.n_qtiles / 2 : 16;
+        const int cap = (fp.causal && fp.n_qtiles < 16) ? 1 : half;
+        while ((grid >> cls_log2) * head_bytes > budget && (2 << cls_log2) <= cap) ++cls_log2;
+#endif
+        while (cls_log2 > 0 && (1 << cls_log2) > fp.n_qtiles) --cls_log2;
+    }
+    fpc.cls_log2 = cls_log2;
+    const long long class_items = ((long long)fp.B * fp.Hq) << cls_log2;  // > total only for a single class
+    fpc.by_class.set(class_items > 0x7fffffffll ? 0x7fffffff : (int)class_items);
+    const int last = fp.n_qtiles & ((1 << cls_log2) - 1);
+    fpc.by_lastcls.set(last ? last : 1);
+    kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, fpc, (int)total);
     e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = (int)e; return -7; }
     return 0;

@@ -47,6 +47,11 @@ struct FwdParams {
     int n_qtiles;
     int o_align32;  // o and its strides are 32-byte aligned: rows can be written with 256-bit stores
     FastDiv by_bh, by_hq, by_group, by_qtiles, by_qpairs;  // B*Hq, Hq, Hq/Hkv, n_qtiles, ceil(n_qtiles/2)
+    // item order of the ping-pong kernel (see pp_decode_item): query tiles come in classes of
+    // 2^cls_log2 consecutive tiles; by_class divides by the items of a full class, by_lastcls by
+    // the size of the last (possibly smaller) class
+    int cls_log2;
+    FastDiv by_class, by_lastcls;
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim

@@ -130,11 +130,20 @@ def test_pingpong_kernel_shape_grid(fa, sq, skv, causal):
 
 @pytest.mark.parametrize("causal", [False, True])
 def test_default_choice_of_kernel_from_4096_keys_on(fa, causal):
-    # fa_forward's own choice (the ping-pong kernel once Skv >= 4096) on a shape the full oracle
+    # fa_forward's own choice (the ping-pong kernel once Skv >= 2048) on a shape the full oracle
     # finishes quickly: few query rows over many keys, rows ending inside a tile, a ragged key tail,
     # bottom-right aligned mask
     full_case(fa, 1, 4, 2, 130, 4200, causal, "fp16", seed=401)
     full_case(fa, 1, 2, 2, 300, 4096, causal, "bf16", seed=402)
+
+
+def test_pingpong_kernel_item_order_in_tile_classes(fa):
+    # shapes whose K/V per head are large enough for the launcher to order the items in classes of
+    # query tiles: 17 tiles per head (classes of 8, 8 and 1), 33 tiles (16, 16, 1), and without a
+    # mask 6 tiles (classes of 4 and 2); every output row must be written exactly once
+    full_case(fa, 1, 8, 8, 2100, 2100, True, "fp16", seed=411)
+    full_case(fa, 1, 4, 2, 4130, 4130, True, "fp16", seed=412)
+    full_case(fa, 2, 16, 16, 700, 2100, False, "fp16", seed=413)
 
 
 def test_pingpong_kernel_many_items_per_cta(fa):
