@@ -239,7 +239,7 @@ def run_product(args, rank, world, local_rank):
     # `traffic`: DRAM bytes per launch from one ncu capture (profiles/): the C2 prefill launch
     # itself, and for decode a 4.3 GB case of the same kernel whose dram bytes were 1.007 x its
     # algorithmic bytes, scaled to this launch by the cache bytes it scans
-    c2_traffic = 512.0e6 if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
+    c2_traffic = 300.0e6 if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
     algo_prefill_bytes = (2.0 * pc.B * pc.Sq * pc.Hq + 2.0 * pc.B * pc.Skv * pc.Hkv) * pc.d * 2 + 4.0 * pc.B * pc.Hq * pc.Sq
     out["roofline"] = {"kernel": "fa_fwd_pingpong_kernel (prefill C2, the kernel behind `value`; the library picks it for Skv >= 2048)", "bound": "tensor",
                        "achieved": round(tflops / world, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
