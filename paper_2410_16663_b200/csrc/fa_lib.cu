@@ -296,12 +296,9 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
                         fa::kDecTile, false);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
-        static bool attr_set = false;
-        if (!attr_set) {
-            rc = set_smem(fa::fa_decode_split_mma_kernel, smem);
-            if (rc) return rc;
-            attr_set = true;
-        }
+        int sm_count = 0;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(fa::fa_decode_split_mma_kernel), smem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
         fa::fa_decode_split_mma_kernel<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();

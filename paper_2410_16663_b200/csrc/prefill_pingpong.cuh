@@ -586,15 +586,9 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
                     cudaStream_t st, int* cuda_err) {
     constexpr int smem = (kPpQBufs + kPpNK + kPpNV) * kTileBytes;
     auto kern = fa_fwd_pingpong_kernel<T>;
-    static int sm_count = 0;
+    int sm_count = 0;
     cudaError_t e;
-    if (sm_count == 0) {
-        int dev = 0, n = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        sm_count = n;
-    }
+    if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }
     const long long total = (long long)fp.n_qtiles * fp.B * fp.Hq;
     if (total > 0x7fffffffll) return -3;
     const int grid = (int)(total < sm_count ? total : sm_count);

@@ -601,15 +601,9 @@ int launch_pipelined(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                      cudaStream_t st, int* cuda_err) {
     constexpr int smem = 1024 + (2 + kStages) * kTileBytes;
     auto kern = fa_fwd_pipelined_kernel<T>;
-    static int sm_count = 0;
+    int sm_count = 0;
     cudaError_t e;
-    if (sm_count == 0) {
-        int dev = 0, n = 0;
-        if ((e = cudaGetDevice(&dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) { *cuda_err = (int)e; return -7; }
-        sm_count = n;
-    }
+    if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }
     const int n_qpairs = (fp.n_qtiles + 1) / 2;
     const long long total = (long long)n_qpairs * fp.B * fp.Hq;
     if (total > 0x7fffffffll) return -3;

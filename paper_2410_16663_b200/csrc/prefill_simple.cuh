@@ -80,6 +80,49 @@ __device__ __forceinline__ void load_tile_hint(uint32_t dst, const CUtensorMap* 
 #endif
 }
 
+// Host side, once per kernel and device: the opt-in to more than 48 KB of dynamic shared memory
+// is a per-device attribute of each kernel function, so a process that launches on several GPUs
+// needs it on each, for each kernel.  Returns 0 and the device's SM count, or the CUDA error
+// code.  The table of what has been done is keyed by kernel address and device; concurrent first
+// calls at worst repeat the same idempotent set-up.
+inline int prepare_big_smem_kernel(const void* kern, int smem_bytes, int* sm_count) {
+    constexpr int kMaxDev = 64, kMaxKernels = 16;
+    struct Entry {
+        const void* kern;
+        int sms[kMaxDev];
+    };
+    static Entry table[kMaxKernels] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    Entry* ent = nullptr;
+    for (int i = 0; i < kMaxKernels && !ent; ++i) {
+        const void* k = __atomic_load_n(&table[i].kern, __ATOMIC_ACQUIRE);
+        if (k == kern) ent = &table[i];
+        else if (k == nullptr) {
+            const void* expected = nullptr;
+            if (__atomic_compare_exchange_n(&table[i].kern, &expected, kern, false, __ATOMIC_ACQ_REL, __ATOMIC_ACQUIRE) ||
+                expected == kern)
+                ent = &table[i];
+        }
+    }
+    const bool cached = ent && dev >= 0 && dev < kMaxDev;
+    if (cached) {
+        const int n = __atomic_load_n(&ent->sms[dev], __ATOMIC_ACQUIRE);
+        if (n > 0) {
+            *sm_count = n;
+            return 0;
+        }
+    }
+    int n = 0;
+    if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return (int)e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)) != cudaSuccess)
+        return (int)e;
+    if (cached) __atomic_store_n(&ent->sms[dev], n, __ATOMIC_RELEASE);
+    *sm_count = n;
+    return 0;
+}
+
 // Stores 32 consecutive rows of a 16-bit output tile, one row of 128 elements (64 packed words
 // w) per lane, so that every store instruction writes whole 128-byte lines.  A lane's own row is
 // eight 32-byte sectors; written directly, one instruction would touch 32 different lines with one
