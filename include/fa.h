@@ -145,9 +145,15 @@ int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, v
 /*
  * Host-buffer form of fa_forward for callers whose tensors live in host memory (pinned memory
  * makes the copies asynchronous): copies q, k, v to the device staging area, runs the forward,
- * copies o and lse back, all on `stream`.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16.
+ * copies o and lse back.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16.
  * staging is a DEVICE buffer of at least fa_forward_host_staging_bytes(...) bytes, 1024-byte
- * aligned, owned by the caller.  The results are in o_host / lse_host once the stream is idle.
+ * aligned, owned by the caller.  The call is ordered after the work already on `stream`, and the
+ * results are in o_host / lse_host once `stream` is idle.  Inside, the batch is cut into up to
+ * four parts whose copy-in, forward and copy-out stages overlap: the forward runs on `stream`,
+ * the copies on two streams the library creates once per device (with a handful of events) and
+ * keeps; nothing else is created and no device memory is allocated.  Make the first call on a
+ * device outside stream capture.  Calls that share a staging buffer must be issued on the same
+ * stream.
  */
 int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
                     float* lse_host, int B, int Hq, int Hkv, int Sq, int Skv, int d, int causal,

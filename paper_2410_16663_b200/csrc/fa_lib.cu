@@ -9,6 +9,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "decode.cuh"
 #include "prefill_pingpong.cuh"
 #include "prefill_pipelined.cuh"
@@ -212,6 +214,39 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     }
 }
 
+// Streams and events of fa_forward_host, made once per device and kept for the life of the
+// process (host-side objects; no device memory).
+constexpr int kHostParts = 4;
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, finish = nullptr, in_done[kHostParts] = {}, fwd_done[kHostParts] = {};
+    bool ready = false;
+};
+HostPipe* host_pipe() {
+    constexpr int kMaxDev = 64;
+    static HostPipe pipes[kMaxDev];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    HostPipe& hp = pipes[dev];
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.finish, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kHostParts; ++i)
+            ok = cudaEventCreateWithFlags(&hp.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.fwd_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            t_last_cuda_error = static_cast<int>(cudaGetLastError());
+            return nullptr;
+        }
+        hp.ready = true;
+    }
+    return &hp;
+}
+
 int forward_plain(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv,
                   int Sq, int Skv, int d, int causal, float scale, int dtype, void* stream) {
     fa_params p;
@@ -368,7 +403,6 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
     if (reinterpret_cast<uintptr_t>(staging) & 1023u) return FA_ERR_ALIGN;
     auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
     const size_t qo_b = (size_t)B * Sq * Hq * 128 * 2, kv_b = (size_t)B * Skv * Hkv * 128 * 2;
-    const size_t l_b = (size_t)B * Hq * Sq * 4;
     char* base = static_cast<char*>(staging);
     char* dq = base;
     char* dk = dq + up(qo_b);
@@ -377,17 +411,45 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
     char* dl = dout + up(qo_b);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(dq, q_host, qo_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    if (kv_b) {
-        if ((e = cudaMemcpyAsync(dk, k_host, kv_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(dv, v_host, kv_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    // The batch is cut into up to four parts, and the three stages of a part -- copy in, forward,
+    // copy out -- run on three streams (the caller's for the forward, two of the library's own for
+    // the copies), chained by events: the copy engines of both directions and the SMs then work
+    // at the same time on different parts.  Everything is ordered after the work already on
+    // `stream`, and `stream` waits for the last copy out.
+    HostPipe* hp = host_pipe();
+    if (!hp) return FA_ERR_CUDA;
+    const int parts = B < kHostParts ? B : kHostParts;
+    if ((e = cudaEventRecord(hp->start, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess) return cuda_fail(e);
+    const size_t q1 = (size_t)Sq * Hq * 128 * 2, kv1 = (size_t)Skv * Hkv * 128 * 2, l1 = (size_t)Hq * Sq * 4;
+    for (int c = 0; c < parts; ++c) {
+        const int b0 = (int)((long long)B * c / parts), b1 = (int)((long long)B * (c + 1) / parts);
+        const size_t nb = (size_t)(b1 - b0);
+        if ((e = cudaMemcpyAsync(dq + b0 * q1, static_cast<const char*>(q_host) + b0 * q1, nb * q1,
+                                 cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return cuda_fail(e);
+        if (kv1) {
+            if ((e = cudaMemcpyAsync(dk + b0 * kv1, static_cast<const char*>(k_host) + b0 * kv1, nb * kv1,
+                                     cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpyAsync(dv + b0 * kv1, static_cast<const char*>(v_host) + b0 * kv1, nb * kv1,
+                                     cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return cuda_fail(e);
+        }
+        if ((e = cudaEventRecord(hp->in_done[c], hp->in)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(st, hp->in_done[c], 0)) != cudaSuccess) return cuda_fail(e);
+        int rc = forward_plain(dq + b0 * q1, dk + b0 * kv1, dv + b0 * kv1, dout + b0 * q1,
+                               reinterpret_cast<float*>(dl + b0 * l1), (int)nb, Hq, Hkv, Sq, Skv, d, causal, scale,
+                               dtype, stream);
+        if (rc) return rc;
+        if ((e = cudaEventRecord(hp->fwd_done[c], st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(hp->out, hp->fwd_done[c], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(static_cast<char*>(o_host) + b0 * q1, dout + b0 * q1, nb * q1, cudaMemcpyDeviceToHost,
+                                 hp->out)) != cudaSuccess) return cuda_fail(e);
+        if (lse_host)
+            if ((e = cudaMemcpyAsync(reinterpret_cast<char*>(lse_host) + b0 * l1, dl + b0 * l1, nb * l1,
+                                     cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess) return cuda_fail(e);
     }
-    int rc = forward_plain(dq, dk, dv, dout, reinterpret_cast<float*>(dl), B, Hq, Hkv, Sq, Skv, d, causal, scale,
-                           dtype, stream);
-    if (rc) return rc;
-    if ((e = cudaMemcpyAsync(o_host, dout, qo_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if (lse_host)
-        if ((e = cudaMemcpyAsync(lse_host, dl, l_b, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventRecord(hp->finish, hp->out)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(st, hp->finish, 0)) != cudaSuccess) return cuda_fail(e);
     return FA_OK;
 }
 

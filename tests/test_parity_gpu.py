@@ -368,3 +368,29 @@ def test_forward_host_entry(fa):
     check_status(fa)
     o_ref, l_ref = oracle.attention_full(q, k, v, c.causal, c.scale)
     assert_close_to_oracle(o, lse, o_ref, l_ref, what="host entry")
+
+
+@pytest.mark.parametrize("B", [2, 5])
+def test_forward_host_entry_batch_parts(fa, B):
+    # the host entry cuts the batch into up to four parts that it copies and computes in a
+    # pipeline over its own streams: even and uneven splits, bf16, twice in a row on one staging
+    # buffer (the second call must wait for the first one's copies out), NaN-filled outputs
+    cfg = synth.PrefillConfig("t", B, 4, 2, 200, 333, dtype="bf16", causal=True, seed=70 + B)
+    q, k, v = (t.pin_memory() for t in synth.prefill_inputs(cfg, "cpu"))
+    o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
+    absv = oracle.attention_full(q, k, v.abs(), True, cfg.scale)[0]
+    n = fa.fa_forward_host_staging_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Sq, cfg.Skv, cfg.d)
+    st = torch.empty(n + 1024, dtype=torch.uint8, device=DEV)
+    off = (-st.data_ptr()) % 1024
+    outs = []
+    for _ in range(2):
+        o = torch.full_like(q, float("nan")).pin_memory()
+        lse = torch.full((cfg.B, cfg.Hq, cfg.Sq), float("nan"), dtype=torch.float32).pin_memory()
+        fa.fa_forward_host(q, k, v, o, lse, True, cfg.scale, st[off:off + n])
+        outs.append((o, lse))
+    torch.cuda.synchronize()
+    check_status(fa)
+    for o, lse in outs:
+        assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=True, p_absv=absv, what=f"host entry B={B}")
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
