@@ -8,6 +8,7 @@ With bf16 inputs two format roundings are allowed on top, each bounded exactly f
 and 2^-8 |O| for a stored bf16 output; the fp32-output mode is gated without the latter."""
 import math
 
+import numpy as np
 import pytest
 import torch
 
@@ -135,6 +136,31 @@ def test_default_choice_of_kernel_from_4096_keys_on(fa, causal):
     # bottom-right aligned mask
     full_case(fa, 1, 4, 2, 130, 4200, causal, "fp16", seed=401)
     full_case(fa, 1, 2, 2, 300, 4096, causal, "bf16", seed=402)
+
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        g = int(rng.choice([1, 1, 2, 4, 8]))
+        hkv = int(rng.integers(1, 5))
+        B = int(rng.integers(1, 4))
+        skv = int(rng.choice([int(rng.integers(1, 400)), int(rng.integers(400, 1400)), int(rng.integers(2048, 2700))]))
+        causal = bool(rng.integers(0, 2))
+        sq = int(rng.integers(1, skv + 1)) if causal else int(rng.integers(1, 700))
+        sq = min(sq, 900)
+        if B * hkv * g * sq * skv > 30_000_000:
+            continue
+        out.append((B, hkv * g, hkv, sq, skv, causal, "fp16" if rng.integers(0, 2) else "bf16"))
+    return out
+
+
+@pytest.mark.parametrize("variant", [3, 4])
+def test_random_shapes_both_persistent_kernels(fa, variant):
+    # thirty seeded random problems (batch, head grouping, ragged lengths, masks, both 16-bit
+    # types) through each persistent kernel, every output element against the oracle
+    for i, (B, hq, hkv, sq, skv, causal, dt) in enumerate(_random_shapes(30, seed=2024)):
+        full_case(fa, B, hq, hkv, sq, skv, causal, dt, seed=9000 + i, variant=variant)
 
 
 def test_pingpong_kernel_item_order_in_tile_classes(fa):
