@@ -241,7 +241,7 @@ def run_product(args, rank, world, local_rank):
     # algorithmic bytes, scaled to this launch by the cache bytes it scans
     c2_traffic = 300.0e6 if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
     algo_prefill_bytes = (2.0 * pc.B * pc.Sq * pc.Hq + 2.0 * pc.B * pc.Skv * pc.Hkv) * pc.d * 2 + 4.0 * pc.B * pc.Hq * pc.Sq
-    out["roofline"] = {"kernel": "fa_fwd_pingpong_kernel (prefill C2, the kernel behind `value`; the library picks it for Skv >= 2048)", "bound": "tensor",
+    out["roofline"] = {"kernel": "fa_fwd_pingpong_kernel (prefill C2, the kernel behind `value`; the library picks it for Skv >= 1024)", "bound": "tensor",
                        "achieved": round(tflops / world, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                        "frac": round(tflops / world / peaks["bf16_tflops"], 4),
                        "peak_source": peaks["source"] + " bf16 GEMM burst (of measured; fp16 has the same nominal rate)",

@@ -91,7 +91,7 @@ typedef struct fa_params {
     int64_t k_stride[3];
     int64_t v_stride[3];
     int64_t o_stride[3];
-    int variant; /* 0 = default: the ping-pong kernel when Skv >= 2048, else the paired-tile pipelined
+    int variant; /* 0 = default: the ping-pong kernel when Skv >= 1024, else the paired-tile pipelined
                     kernel.  Others force one kernel, for A/B timing and tests: 1, 2 = simple kernels
                     (P through tensor / shared memory), 3 = ping-pong, 4 = paired-tile pipelined. */
 } fa_params;

@@ -192,10 +192,10 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (rc) return rc;
 
     // Default choice, from timings of both kernels on B200: the ping-pong kernel (one query tile
-    // per CTA, Q K^T running ahead of the softmax) wins from 2048 keys on; the paired-tile kernel
+    // per CTA, Q K^T running ahead of the softmax) wins from 1024 keys on; the paired-tile kernel
     // keeps an edge on shorter sequences, where items change every few steps.
     int variant = p.variant;
-    if (variant == 0) variant = (p.Skv >= 2048) ? 3 : 4;
+    if (variant == 0) variant = (p.Skv >= 1024) ? 3 : 4;
     switch (variant) {
         case 4:  // pipelined kernel, two query tiles per CTA
             return bf16 ? fa::launch_pipelined<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
@@ -206,9 +206,15 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         case 2:  // simple kernel, P handed over through shared memory
             return bf16 ? launch_simple<__nv_bfloat16, false>(tq, tk, tv, fp, st)
                         : launch_simple<__half, false>(tq, tk, tv, fp, st);
-        case 3:  // ping-pong kernel: one query tile per CTA, two softmax warpgroups alternate over kv steps
-            return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
-                        : fa::launch_pingpong<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
+        case 3: {  // ping-pong kernel: one query tile per CTA, two softmax warpgroups alternate over kv steps
+            CUtensorMap to = tq;
+            if (!fp.o_fp32) {  // the output leaves through TMA stores of 32 rows x 64 columns
+                rc = encode_map(&to, p.o, p.B, p.Sq, p.Hq, p.o_stride[0], p.o_stride[1], p.o_stride[2], 32, bf16);
+                if (rc) return rc;
+            }
+            return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
+                        : fa::launch_pingpong<__half>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
+        }
         default:
             return FA_ERR_UNSUPPORTED;
     }

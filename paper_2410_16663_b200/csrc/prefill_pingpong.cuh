@@ -49,7 +49,8 @@ static_assert((kPpQBufs + kPpNK + kPpNV) * kTileBytes + 3072 <= 232448, "shared 
 // ---- barriers: indices into one array
 namespace ppb {
 constexpr int q_full = 0;                       // [2]  TMA -> S thread
-constexpr int q_empty = 2;                      // [2]  S thread (commit) -> loader
+constexpr int q_empty = 2;                      // [2]  S thread (commit) -> loader; with the output staged in the
+                                                //      Q buffer, the four epilogue warps (count 4) -> loader
 constexpr int k_full = 4;                       // [NK]
 constexpr int k_empty = k_full + kPpNK;         // [NK]
 constexpr int v_full = k_empty + kPpNK;         // [NV]
@@ -165,7 +166,7 @@ struct PpRing {
 };
 
 // The thread that issues S = Q K^T of every step.
-template <typename T>
+template <typename T, bool kTmaOut>
 __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK, uint32_t tmem, const FwdParams& p,
                                          int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
@@ -194,7 +195,8 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
             }
             mma_commit(pp_bar(bar0, ppb::s_full + buf));
             mma_commit(pp_bar(bar0, ppb::k_empty + ring.slot));
-            if (j == it.n - 1) mma_commit(pp_bar(bar0, ppb::q_empty + qb));
+            // with the output staged in the Q buffer the item's epilogue hands the buffer back
+            if (!kTmaOut && j == it.n - 1) mma_commit(pp_bar(bar0, ppb::q_empty + qb));
         }
     }
 }
@@ -301,8 +303,8 @@ struct PpSoftmax {
 
     // Step g of the CTA = step j of the item.  kMasked: the tile is crossed by the diagonal or by
     // the end of the keys.  Returns false when a wait gave up.
-    template <bool kMasked>
-    __device__ __forceinline__ bool step(uint32_t (&s)[128], uint32_t g, int j) {
+    template <int kMasked>  // 0: no mask code; 1: masked tile; 2: decided at run time by `masked`
+    __device__ __forceinline__ bool step(uint32_t (&s)[128], uint32_t g, int j, bool masked = false) {
         if (!pp_warp_wait(pp_bar(bar0, ppb::s_full + w), (g >> 1) & 1, abort_flag, 110 + w)) return false;
         tc_fence_after();
         tmem_ld_x32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
@@ -313,7 +315,7 @@ struct PpSoftmax {
         tc_fence_before();  // for the arrival below that hands the S buffer back
         // probe early, look at the answer after the row max
         const bool m_there = g > 0 && mbar_test(pp_bar(bar0, ppb::m_ready + (1 - w)), ((g - 1) >> 1) & 1);
-        if (kMasked) {
+        if (kMasked == 1 || (kMasked == 2 && masked)) {
             // hidden scores become -inf (the scale is strictly positive, so they come out as exact zeros)
             const int kv0 = j * kTile;
             int lim = Skv - kv0;
@@ -400,10 +402,21 @@ struct PpSoftmax {
     }
 };
 
-template <typename T>
+// kTmaOut: the output has the operands' 16-bit type; an item's O goes, scaled and rounded, into
+// the item's Q buffer (which Q K^T has finished with by then) in the swizzled layout of a tile,
+// and each warp sends its 32 rows to global memory with two TMA stores (tm_o: boxes of 32 rows x
+// 64 columns).  Rows past the end of the queries are clipped by the tensor map.  Otherwise
+// (fp32 output) every thread stores its own row.
+// kSingle: the step exists once, and a branch skips its mask code on tiles every row sees in
+// full; otherwise those tiles take a loop of their own without mask code.  The single copy is a
+// little slower per step and much smaller: with it, what an item executes from its first step
+// to its epilogue stays within the 32 KB the instruction cache serves at full rate, which is
+// what counts when an item has few steps.
+template <typename T, bool kTmaOut, bool kSingle>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const FwdParams p, const int total_items) {
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                       const FwdParams p, const int total_items) {
     // Shared memory is used to the last byte: 3 KiB of static state (sized so that the dynamic
     // part that follows it starts on a 1024-byte boundary, which the 128-byte swizzle needs)
     // plus seven 32 KiB tiles.  The alignment is checked rather than assumed.
@@ -425,7 +438,8 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
     if (tid == 0) {
         for (int i = 0; i < ppb::count; ++i) {
-            mbar_init(pp_bar(bar0, i), i >= ppb::p_full ? 128 : 1);
+            const bool q_back = kTmaOut && (i == ppb::q_empty || i == ppb::q_empty + 1);
+            mbar_init(pp_bar(bar0, i), i >= ppb::p_full ? 128 : (q_back ? 4 : 1));
         }
         ss.abort_flag = 0;
         fence_mbar_init();
@@ -466,6 +480,20 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         uint32_t g = 0;        // step counter of the CTA
         uint32_t items2 = 0;   // items with at least two steps seen so far
         bool ok = true;
+        // Q buffer whose TMA stores this warp has issued but not yet waited for (-1: none).  The
+        // wait (until the stores have read the buffer) and the hand-back to the loader come after
+        // this warp's next step: early enough for the load of the item after the next, and off
+        // the path from one item's last step to the next item's first.
+        int q_back = -1;
+        auto hand_back_q = [&]() {
+            if (kTmaOut && q_back >= 0) {
+                if (lane == 0) {
+                    tma_store_wait_read();
+                    mbar_arrive(pp_bar(bar0, ppb::q_empty + q_back));
+                }
+                q_back = -1;
+            }
+        };
         for (int ord = 0; ok; ++ord) {
             const int idx = item_of_round(ord, total_items);
             if (idx >= total_items) break;
@@ -487,8 +515,22 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             // this warpgroup's steps of the item: those with an absolute step number of its parity
             const uint32_t g_item = g;
             int j = (int)((g_item ^ (uint32_t)w) & 1u);
+            // no step of this warpgroup in the item (one step, the other warpgroup's): the next
+            // step it takes belongs to the item whose Q load waits for the buffer, so hand it back now
+            if (j >= n) hand_back_q();
+            if (kSingle) {
+            for (; j < n && ok; j += 2) {
+                ok = sm.template step<2>(s, g_item + (uint32_t)j, j, j >= n_full);
+                hand_back_q();
+                if (ok && j == n - 2) {
+                    ss.l_xch[xb][r] = sm.l_part;
+                    mbar_arrive(pp_bar(bar0, ppb::l_pub + xb));
+                }
+            }
+            } else {
             for (; j < n_full && ok; j += 2) {
-                ok = sm.template step<false>(s, g_item + (uint32_t)j, j);
+                ok = sm.template step<0>(s, g_item + (uint32_t)j, j);
+                hand_back_q();
                 if (ok && j == n - 2) {
                     // the other warpgroup runs the last step and the epilogue: hand it this row sum
                     // (it is relative to the reference this step left, which that step receives)
@@ -497,11 +539,13 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
             }
             for (; j < n && ok; j += 2) {
-                ok = sm.template step<true>(s, g_item + (uint32_t)j, j);
+                ok = sm.template step<1>(s, g_item + (uint32_t)j, j);
+                hand_back_q();
                 if (ok && j == n - 2) {
                     ss.l_xch[xb][r] = sm.l_part;
                     mbar_arrive(pp_bar(bar0, ppb::l_pub + xb));
                 }
+            }
             }
             const float l_part = sm.l_part, m_loc = sm.m_loc, m_before = sm.m_before;
             if (ok && ((g_item + (uint32_t)n - 1u) & 1u) == (uint32_t)w) {
@@ -532,13 +576,32 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                                     : -INFINITY;
                     p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
                 }
-                if (!p.o_fp32 && p.o_align32) {
-                    // 16-bit output, rows 32-byte aligned: whole-line stores through a lane exchange
-                    uint32_t wv[64];
+                if (kTmaOut) {
+                    const uint32_t q_buf = sQ + (uint32_t)(ord & 1) * kTileBytes;
+                    const uint32_t row_base = q_buf + (uint32_t)r * 128u;
 #pragma unroll
-                    for (int i = 0; i < 64; ++i)
-                        wv[i] = pack2<T>(__uint_as_float(s[2 * i]) * inv_l, __uint_as_float(s[2 * i + 1]) * inv_l);
-                    store_rows_coalesced<T>(static_cast<T*>(p.o) + obase, p.o_ss, p.Sq - (row - lane), wv);
+                    for (int c = 0; c < 16; ++c) {
+                        // 16-byte chunk c & 7 of the row's half c >> 3, at its swizzled place
+                        const uint32_t addr = row_base + (uint32_t)(c >> 3) * kHalfBytes + (((uint32_t)(c & 7) ^ ((uint32_t)r & 7u)) << 4);
+                        const uint32_t w0 = pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l);
+                        const uint32_t w1 = pack2<T>(__uint_as_float(s[8 * c + 2]) * inv_l, __uint_as_float(s[8 * c + 3]) * inv_l);
+                        const uint32_t w2 = pack2<T>(__uint_as_float(s[8 * c + 4]) * inv_l, __uint_as_float(s[8 * c + 5]) * inv_l);
+                        const uint32_t w3 = pack2<T>(__uint_as_float(s[8 * c + 6]) * inv_l, __uint_as_float(s[8 * c + 7]) * inv_l);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int row0 = it.q0 + (warp & 3) * 32;
+                        if (row0 < p.Sq) {
+                            const uint32_t src = q_buf + (uint32_t)(warp & 3) * 4096u;
+                            tma_store_4d(&tm_o, src, 0, it.h, row0, it.b);
+                            tma_store_4d(&tm_o, src + kHalfBytes, 64, it.h, row0, it.b);
+                            tma_store_commit();
+                        }
+                    }
+                    q_back = ord & 1;  // handed back to the loader after this warp's next step
+                    __syncwarp();
                 } else if (row < p.Sq) {
                     if (p.o_fp32) {
                         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
@@ -562,10 +625,12 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             g = g_item + (uint32_t)n;
             if (n >= 2) ++items2;
         }
+        // the stores read shared memory, which has to outlive them
+        if (kTmaOut && lane == 0) tma_store_wait_all();
     } else {
         setmaxnreg_dec<kPipeOtherRegs>();
         if (lane == 0) {
-            if (warp == 8) pp_run_s<T>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
+            if (warp == 8) pp_run_s<T, kTmaOut>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
             else if (warp == 10) pp_run_pv<T>(bar0, sV, tmem_base, p, total_items, abort_flag);
             else if (warp == 9) pp_run_load_qk(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
             else pp_run_load_v(bar0, sV, &tm_v, p, total_items, abort_flag);
@@ -581,11 +646,17 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     }
 }
 
+// to: map over the output with boxes of 32 rows x 64 columns; read only when the output has the
+// operands' type (any valid map otherwise).
 template <typename T>
-int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& fp,
-                    cudaStream_t st, int* cuda_err) {
+int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                    const FwdParams& fp, cudaStream_t st, int* cuda_err) {
     constexpr int smem = (kPpQBufs + kPpNK + kPpNV) * kTileBytes;
-    auto kern = fa_fwd_pingpong_kernel<T>;
+    // the single-copy step up to 32 kv tiles per item (timed: ahead by 3 % at 2048 keys, level at
+    // 4096, behind by 1 % at 8192)
+    const bool single = fp.o_fp32 || fp.Skv <= 32 * kTile;
+    auto kern = fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true>
+                          : (single ? fa_fwd_pingpong_kernel<T, true, true> : fa_fwd_pingpong_kernel<T, true, false>);
     int sm_count = 0;
     cudaError_t e;
     if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }
@@ -620,7 +691,7 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
     fpc.by_class.set(class_items > 0x7fffffffll ? 0x7fffffff : (int)class_items);
     const int last = fp.n_qtiles & ((1 << cls_log2) - 1);
     fpc.by_lastcls.set(last ? last : 1);
-    kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, fpc, (int)total);
+    kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, to, fpc, (int)total);
     e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = (int)e; return -7; }
     return 0;

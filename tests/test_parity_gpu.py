@@ -131,7 +131,7 @@ def test_pingpong_kernel_shape_grid(fa, sq, skv, causal):
 
 @pytest.mark.parametrize("causal", [False, True])
 def test_default_choice_of_kernel_from_4096_keys_on(fa, causal):
-    # fa_forward's own choice (the ping-pong kernel once Skv >= 2048) on a shape the full oracle
+    # fa_forward's own choice (the ping-pong kernel once Skv >= 1024) on a shape the full oracle
     # finishes quickly: few query rows over many keys, rows ending inside a tile, a ragged key tail,
     # bottom-right aligned mask
     full_case(fa, 1, 4, 2, 130, 4200, causal, "fp16", seed=401)
@@ -198,7 +198,9 @@ def test_scale_zero_and_large_scale(fa):
     full_case(fa, 1, 2, 2, 130, 260, False, "fp16", seed=6, scale=1.0, fp16_ulp=True)  # peaked softmax
 
 
-def test_bhsd_strided_layout(fa):
+@pytest.mark.parametrize("variant", [0, 3, 4])
+def test_bhsd_strided_layout(fa, variant):
+    # (the ping-pong kernel writes its 16-bit output through a tensor map built from these strides)
     cfg = synth.PrefillConfig("t", 2, 4, 2, 300, 300, dtype="fp16", causal=True, seed=9)
     q, k, v = synth.prefill_inputs(cfg, "cpu")
     o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
@@ -208,14 +210,17 @@ def test_bhsd_strided_layout(fa):
     vd = v.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
     o = torch.empty(2, 4, 300, 128, dtype=torch.float16, device=DEV).permute(0, 2, 1, 3)
     lse = torch.empty(2, 4, 300, dtype=torch.float32, device=DEV)
-    fa.fa_forward_ex(qd, kd, vd, o, lse, True, cfg.scale)
+    fa.fa_forward_ex(qd, kd, vd, o, lse, True, cfg.scale, variant=variant)
     torch.cuda.synchronize()
     check_status(fa)
     assert_close_to_oracle(o, lse, o_ref, l_ref, what="BHSD views")
 
 
-def test_output_aligned_to_16_but_not_32_bytes(fa):
-    # rows that start on a 16-byte but not a 32-byte boundary take the 128-bit store path
+@pytest.mark.parametrize("variant", [0, 3, 4])
+def test_output_aligned_to_16_but_not_32_bytes(fa, variant):
+    # rows that start on a 16-byte but not a 32-byte boundary take the 128-bit store path of the
+    # paired-tile kernel; the ping-pong kernel's TMA stores need 16 bytes only.  Nothing may be
+    # written outside the output: its last query tile has 4 live rows of 128.
     cfg = synth.PrefillConfig("t", 1, 2, 2, 260, 260, dtype="fp16", causal=True, seed=12)
     q, k, v = synth.prefill_inputs(cfg, "cpu")
     o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
@@ -225,7 +230,7 @@ def test_output_aligned_to_16_but_not_32_bytes(fa):
     o = buf[base + 8: base + 8 + n].view(1, 260, 2, 128)
     assert o.data_ptr() % 32 == 16
     lse = torch.empty(1, 2, 260, dtype=torch.float32, device=DEV)
-    fa.fa_forward_ex(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, True, cfg.scale)
+    fa.fa_forward_ex(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, True, cfg.scale, variant=variant)
     torch.cuda.synchronize()
     check_status(fa)
     assert_close_to_oracle(o, lse, o_ref, l_ref, what="16-byte aligned output")
