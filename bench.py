@@ -273,6 +273,7 @@ def run_product(args, rank, world, local_rank):
                                           "note": "20 launches without the decode passes between them (inputs 256 MiB > L2); context, not `value`"}
         if not args.small:
             out["prefill_long_context"] = run_long_context(fa, dev, peaks)
+        out["decode_paged"] = run_decode_paged(fa, dec[0], dev, peaks)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
         out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
         print(json.dumps(out), flush=True)
@@ -306,6 +307,32 @@ def run_long_context(fa, dev, peaks):
     if rc != 0:
         raise SystemExit(f"device status {rc} at {where} block {blk}")
     return res
+
+
+def run_decode_paged(fa, d, dev, peaks, page_size=256, iters=5):
+    """The first decode configuration once more with its cache in pages of 256 keys handed out in
+    a seeded random order (fa_decode_paged), outside the timed steps: the same cache bytes
+    through a block table."""
+    cfg = d["cfg"]
+    kp, vp, table = synth.paged_cache(d["k"], d["v"], d["sl_host"], page_size, seed=cfg.seed + 11, spare_pages=4)
+    table = table.to(dev)
+    for _ in range(3):
+        fa.fa_decode_paged(d["q"], kp, vp, table, d["o"], d["lse"], d["sl"], cfg.scale, d["ws"])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_decode_paged(d["q"], kp, vp, table, d["o"], d["lse"], d["sl"], cfg.scale, d["ws"])
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    gbs = d["bytes"] / (ms * 1e-3) / 1e9
+    return {"workload": f"{cfg.name} with the cache in {page_size}-key pages in random order", "ms": round(ms, 4),
+            "gbs": round(gbs, 1), "kv_bytes": d["bytes"], "pages": int(kp.shape[0]),
+            "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4), "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
 
 
 def run_e2e(args, fa, pc, dec, dev):

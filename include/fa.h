@@ -118,6 +118,29 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * Decode over a paged cache: the same computation as fa_decode (Appendix C), with the cached
+ * keys and values of a sequence scattered over fixed-size pages of a pool shared by all
+ * sequences, as serving systems keep them for batched decoding (the batch 8/16 serving runs of
+ * the evaluation section).  Key j of sequence b is row (j mod page_size) of page
+ * block_table[b * table_stride + j / page_size].
+ *   k_pages, v_pages [num_pages, page_size, Hkv, d] fp16 on the device, 16-byte aligned;
+ *   page_size a positive multiple of 128 (a 128-key tile never straddles two pages);
+ *   block_table int32 on the DEVICE, table_stride >= max_pages entries per sequence; only the
+ *   entries that cover keys [0, seqlens_k[b]) are read and they must lie in [0, num_pages)
+ *   (a page index outside that range reads as zeros and never faults); rows of a page past the
+ *   end of its sequence may hold anything (NaN too);
+ *   seqlens_k [B] int32 on the DEVICE, clamped to [0, max_pages * page_size];
+ *   q, o, lse, scale, stream as for fa_decode; workspace of at least
+ *   fa_decode_workspace_bytes(B, Hq, Hkv, max_pages * page_size, d) bytes.
+ * Errors: FA_ERR_SHAPE for page_size not a multiple of 128 or table_stride < max_pages;
+ * otherwise as fa_decode.
+ */
+int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                    void* o, float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages,
+                    int page_size, int max_pages, int table_stride, int d, float scale, void* workspace,
+                    size_t workspace_bytes, void* stream);
+
+/*
  * Decode for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * convenience of this library).  Some hosts of this code may not call cudaMalloc at all: code
  * running inside a framework that owns the memory pool and forbids outside allocations, a

@@ -159,6 +159,32 @@ def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
     return O, LSE
 
 
+def decode_paged(q, k_pages, v_pages, block_table, seqlens, scale: float, nthreads: int = 0):
+    """Decode-stage attention over a paged cache (the decode computation of Appendix C; only
+    the addressing differs): key j of sequence b is row ``j % page_size`` of page
+    ``block_table[b][j // page_size]`` of the ``[num_pages, page_size, Hkv, d]`` pools.  The
+    keys and values of every sequence are first collected, position by position, into
+    contiguous caches; the result is then ``decode`` on those.  Positions at or beyond
+    ``seqlens[b]`` are filled with zeros (they are never read by ``decode``)."""
+    k_pages = torch.as_tensor(k_pages)
+    v_pages = torch.as_tensor(v_pages)
+    table = np.asarray(block_table, dtype=np.int64)
+    sl = np.asarray(seqlens, dtype=np.int64).reshape(-1)
+    num_pages, page_size, Hkv, d = k_pages.shape
+    B = sl.shape[0]
+    Smax = max(1, int(sl.max()) if B else 1)
+    k = torch.zeros(B, Smax, Hkv, d, dtype=k_pages.dtype)
+    v = torch.zeros(B, Smax, Hkv, d, dtype=v_pages.dtype)
+    for b in range(B):
+        for j in range(int(sl[b])):
+            page = int(table[b, j // page_size])
+            if not 0 <= page < num_pages:
+                raise ValueError(f"sequence {b}: key {j} maps to page {page} outside the pool")
+            k[b, j] = k_pages[page, j % page_size]
+            v[b, j] = v_pages[page, j % page_size]
+    return decode(q, k, v, sl.astype(np.int32), scale, nthreads)
+
+
 def bruteforce(q, k, v, causal: bool, scale: float):
     """Extended-precision direct evaluation for tiny inputs (d <= 64): exp(s)/sum exp(s)
     with no max subtraction.  Inputs are converted to contiguous float64."""

@@ -24,6 +24,11 @@ struct DecodeParams {
     int chunk;            // keys per chunk (multiple of kDecTile)
     int n_chunks;         // ceil(Smax / chunk)
     float scale_log2;
+    // paged cache (block_table != nullptr): key j of sequence b is row j % page_size of page
+    // block_table[b * table_stride + j / page_size]; the tensor maps then run over
+    // [pages, page_size, Hkv, 128] and page_size is a multiple of kDecTile
+    const int* block_table;
+    int page_size, table_stride;
 };
 
 
@@ -98,17 +103,27 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     if (warp == 4) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
+            // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
+            // the table read is not on the path that refills a freed slot
+            const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
+            int page_next = table ? table[k_begin / p.page_size] : 0;
             for (int t = 0; t < n_tiles; ++t) {
                 const int st = t % kDecStages;
                 const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                int row0 = k_begin + t * kDecTile;  // first key of the tile within the sequence
+                int slab = b;                        // outermost coordinate: the sequence, or the page
+                if (table) {
+                    slab = page_next;
+                    if (t + 1 < n_tiles) page_next = table[(row0 + kDecTile) / p.page_size];
+                    row0 %= p.page_size;
+                }
                 if (!mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22)) break;
-                const int row0 = k_begin + t * kDecTile;
                 mbar_expect_tx(bk, kDecTileBytes);
-                tma_load_4d(sK + st * kDecTileBytes, &tm_k, bk, 0, hk, row0, b);
-                tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes, &tm_k, bk, 64, hk, row0, b);
+                tma_load_4d(sK + st * kDecTileBytes, &tm_k, bk, 0, hk, row0, slab);
+                tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes, &tm_k, bk, 64, hk, row0, slab);
                 mbar_expect_tx(bv, kDecTileBytes);
-                tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, b);
-                tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, b);
+                tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, slab);
+                tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
             }
         }
         __syncwarp();

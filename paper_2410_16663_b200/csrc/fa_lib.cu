@@ -298,9 +298,14 @@ size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {
     return (size_t)B * Hq * nc * (128 + 1) * sizeof(float);
 }
 
-int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
-              int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
-              void* stream) {
+}  // extern "C"
+
+namespace {
+// Decode over a contiguous cache (block_table == nullptr; k_cache, v_cache [B,Skv_max,Hkv,128])
+// or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
+int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+                int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
+                void* stream, const int* block_table, int num_pages, int page_size, int table_stride) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
     if (Hq % Hkv) return FA_ERR_SHAPE;
     if (d != 128) return FA_ERR_UNSUPPORTED;
@@ -326,14 +331,20 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
     dp.o_part = static_cast<float*>(workspace);
     dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
     dp.scale_log2 = scale * 1.4426950408889634f;
+    dp.block_table = block_table;
+    dp.page_size = block_table ? page_size : 1;
+    dp.table_stride = table_stride;
     const int g = Hq / Hkv;
 
     if (Skv_max > 0) {
+        // the outermost dimension of the maps is the sequence, or the page
+        const int slabs = block_table ? num_pages : B;
+        const int slab_rows = block_table ? page_size : Skv_max;
         CUtensorMap tk, tv;
-        rc = encode_map(&tk, k_cache, B, Skv_max, Hkv, (int64_t)Skv_max * Hkv * 128, (int64_t)Hkv * 128, 128,
+        rc = encode_map(&tk, k_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
                         fa::kDecTile, false);
         if (rc) return rc;
-        rc = encode_map(&tv, v_cache, B, Skv_max, Hkv, (int64_t)Skv_max * Hkv * 128, (int64_t)Hkv * 128, 128,
+        rc = encode_map(&tv, v_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
                         fa::kDecTile, false);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
@@ -349,6 +360,30 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+}  // namespace
+
+extern "C" {
+
+int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+              int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
+              void* stream) {
+    return decode_impl(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, workspace,
+                       workspace_bytes, stream, nullptr, 0, 0, 0);
+}
+
+int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+                    float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
+                    int max_pages, int table_stride, int d, float scale, void* workspace, size_t workspace_bytes,
+                    void* stream) {
+    if (num_pages < 0 || page_size <= 0 || max_pages < 0 || page_size % fa::kDecTile) return FA_ERR_SHAPE;
+    if (table_stride < max_pages) return FA_ERR_SHAPE;
+    if ((long long)max_pages * page_size > 0x7fffffffll) return FA_ERR_SHAPE;
+    if (B > 0 && max_pages > 0 && !block_table) return FA_ERR_NULL;
+    if (max_pages > 0 && num_pages == 0) return FA_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(block_table) & 3u) return FA_ERR_ALIGN;
+    return decode_impl(q, k_pages, v_pages, o, lse, seqlens_k, B, Hq, Hkv, max_pages * page_size, d, scale, workspace,
+                       workspace_bytes, stream, block_table, num_pages, page_size, table_stride);
 }
 
 // ---- decode without a caller workspace -------------------------------------------------------

@@ -134,6 +134,45 @@ def decode_inputs(cfg: DecodeConfig, device="cpu", poison: bool = True):
     return q, k, v, seqlens
 
 
+def paged_cache(k, v, seqlens, page_size: int, seed: int, spare_pages: int = 3, poison: bool = True):
+    """The caches of ``decode_inputs`` laid out in pages: returns ``(k_pages, v_pages, block_table)``.
+
+    ``k_pages``/``v_pages`` are ``[num_pages, page_size, Hkv, d]``; sequence b's keys
+    ``[p*page_size, (p+1)*page_size)`` live in page ``block_table[b, p]``.  Pages are handed out in
+    a seeded random order from a pool with ``spare_pages`` pages nobody uses; table entries past a
+    sequence's last page are -1, and unused pages and the rows of a last page past the end of
+    its sequence hold NaN bit patterns when ``poison`` is set.  Layout only: no arithmetic.
+    """
+    B, Smax, Hkv, d = k.shape
+    max_pages = (Smax + page_size - 1) // page_size
+    need = [(int(n) + page_size - 1) // page_size for n in seqlens]
+    num_pages = sum(need) + spare_pages
+    gen = _gen(seed, "cpu")
+    order = torch.randperm(num_pages, generator=gen).tolist()
+    bits = FP16_NAN_BITS if k.dtype == torch.float16 else BF16_NAN_BITS
+    k_pages = torch.empty(num_pages, page_size, Hkv, d, dtype=k.dtype, device=k.device)
+    v_pages = torch.empty_like(k_pages)
+    if poison:
+        k_pages.view(torch.int16).fill_(bits)
+        v_pages.view(torch.int16).fill_(bits)
+    else:
+        k_pages.zero_()
+        v_pages.zero_()
+    table = torch.full((B, max(1, max_pages)), -1, dtype=torch.int32)
+    nxt = 0
+    for b in range(B):
+        n = int(seqlens[b])
+        for p in range(need[b]):
+            page = order[nxt]
+            nxt += 1
+            table[b, p] = page
+            lo = p * page_size
+            rows = min(page_size, n - lo)
+            k_pages[page, :rows] = k[b, lo:lo + rows]
+            v_pages[page, :rows] = v[b, lo:lo + rows]
+    return k_pages, v_pages, table
+
+
 def sample_rows(cfg: PrefillConfig, n_random: int, seed: int, pairs=None, tile: int = 128):
     """Rows (b, h, i) for row-sampled checks: the first four and the last row, both sides of
     tile boundaries near the start, middle and end, and uniformly random rows, over a few

@@ -106,6 +106,30 @@ def test_decode_validation_and_workspace_size(fa):
     assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 0, 8, 2, 256, 128, 0.1, P(ws), need, None) == fa.FA_OK
 
 
+def test_paged_decode_validation(fa):
+    L = fa.lib
+    q, pool, o = _t(2, 1, 8, 128), _t(6, 128, 2, 128), _t(2, 1, 8, 128)
+    sl = torch.zeros(2, dtype=torch.int32)
+    table = torch.zeros(2, 3, dtype=torch.int32)
+    ws = torch.zeros(1 << 16, dtype=torch.uint8)
+    P = lambda t: t.data_ptr()
+    need = fa.fa_decode_workspace_bytes(2, 8, 2, 3 * 128, 128)
+    call = lambda **kw: L.fa_decode_paged(
+        P(q), P(pool), P(pool), kw.get("table", P(table)), P(o), None, P(sl), kw.get("B", 2), 8, kw.get("Hkv", 2),
+        kw.get("num_pages", 6), kw.get("page_size", 128), kw.get("max_pages", 3), kw.get("stride", 3), 128, 0.1,
+        P(ws), kw.get("wbytes", need), None)
+    assert call(page_size=64) == fa.FA_ERR_SHAPE        # not a multiple of the 128-key tile
+    assert call(page_size=192) == fa.FA_ERR_SHAPE
+    assert call(page_size=0) == fa.FA_ERR_SHAPE
+    assert call(stride=2) == fa.FA_ERR_SHAPE            # rows of the table overlap
+    assert call(num_pages=0) == fa.FA_ERR_SHAPE
+    assert call(table=None) == fa.FA_ERR_NULL
+    assert call(table=P(table) + 2) == fa.FA_ERR_ALIGN
+    assert call(Hkv=3) == fa.FA_ERR_SHAPE
+    assert call(wbytes=need - 1) == fa.FA_ERR_WORKSPACE
+    assert call(B=0) == fa.FA_OK
+
+
 def test_host_entry_validation(fa):
     L = fa.lib
     q = _t(1, 4, 4, 128)

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import oracle
+from paper_2410_16663_b200 import inputs as synth
 
 F64 = torch.float64
 
@@ -283,6 +284,55 @@ def test_decode_equals_attention_over_the_valid_prefix_and_ignores_padding():
         Ob, Lb = oracle.attention_full(q[b:b + 1], k[b:b + 1, :n].contiguous(),
                                        v[b:b + 1, :n].contiguous(), False, 0.4)
         assert torch.equal(O[b], Ob[0, 0]) and torch.equal(LSE[b], Lb[0, :, 0])
+
+
+def test_paged_decode_equals_decode_on_the_same_keys_wherever_the_pages_lie():
+    # the paged form only changes where a key is stored: build the pools by hand (page p of
+    # sequence b at a chosen pool slot), compare with decode on the contiguous caches, then move
+    # the pages around (with the table) and check that nothing changes; tiny page size so that
+    # several pages and a ragged last page occur
+    B, Hq, Hkv, Smax, d, ps = 3, 4, 2, 11, 4, 4
+    q, k, v = rnd((B, 1, Hq, d), 50), rnd((B, Smax, Hkv, d), 51), rnd((B, Smax, Hkv, d), 52)
+    seqlens = [11, 4, 0]
+    O_ref, L_ref = oracle.decode(q, k, v, seqlens, 0.4)
+    for order in ([5, 2, 7, 0, 3, 1, 6, 4], [0, 1, 2, 3, 4, 5, 6, 7]):
+        kp = torch.full((8, ps, Hkv, d), float("nan"), dtype=k.dtype)
+        vp = torch.full((8, ps, Hkv, d), float("nan"), dtype=v.dtype)
+        table = -np.ones((B, 3), dtype=np.int32)
+        nxt = 0
+        for b, n in enumerate(seqlens):
+            for p in range((n + ps - 1) // ps):
+                slot = order[nxt]; nxt += 1
+                table[b, p] = slot
+                for r in range(min(ps, n - p * ps)):
+                    kp[slot, r] = k[b, p * ps + r]
+                    vp[slot, r] = v[b, p * ps + r]
+        O, LSE = oracle.decode_paged(q, kp, vp, table, seqlens, 0.4)
+        assert torch.equal(O, O_ref) and torch.equal(LSE, L_ref)
+    # a table entry outside the pool is an error, not a silent read
+    table[0, 1] = 8
+    with pytest.raises(ValueError):
+        oracle.decode_paged(q, kp, vp, table, seqlens, 0.4)
+
+
+def test_paged_cache_layout_of_the_input_generator_round_trips():
+    # the seeded generator's page layout, read back position by position, is the contiguous cache
+    cfg = synth.DecodeConfig("t", 4, 4, 2, 700, 1, 700, seed=77)
+    q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=True)
+    sl[1] = 0
+    sl[2] = 512            # ends exactly on a page boundary
+    kp, vp, table = synth.paged_cache(k, v, sl, 256, seed=3, spare_pages=2)
+    assert kp.shape[0] == sum((int(n) + 255) // 256 for n in sl) + 2
+    used = table[table >= 0]
+    assert len(set(used.tolist())) == used.numel()          # no page handed out twice
+    for b in range(cfg.B):
+        for j in (0, 1, 255, 256, 257, int(sl[b]) - 1):
+            if 0 <= j < int(sl[b]):
+                page = int(table[b, j // 256])
+                assert torch.equal(kp[page, j % 256], k[b, j]) and torch.equal(vp[page, j % 256], v[b, j])
+    O1, L1 = oracle.decode(q, k, v, sl, cfg.scale)
+    O2, L2 = oracle.decode_paged(q, kp, vp, table, sl, cfg.scale)
+    assert torch.equal(O1, O2) and torch.equal(L1, L2)
 
 
 def test_argument_errors_are_reported():
