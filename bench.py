@@ -274,6 +274,7 @@ def run_product(args, rank, world, local_rank):
         if not args.small:
             out["prefill_long_context"] = run_long_context(fa, dev, peaks)
         out["decode_paged"] = run_decode_paged(fa, dec[0], dev, peaks)
+        out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
         out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
         print(json.dumps(out), flush=True)
@@ -307,6 +308,37 @@ def run_long_context(fa, dev, peaks):
     if rc != 0:
         raise SystemExit(f"device status {rc} at {where} block {blk}")
     return res
+
+
+def run_varlen(fa, dev, peaks, small=False, iters=10):
+    """A packed batch of causal self-attention requests of different lengths (fa_forward_varlen),
+    outside the timed steps: 32 requests with lengths uniform in [256, 8192] (8 in [64, 1024] for
+    the small debugging run), Hq = Hkv = 32, bf16."""
+    cfg = synth.serving_batch("serving-8x", 8, 64, 1024, seed=31, Hq=8, Hkv=8) if small else \
+        synth.serving_batch("serving-32x", 32, 256, 8192, seed=31)
+    q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, dev)
+    cu_q, cu_k = cu_q.to(dev), cu_k.to(dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.Hq, q.shape[0], dtype=torch.float32, device=dev)
+    mq, mk = max(cfg.seqlens_q), max(cfg.seqlens_k)
+    for _ in range(3):
+        fa.fa_forward_varlen(q, k, v, o, lse, cu_q, cu_k, mq, mk, cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_forward_varlen(q, k, v, o, lse, cu_q, cu_k, mq, mk, cfg.causal, cfg.scale)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    tf = cfg.flops() / (ms * 1e-3) / 1e12
+    return {"workload": f"{len(cfg.seqlens_q)} causal requests, lengths {min(cfg.seqlens_q)}..{mq} "
+                        f"(sum {int(q.shape[0])}), Hq=Hkv={cfg.Hq}, bf16, packed", "ms": round(ms, 4),
+            "tflops": round(tf, 1), "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4),
+            "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4)}
 
 
 def run_decode_paged(fa, d, dev, peaks, page_size=256, iters=5):

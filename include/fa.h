@@ -99,6 +99,28 @@ typedef struct fa_params {
 int fa_forward_ex(const fa_params* p, void* stream);
 
 /*
+ * Forward over a packed batch of sequences of different lengths (the batched serving runs of the
+ * evaluation section process requests of unequal length together): the same computation as
+ * fa_forward, sequence by sequence.  Sequence b owns rows [cu_seqlens_q[b], cu_seqlens_q[b+1])
+ * of q and o and rows [cu_seqlens_k[b], cu_seqlens_k[b+1]) of k and v; with the causal mask its
+ * diagonal is aligned bottom-right, as in fa_forward, sequence by sequence.
+ *   q, o [total_q, Hq, d]; k, v [total_k, Hkv, d], contiguous, 16-byte aligned, dtype as given
+ *   (FA_DTYPE_FP16 or FA_DTYPE_BF16; o has the same type); lse [Hq, total_q] float or NULL;
+ *   cu_seqlens_q, cu_seqlens_k: int32 [B + 1] on the DEVICE, non-decreasing, first entry 0, last
+ *   entry total_q / total_k; max_seqlen_q / max_seqlen_k: upper bounds of the sequence lengths
+ *   (they size the launch: a longer sequence would be cut off at the bound).
+ *   A sequence without keys, and under the causal mask every row that sees no key (a sequence
+ *   with more queries than keys), gives O = 0 and LSE = -inf.  The prefix sums are read by the
+ *   kernel only and are not validated.  K and V rows of the NEXT sequence may be loaded and
+ *   multiplied by exact zeros; like everything in k and v they must be finite.
+ * Errors: as fa_forward; FA_ERR_SHAPE also for max_seqlen_q > total_q or max_seqlen_k > total_k.
+ */
+int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, float* lse,
+                      const int* cu_seqlens_q, const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q,
+                      int total_k, int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale,
+                      int dtype, void* stream);
+
+/*
  * Decode stage (Appendix C): one query row per sequence over that sequence's cached keys
  * and values, split along the cache into chunks whose partial results (fp32 O and LSE) are
  * merged by a second kernel with the same rowmax/rowsum recurrence (Appendix A) applied

@@ -140,6 +140,38 @@ def attention_rows(q, k, v, causal: bool, scale: float, rows, nthreads: int = 0)
     return O, LSE
 
 
+def attention_varlen(q, k, v, cu_seqlens_q, cu_seqlens_k, causal: bool, scale: float, nthreads: int = 0):
+    """Standard attention on a packed batch: sequence b owns rows ``[cu_q[b], cu_q[b+1])`` of q
+    ``[total_q,Hq,d]`` and rows ``[cu_k[b], cu_k[b+1])`` of k, v ``[total_k,Hkv,d]``; each
+    sequence is one ``attention_full`` problem.  Returns ``(O [total_q,Hq,d], LSE [Hq,total_q])``
+    float64.  A sequence without keys, and rows that see no key, give O = 0 and LSE = -inf."""
+    q = torch.as_tensor(q)
+    k = torch.as_tensor(k)
+    v = torch.as_tensor(v)
+    cq = np.asarray(cu_seqlens_q, dtype=np.int64).reshape(-1)
+    ck = np.asarray(cu_seqlens_k, dtype=np.int64).reshape(-1)
+    if cq.shape != ck.shape or cq[0] != 0 or ck[0] != 0 or cq[-1] != q.shape[0] or ck[-1] != k.shape[0]:
+        raise ValueError("prefix sums do not match the packed tensors")
+    total_q, Hq, d = q.shape
+    O = torch.zeros(total_q, Hq, d, dtype=torch.float64)
+    LSE = torch.full((Hq, total_q), float("-inf"), dtype=torch.float64)
+    for b in range(cq.shape[0] - 1):
+        q0, q1, k0, k1 = int(cq[b]), int(cq[b + 1]), int(ck[b]), int(ck[b + 1])
+        if q1 < q0 or k1 < k0:
+            raise ValueError("prefix sums must not decrease")
+        if q1 == q0 or k1 == k0:
+            continue
+        n_q, n_k = q1 - q0, k1 - k0
+        lo = 0
+        if causal and n_q > n_k:
+            lo = n_q - n_k          # the first lo rows see no key under the bottom-right mask
+        Ob, Lb = attention_full(q[q0 + lo:q1].unsqueeze(0).contiguous(), k[k0:k1].unsqueeze(0).contiguous(),
+                                v[k0:k1].unsqueeze(0).contiguous(), causal, scale, nthreads)
+        O[q0 + lo:q1] = Ob[0]
+        LSE[:, q0 + lo:q1] = Lb[0]
+    return O, LSE
+
+
 def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
     """Decode-stage attention: q ``[B,1,Hq,d]`` over the first ``seqlens[b]`` rows of
     the ``[B,Smax,Hkv,d]`` caches.  Returns ``(O [B,Hq,d], LSE [B,Hq])`` float64."""

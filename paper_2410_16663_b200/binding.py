@@ -45,6 +45,8 @@ lib.fa_decode.restype = _i
 lib.fa_decode.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_workspace_bytes.restype = _sz
 lib.fa_decode_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
+lib.fa_forward_varlen.restype = _i
+lib.fa_forward_varlen.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p]
 lib.fa_decode_paged.restype = _i
 lib.fa_decode_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_noalloc.restype = _i
@@ -63,7 +65,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -128,6 +130,20 @@ def fa_forward_ex(q, k, v, o, lse, causal: bool, scale: float, variant: int = 0,
     p.variant = int(variant)
     rc = lib.fa_forward_ex(ctypes.byref(p), _stream())
     return _check(rc, "fa_forward_ex", raise_on_error)
+
+
+def fa_forward_varlen(q, k, v, o, lse, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int,
+                      causal: bool, scale: float, raise_on_error: bool = True) -> int:
+    """``fa_forward_varlen``: q, o [total_q,Hq,d], k, v [total_k,Hkv,d] contiguous device tensors,
+    lse [Hq,total_q] or None, cu_seqlens_* int32 [B+1] on the device."""
+    total_q, Hq, d = q.shape
+    total_k, Hkv, _ = k.shape
+    B = cu_seqlens_q.numel() - 1
+    dt = FA_DTYPE_BF16 if q.dtype == torch.bfloat16 else FA_DTYPE_FP16
+    rc = lib.fa_forward_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens_q),
+                               _ptr(cu_seqlens_k), B, Hq, Hkv, total_q, total_k, int(max_seqlen_q),
+                               int(max_seqlen_k), d, int(bool(causal)), float(scale), dt, _stream())
+    return _check(rc, "fa_forward_varlen", raise_on_error)
 
 
 def fa_decode_workspace_bytes(B: int, Hq: int, Hkv: int, Skv_max: int, d: int) -> int:

@@ -170,6 +170,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.cls_log2 = 0;  // set by the ping-pong launcher
     fp.by_class.set(1);
     fp.by_lastcls.set(1);
+    fp.cu_q = nullptr;
+    fp.cu_k = nullptr;
+    fp.total_q = 0;
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
     const bool bf16 = p.dtype == FA_DTYPE_BF16;
@@ -289,6 +292,76 @@ int fa_forward_bf16(const void* q, const void* k, const void* v, void* o, float*
 int fa_forward_ex(const fa_params* p, void* stream) {
     if (!p) return FA_ERR_NULL;
     return forward_impl(*p, static_cast<cudaStream_t>(stream));
+}
+
+int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens_q,
+                      const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q, int total_k, int max_seqlen_q,
+                      int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || total_q < 0 || total_k < 0 || max_seqlen_q < 0 || max_seqlen_k < 0 || d <= 0)
+        return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (max_seqlen_q > total_q || max_seqlen_k > total_k) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
+    if (Hq > 65535 || B > 65535) return FA_ERR_UNSUPPORTED;
+    if (B == 0 || total_q == 0 || max_seqlen_q == 0) return FA_OK;
+    if (!q || !o || !cu_seqlens_q || !cu_seqlens_k) return FA_ERR_NULL;
+    if (total_k > 0 && (!k || !v)) return FA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return FA_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(cu_seqlens_q) | reinterpret_cast<uintptr_t>(cu_seqlens_k) |
+         reinterpret_cast<uintptr_t>(lse)) & 3u)
+        return FA_ERR_ALIGN;
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf16 = dtype == FA_DTYPE_BF16;
+
+    fa::FwdParams fp;
+    fp.o = o;
+    fp.lse = lse;
+    fp.B = B; fp.Hq = Hq; fp.Hkv = Hkv; fp.Sq = max_seqlen_q; fp.Skv = max_seqlen_k;
+    fp.causal = causal ? 1 : 0;
+    fp.scale_log2 = fmaxf(scale * 1.4426950408889634f, 1e-30f);
+    fp.o_sb = 0; fp.o_ss = (long long)Hq * 128; fp.o_sh = 128;
+    fp.o_fp32 = 0;
+    fp.o_align32 = 0;
+    fp.n_qtiles = (max_seqlen_q + fa::kTile - 1) / fa::kTile;
+    fp.by_bh.set(B * Hq);
+    fp.by_hq.set(Hq);
+    fp.by_group.set(Hq / Hkv);
+    fp.by_qtiles.set(fp.n_qtiles);
+    fp.by_qpairs.set((fp.n_qtiles + 1) / 2);
+    fp.cls_log2 = 0;
+    fp.by_class.set(1);
+    fp.by_lastcls.set(1);
+    fp.cu_q = cu_seqlens_q;
+    fp.cu_k = cu_seqlens_k;
+    fp.total_q = total_q;
+
+    if (total_k == 0 || max_seqlen_k == 0) {
+        // no keys anywhere: O = 0, LSE = -inf over the packed rows, seen as one sequence
+        fa::FwdParams fe = fp;
+        fe.B = 1; fe.Sq = total_q;
+        const long long rows = (long long)total_q * Hq;
+        const int blocks = (int)((rows + 127) / 128 < 4096 ? (rows + 127) / 128 : 4096);
+        if (bf16) fa::fa_fill_empty_kernel<__nv_bfloat16><<<blocks, 128, 0, st>>>(fe);
+        else fa::fa_fill_empty_kernel<__half><<<blocks, 128, 0, st>>>(fe);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
+    // the packed tensors as one batch entry; a sequence's rows are reached through the prefix sums
+    CUtensorMap tq, tk, tv, to;
+    rc = encode_map(&tq, q, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tk, k, 1, total_k, Hkv, (int64_t)total_k * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tv, v, 1, total_k, Hkv, (int64_t)total_k * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&to, o, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 32, bf16);
+    if (rc) return rc;
+    return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
+                : fa::launch_pingpong<__half>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
 }
 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {

@@ -79,6 +79,9 @@ static_assert(sizeof(PpStatic) == 3072, "static shared state must fill exactly 3
 
 struct PpItem {
     int b, h, hk, q0, n;
+    // packed variable-length batches only: first row of the sequence in q/o and in k/v, and
+    // the sequence's own lengths
+    int q_base, k_base, Sq, Skv;
 };
 
 // Work item `idx`.  The query tiles of a head are taken in classes of C = 2^cls_log2 consecutive
@@ -88,6 +91,10 @@ struct PpItem {
 // read them, and the rounds still get shorter and shorter items, which keeps the static
 // assignment balanced (the launcher picks C from the K/V bytes of a head, see launch_pingpong).
 // C >= n_qtiles is the plain head-by-head order used for very long sequences.
+// kVarlen: the sequence's lengths come from the prefix sums; n == 0 marks an item past the end
+// of its sequence (every role skips it), and a live item visits at least one kv tile (so that
+// rows without any visible key are still written, as zeros).
+template <bool kVarlen>
 __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
     PpItem it;
     int c, rem;  // class, index inside the class
@@ -104,9 +111,38 @@ __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
     p.by_hq.divmod(bh, it.b, it.h);
     it.hk = p.by_group.div(it.h);
     it.q0 = qt * kTile;
-    it.n = kv_tiles_for(it.q0, kTile, p.Sq, p.Skv, p.causal);
+    if (kVarlen) {
+        it.q_base = p.cu_q[it.b];
+        it.k_base = p.cu_k[it.b];
+        it.Sq = p.cu_q[it.b + 1] - it.q_base;
+        it.Skv = p.cu_k[it.b + 1] - it.k_base;
+        it.n = (it.q0 < it.Sq) ? max(1, kv_tiles_for(it.q0, kTile, it.Sq, it.Skv, p.causal)) : 0;
+    } else {
+        it.n = kv_tiles_for(it.q0, kTile, p.Sq, p.Skv, p.causal);
+    }
     return it;
 }
+
+// The items of this CTA in order.  `ord` counts the items the CTA works on (it selects the
+// double buffers); with variable-length batches the items past the end of their sequence are
+// passed over, identically in every role.
+template <bool kVarlen>
+struct PpItems {
+    int round = -1, ord = -1;
+    PpItem it;
+    __device__ __forceinline__ bool next(const FwdParams& p, int total_items) {
+        for (;;) {
+            ++round;
+            const int idx = item_of_round(round, total_items);
+            if (idx >= total_items) return false;
+            it = pp_decode_item<kVarlen>(p, idx);
+            if (!kVarlen || it.n > 0) {
+                ++ord;
+                return true;
+            }
+        }
+    }
+};
 
 // Row max of 128 raw scores.
 __device__ __forceinline__ float pp_row_max(const uint32_t (&s)[128]) {
@@ -166,17 +202,17 @@ struct PpRing {
 };
 
 // The thread that issues S = Q K^T of every step.
-template <typename T, bool kTmaOut>
+template <typename T, bool kTmaOut, bool kVarlen>
 __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK, uint32_t tmem, const FwdParams& p,
                                          int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
     constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, false);
     uint32_t g = 0;
     PpRing<kPpNK> ring;
-    for (int ord = 0;; ++ord) {
-        const int idx = item_of_round(ord, total_items);
-        if (idx >= total_items) break;
-        const PpItem it = pp_decode_item(p, idx);
+    PpItems<kVarlen> items;
+    while (items.next(p, total_items)) {
+        const int ord = items.ord;
+        const PpItem& it = items.it;
         const uint32_t qb = ord & 1;
         if (!mbar_wait(pp_bar(bar0, ppb::q_full + qb), (ord >> 1) & 1, abort_flag, 130)) return;
         const uint32_t a_lo = desc_lo(sQ + qb * kTileBytes, 16);
@@ -202,17 +238,17 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
 }
 
 // The thread that issues O += P V of every step.
-template <typename T>
+template <typename T, bool kVarlen>
 __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t tmem, const FwdParams& p,
                                           int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
     constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, true);
     uint32_t g = 0;
     PpRing<kPpNV> ring;
-    for (int ord = 0;; ++ord) {
-        const int idx = item_of_round(ord, total_items);
-        if (idx >= total_items) break;
-        const PpItem it = pp_decode_item(p, idx);
+    PpItems<kVarlen> items;
+    while (items.next(p, total_items)) {
+        const int ord = items.ord;
+        const PpItem& it = items.it;
         for (int j = 0; j < it.n; ++j, ++g, ring.next()) {
             const uint32_t buf = g & 1;
             if (!mbar_wait(pp_bar(bar0, ppb::v_full + ring.slot), ring.par, abort_flag, 140)) return;
@@ -232,7 +268,9 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
     }
 }
 
-// The thread that loads Q of every item and K of every step.
+// The thread that loads Q of every item and K of every step.  (Packed batches: the tensor maps
+// have one batch entry that holds every sequence back to back.)
+template <bool kVarlen>
 __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint32_t sK, const CUtensorMap* tm_q,
                                                const CUtensorMap* tm_k, const FwdParams& p, int total_items,
                                                volatile uint32_t* abort_flag) {
@@ -240,37 +278,41 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
     tma_prefetch_desc(tm_k);
     const uint64_t pol_q = l2_policy_evict_first(), pol_kv = l2_policy_evict_last();
     PpRing<kPpNK> ring;
-    for (int ord = 0;; ++ord) {
-        const int idx = item_of_round(ord, total_items);
-        if (idx >= total_items) break;
-        const PpItem it = pp_decode_item(p, idx);
+    PpItems<kVarlen> items;
+    while (items.next(p, total_items)) {
+        const int ord = items.ord;
+        const PpItem& it = items.it;
         const uint32_t qb = ord & 1;
         // passes at once the first time each buffer is used
         if (!mbar_wait(pp_bar(bar0, ppb::q_empty + qb), ((ord >> 1) & 1) ^ 1, abort_flag, 150)) return;
         mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
-        load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h, it.q0, it.b, pol_q);
+        load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
+                       kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
-            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, j * kTile, it.b, pol_kv);
+            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk,
+                           kVarlen ? it.k_base + j * kTile : j * kTile, kVarlen ? 0 : it.b, pol_kv);
         }
     }
 }
 
 // The thread that loads V of every step.
+template <bool kVarlen>
 __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const CUtensorMap* tm_v, const FwdParams& p,
                                               int total_items, volatile uint32_t* abort_flag) {
     tma_prefetch_desc(tm_v);
     const uint64_t pol_kv = l2_policy_evict_last();
     PpRing<kPpNV> ring;
-    for (int ord = 0;; ++ord) {
-        const int idx = item_of_round(ord, total_items);
-        if (idx >= total_items) break;
-        const PpItem it = pp_decode_item(p, idx);
+    PpItems<kVarlen> items;
+    while (items.next(p, total_items)) {
+        const int ord = items.ord;
+        const PpItem& it = items.it;
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
-            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, j * kTile, it.b, pol_kv);
+            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk,
+                           kVarlen ? it.k_base + j * kTile : j * kTile, kVarlen ? 0 : it.b, pol_kv);
         }
     }
 }
@@ -412,7 +454,8 @@ struct PpSoftmax {
 // little slower per step and much smaller: with it, what an item executes from its first step
 // to its epilogue stays within the 32 KB the instruction cache serves at full rate, which is
 // what counts when an item has few steps.
-template <typename T, bool kTmaOut, bool kSingle>
+// kVarlen (needs kTmaOut): a packed batch of sequences of different lengths (see FwdParams).
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -494,12 +537,18 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 q_back = -1;
             }
         };
-        for (int ord = 0; ok; ++ord) {
-            const int idx = item_of_round(ord, total_items);
-            if (idx >= total_items) break;
-            const PpItem it = pp_decode_item(p, idx);
+        PpItems<kVarlen> items;
+        while (ok && items.next(p, total_items)) {
+            const int ord = items.ord;
+            const PpItem& it = items.it;
             const int n = it.n;
-            const int row = it.q0 + r;
+            const int row = it.q0 + r;   // within the sequence
+            const int Sq_i = kVarlen ? it.Sq : p.Sq, Skv_i = kVarlen ? it.Skv : p.Skv;
+            const int off_i = kVarlen ? it.Skv - it.Sq : off;
+            if (kVarlen) {
+                sm.Skv = Skv_i;
+                sm.off = off_i;
+            }
             sm.row = row;
             sm.l_part = 0.f;
             sm.m_loc = -INFINITY;
@@ -509,8 +558,8 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             // kv tiles every row of the query tile sees in full: they come first and take the
             // loop without mask code; the few tiles crossed by the diagonal or by the end of the
             // keys follow
-            int n_full = p.Skv / kTile;
-            if (p.causal) n_full = min(n_full, max(0, (it.q0 + off + 1) / kTile));
+            int n_full = Skv_i / kTile;
+            if (p.causal) n_full = min(n_full, max(0, (it.q0 + off_i + 1) / kTile));
             n_full = min(n_full, n);
             // this warpgroup's steps of the item: those with an absolute step number of its parity
             const uint32_t g_item = g;
@@ -570,11 +619,13 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 tc_fence_before();
                 mbar_arrive(pp_bar(bar0, ppb::o_free));
                 const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-                const long long obase = (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
-                if (row < p.Sq && p.lse != nullptr) {
+                const long long obase = kVarlen ? (long long)(it.q_base + row) * p.o_ss + (long long)it.h * p.o_sh
+                                                : (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
+                if (row < Sq_i && p.lse != nullptr) {
                     const float lse = (l_run > 0.f) ? (m_loc * scale_log2 + log2f(l_run)) * 0.6931471805599453f
                                                     : -INFINITY;
-                    p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
+                    if (kVarlen) p.lse[(long long)it.h * p.total_q + it.q_base + row] = lse;
+                    else p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
                 }
                 if (kTmaOut) {
                     const uint32_t q_buf = sQ + (uint32_t)(ord & 1) * kTileBytes;
@@ -591,18 +642,30 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) {
-                        const int row0 = it.q0 + (warp & 3) * 32;
-                        if (row0 < p.Sq) {
-                            const uint32_t src = q_buf + (uint32_t)(warp & 3) * 4096u;
-                            tma_store_4d(&tm_o, src, 0, it.h, row0, it.b);
-                            tma_store_4d(&tm_o, src + kHalfBytes, 64, it.h, row0, it.b);
-                            tma_store_commit();
-                        }
+                    const int row0 = it.q0 + (warp & 3) * 32;   // first row of this warp
+                    // packed batches: the rows after a sequence's last belong to the next
+                    // sequence, so only a warp whose 32 rows all exist may use the box store
+                    const bool box = kVarlen ? (row0 + 32 <= Sq_i) : (row0 < Sq_i);
+                    if (lane == 0 && box) {
+                        const uint32_t src = q_buf + (uint32_t)(warp & 3) * 4096u;
+                        tma_store_4d(&tm_o, src, 0, it.h, kVarlen ? it.q_base + row0 : row0, kVarlen ? 0 : it.b);
+                        tma_store_4d(&tm_o, src + kHalfBytes, 64, it.h, kVarlen ? it.q_base + row0 : row0, kVarlen ? 0 : it.b);
+                        tma_store_commit();
                     }
                     q_back = ord & 1;  // handed back to the loader after this warp's next step
                     __syncwarp();
-                } else if (row < p.Sq) {
+                    if (kVarlen && !box && row < Sq_i) {
+                        // the ragged end of a sequence: each thread writes its own row
+                        T* dst = static_cast<T*>(p.o) + obase;
+#pragma unroll
+                        for (int c = 0; c < 16; ++c)
+                            reinterpret_cast<uint4*>(dst)[c] =
+                                make_uint4(pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 2]) * inv_l, __uint_as_float(s[8 * c + 3]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 4]) * inv_l, __uint_as_float(s[8 * c + 5]) * inv_l),
+                                           pack2<T>(__uint_as_float(s[8 * c + 6]) * inv_l, __uint_as_float(s[8 * c + 7]) * inv_l));
+                    }
+                } else if (row < Sq_i) {
                     if (p.o_fp32) {
                         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
 #pragma unroll
@@ -630,10 +693,10 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else {
         setmaxnreg_dec<kPipeOtherRegs>();
         if (lane == 0) {
-            if (warp == 8) pp_run_s<T, kTmaOut>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
-            else if (warp == 10) pp_run_pv<T>(bar0, sV, tmem_base, p, total_items, abort_flag);
-            else if (warp == 9) pp_run_load_qk(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
-            else pp_run_load_v(bar0, sV, &tm_v, p, total_items, abort_flag);
+            if (warp == 8) pp_run_s<T, kTmaOut, kVarlen>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
+            else if (warp == 10) pp_run_pv<T, kVarlen>(bar0, sV, tmem_base, p, total_items, abort_flag);
+            else if (warp == 9) pp_run_load_qk<kVarlen>(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
+            else pp_run_load_v<kVarlen>(bar0, sV, &tm_v, p, total_items, abort_flag);
         }
         __syncwarp();
     }
@@ -655,8 +718,12 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
     // the single-copy step up to 32 kv tiles per item (timed: ahead by 3 % at 2048 keys, level at
     // 4096, behind by 1 % at 8192)
     const bool single = fp.o_fp32 || fp.Skv <= 32 * kTile;
-    auto kern = fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true>
-                          : (single ? fa_fwd_pingpong_kernel<T, true, true> : fa_fwd_pingpong_kernel<T, true, false>);
+    const bool varlen = fp.cu_q != nullptr;
+    if (varlen && fp.o_fp32) return -3;
+    auto kern = varlen ? fa_fwd_pingpong_kernel<T, true, true, true>
+                       : (fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true, false>
+                                    : (single ? fa_fwd_pingpong_kernel<T, true, true, false>
+                                              : fa_fwd_pingpong_kernel<T, true, false, false>));
     int sm_count = 0;
     cudaError_t e;
     if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }

@@ -52,6 +52,12 @@ struct FwdParams {
     // the size of the last (possibly smaller) class
     int cls_log2;
     FastDiv by_class, by_lastcls;
+    // packed variable-length batch (ping-pong kernel only; nullptr otherwise): sequence b owns
+    // rows [cu_q[b], cu_q[b+1]) of q and o and rows [cu_k[b], cu_k[b+1]) of k and v; Sq and Skv
+    // above are then the longest sequence's, and lse is [Hq, total_q]
+    const int* cu_q;
+    const int* cu_k;
+    int total_q;
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim

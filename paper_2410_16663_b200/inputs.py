@@ -47,6 +47,49 @@ class PrefillConfig:
 
 
 @dataclass(frozen=True)
+class VarlenConfig:
+    """A packed batch of sequences of different lengths (query and key lengths per sequence)."""
+    name: str
+    Hq: int
+    Hkv: int
+    seqlens_q: tuple
+    seqlens_k: tuple
+    d: int = 128
+    dtype: str = "fp16"
+    causal: bool = True
+    seed: int = 0
+
+    @property
+    def scale(self) -> float:
+        return 1.0 / math.sqrt(self.d)
+
+    @property
+    def torch_dtype(self):
+        return torch.float16 if self.dtype == "fp16" else torch.bfloat16
+
+    def flops(self) -> float:
+        """Credited FLOPs: 4*Hq*d per visible (query, key) pair of every sequence."""
+        pairs = 0
+        for nq, nk in zip(self.seqlens_q, self.seqlens_k):
+            if self.causal:
+                lo = max(0, nq - nk)                 # rows that see no key
+                rows = nq - lo
+                pairs += rows * (nk - rows) + rows * (rows + 1) // 2
+            else:
+                pairs += nq * nk
+        return 4.0 * self.Hq * self.d * pairs
+
+
+def serving_batch(name: str, n_seqs: int, len_lo: int, len_hi: int, seed: int, Hq: int = 32, Hkv: int = 32,
+                  dtype: str = "bf16") -> VarlenConfig:
+    """Self-attention prefill of ``n_seqs`` requests whose lengths are uniform in [len_lo, len_hi]."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(int(seed) + 13)
+    lens = tuple(int(x) for x in torch.randint(len_lo, len_hi + 1, (n_seqs,), generator=gen))
+    return VarlenConfig(name, Hq, Hkv, lens, lens, dtype=dtype, causal=True, seed=seed)
+
+
+@dataclass(frozen=True)
 class DecodeConfig:
     name: str
     B: int
@@ -103,6 +146,21 @@ def prefill_inputs(cfg: PrefillConfig, device="cpu"):
     k = _randn((cfg.B, cfg.Skv, cfg.Hkv, cfg.d), dt, gen, device)
     v = _randn((cfg.B, cfg.Skv, cfg.Hkv, cfg.d), dt, gen, device)
     return q, k, v
+
+
+def varlen_inputs(cfg: VarlenConfig, device="cpu"):
+    """q [total_q,Hq,d], k and v [total_k,Hkv,d], cu_seqlens_q, cu_seqlens_k (int32 [B+1], host)."""
+    device = torch.device(device)
+    gen = _gen(cfg.seed, device)
+    dt = cfg.torch_dtype
+    cu_q = torch.zeros(len(cfg.seqlens_q) + 1, dtype=torch.int32)
+    cu_k = torch.zeros(len(cfg.seqlens_k) + 1, dtype=torch.int32)
+    cu_q[1:] = torch.cumsum(torch.tensor(cfg.seqlens_q, dtype=torch.int64), 0).to(torch.int32)
+    cu_k[1:] = torch.cumsum(torch.tensor(cfg.seqlens_k, dtype=torch.int64), 0).to(torch.int32)
+    q = _randn((int(cu_q[-1]), cfg.Hq, cfg.d), dt, gen, device)
+    k = _randn((int(cu_k[-1]), cfg.Hkv, cfg.d), dt, gen, device)
+    v = _randn((int(cu_k[-1]), cfg.Hkv, cfg.d), dt, gen, device)
+    return q, k, v, cu_q, cu_k
 
 
 def decode_seqlens(cfg: DecodeConfig) -> torch.Tensor:

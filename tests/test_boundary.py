@@ -106,6 +106,29 @@ def test_decode_validation_and_workspace_size(fa):
     assert L.fa_decode(P(q), P(kc), P(kc), P(o), None, P(sl), 0, 8, 2, 256, 128, 0.1, P(ws), need, None) == fa.FA_OK
 
 
+def test_varlen_validation(fa):
+    L = fa.lib
+    q, k, o = _t(20, 4, 128), _t(30, 2, 128), _t(20, 4, 128)
+    cu = torch.zeros(3, dtype=torch.int32)
+    P = lambda t: t.data_ptr()
+    call = lambda **kw: L.fa_forward_varlen(
+        kw.get("q", P(q)), P(k), P(k), P(o), None, kw.get("cu", P(cu)), P(cu), kw.get("B", 2), 4, kw.get("Hkv", 2),
+        20, 30, kw.get("max_q", 12), kw.get("max_k", 16), kw.get("d", 128), 1, kw.get("scale", 0.1),
+        kw.get("dtype", fa.FA_DTYPE_FP16), None)
+    assert call(Hkv=3) == fa.FA_ERR_SHAPE
+    assert call(max_q=21) == fa.FA_ERR_SHAPE
+    assert call(max_k=31) == fa.FA_ERR_SHAPE
+    assert call(d=64) == fa.FA_ERR_UNSUPPORTED
+    assert call(dtype=fa.FA_DTYPE_FP32) == fa.FA_ERR_UNSUPPORTED
+    assert call(scale=float("nan")) == fa.FA_ERR_UNSUPPORTED
+    assert call(cu=None) == fa.FA_ERR_NULL
+    assert call(q=None) == fa.FA_ERR_NULL
+    assert call(q=P(q) + 8) == fa.FA_ERR_ALIGN
+    assert call(cu=P(cu) + 2) == fa.FA_ERR_ALIGN
+    assert call(B=0) == fa.FA_OK
+    assert call(max_q=0) == fa.FA_OK
+
+
 def test_paged_decode_validation(fa):
     L = fa.lib
     q, pool, o = _t(2, 1, 8, 128), _t(6, 128, 2, 128), _t(2, 1, 8, 128)

@@ -286,6 +286,44 @@ def test_decode_equals_attention_over_the_valid_prefix_and_ignores_padding():
         assert torch.equal(O[b], Ob[0, 0]) and torch.equal(LSE[b], Lb[0, :, 0])
 
 
+def test_varlen_attention_is_attention_of_each_sequence_alone():
+    # a packed batch with equal lengths is the batched problem; with unequal lengths every
+    # sequence must come out as if it were alone (checked against the extended-precision brute
+    # force on its own slice), whatever its neighbours hold
+    B, S, Hq, Hkv, d = 3, 7, 4, 2, 8
+    q, k, v = rnd((B, S, Hq, d), 60), rnd((B, S, Hkv, d), 61), rnd((B, S, Hkv, d), 62)
+    cu = [0, 7, 14, 21]
+    for causal in (False, True):
+        O_ref, L_ref = oracle.attention_full(q, k, v, causal, 0.3)
+        O, LSE = oracle.attention_varlen(q.reshape(B * S, Hq, d), k.reshape(B * S, Hkv, d), v.reshape(B * S, Hkv, d),
+                                         cu, cu, causal, 0.3)
+        assert torch.equal(O.reshape(B, S, Hq, d), O_ref)
+        assert torch.equal(LSE.reshape(Hq, B, S).permute(1, 0, 2), L_ref)
+    lens_q, lens_k = [5, 0, 3, 2, 6], [9, 4, 3, 0, 2]        # chunked, no queries, square, no keys, more queries than keys
+    cq, ck = np.concatenate([[0], np.cumsum(lens_q)]), np.concatenate([[0], np.cumsum(lens_k)])
+    qp, kp, vp = rnd((int(cq[-1]), Hq, d), 63), rnd((int(ck[-1]), Hkv, d), 64), rnd((int(ck[-1]), Hkv, d), 65)
+    for causal in (False, True):
+        O, LSE = oracle.attention_varlen(qp, kp, vp, cq, ck, causal, 0.3)
+        for b, (nq, nk) in enumerate(zip(lens_q, lens_k)):
+            rows = slice(int(cq[b]), int(cq[b + 1]))
+            if nq == 0:
+                continue
+            if nk == 0:
+                assert float(O[rows].abs().max()) == 0.0 and torch.isneginf(LSE[:, rows]).all()
+                continue
+            hidden = max(0, nq - nk) if causal else 0      # rows above the bottom-right diagonal's first column
+            if hidden:
+                top = slice(int(cq[b]), int(cq[b]) + hidden)
+                assert float(O[top].abs().max()) == 0.0 and torch.isneginf(LSE[:, top]).all()
+            vis = slice(int(cq[b]) + hidden, int(cq[b + 1]))
+            Ob, Lb = oracle.bruteforce(qp[vis].unsqueeze(0), kp[int(ck[b]):int(ck[b + 1])].unsqueeze(0),
+                                       vp[int(ck[b]):int(ck[b + 1])].unsqueeze(0), causal, 0.3)
+            assert float((O[vis] - Ob[0]).abs().max()) < 1e-12
+            assert float((LSE[:, vis] - Lb[0]).abs().max()) < 1e-12
+    with pytest.raises(ValueError):
+        oracle.attention_varlen(qp, kp, vp, cq[:-1], ck[:-1], False, 0.3)   # sums do not reach the end
+
+
 def test_paged_decode_equals_decode_on_the_same_keys_wherever_the_pages_lie():
     # the paged form only changes where a key is stored: build the pools by hand (page p of
     # sequence b at a chosen pool slot), compare with decode on the contiguous caches, then move

@@ -317,6 +317,72 @@ def test_c4_gqa_sampled(fa):
     assert sampled_case(fa, synth.C4_NC, 64) >= 256
 
 
+# ------------------------------------------------------------------ packed variable-length batches
+def varlen_case(fa, cfg, what):
+    q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
+    o_ref, l_ref = oracle.attention_varlen(q, k, v, cu_q, cu_k, cfg.causal, cfg.scale)
+    absv = oracle.attention_varlen(q, k, v.abs(), cu_q, cu_k, cfg.causal, cfg.scale)[0] if cfg.dtype == "bf16" else None
+    o, chk_o = guard_alloc(tuple(q.shape), q.dtype, DEV)
+    lse, chk_l = guard_alloc((cfg.Hq, q.shape[0]), torch.float32, DEV)
+    fa.fa_forward_varlen(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, cu_q.to(DEV), cu_k.to(DEV),
+                         max(cfg.seqlens_q), max(cfg.seqlens_k), cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l()
+    # the comparison helper takes [B,S,H,d] and [B,H,S]: the packed rows as one sequence
+    assert_close_to_oracle(o.unsqueeze(0), lse.unsqueeze(0), o_ref.unsqueeze(0), l_ref.unsqueeze(0),
+                           stored_bf16=(cfg.dtype == "bf16"), p_absv=None if absv is None else absv.unsqueeze(0), what=what)
+    return o, lse
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_varlen_ragged_batch(fa, causal, dtype):
+    # lengths on both sides of the 32-row store boxes and the 128-row tiles, an empty sequence,
+    # a sequence without keys, chunked prefill (fewer queries than keys), more queries than keys
+    # (causal: its first rows see nothing), GQA; every row of O and LSE is compared and the
+    # guard bands around both must stay untouched
+    lq = (1, 127, 128, 129, 300, 0, 40, 33, 200, 31, 260)
+    lk = (1, 127, 128, 129, 300, 0, 700, 0, 90, 31, 515)
+    cfg = synth.VarlenConfig("t", 4, 2, lq, lk, dtype=dtype, causal=causal, seed=600 + int(causal))
+    varlen_case(fa, cfg, f"varlen ragged causal{int(causal)} {dtype}")
+
+
+def test_varlen_many_short_sequences_and_one_long(fa):
+    # more items than CTAs, most of them past the end of their sequence (the launch is sized by
+    # the longest sequence): skipped items must not disturb the double buffers
+    lens = tuple([17, 130, 64, 5] * 40 + [2500])
+    cfg = synth.VarlenConfig("t", 2, 1, lens, lens, dtype="fp16", causal=True, seed=611)
+    varlen_case(fa, cfg, "varlen many short + one long")
+
+
+def test_varlen_equal_lengths_match_the_batched_call_bit_for_bit(fa):
+    # C2 as a packed batch must give exactly what fa_forward gives (same kernel arithmetic in the
+    # same order; fa_forward on C2 is checked against the oracle elsewhere)
+    c = synth.C2
+    q, k, v = synth.prefill_inputs(c, DEV)
+    o1 = torch.empty_like(q); l1 = torch.empty(c.B, c.Hq, c.Sq, dtype=torch.float32, device=DEV)
+    fa.fa_forward(q, k, v, o1, l1, c.causal, c.scale)
+    cu = torch.arange(0, (c.B + 1) * c.Sq, c.Sq, dtype=torch.int32, device=DEV)
+    o2 = torch.empty(c.B * c.Sq, c.Hq, c.d, dtype=q.dtype, device=DEV)
+    l2 = torch.empty(c.Hq, c.B * c.Sq, dtype=torch.float32, device=DEV)
+    fa.fa_forward_varlen(q.view(-1, c.Hq, c.d), k.view(-1, c.Hkv, c.d), v.view(-1, c.Hkv, c.d), o2, l2, cu, cu,
+                         c.Sq, c.Skv, c.causal, c.scale)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert torch.equal(o1.view(-1, c.Hq, c.d), o2)
+    assert torch.equal(l1, l2.view(c.Hq, c.B, c.Sq).permute(1, 0, 2))
+
+
+def test_varlen_without_any_keys(fa):
+    cfg = synth.VarlenConfig("t", 2, 2, (5, 130), (0, 0), dtype="fp16", causal=False, seed=612)
+    q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, DEV)
+    o = torch.full_like(q, float("nan")); lse = torch.full((2, 135), float("nan"), device=DEV)
+    fa.fa_forward_varlen(q, k, v, o, lse, cu_q.to(DEV), cu_k.to(DEV), 130, 0, False, cfg.scale)
+    torch.cuda.synchronize()
+    assert float(o.abs().max()) == 0.0 and torch.isneginf(lse).all()
+
+
 # ------------------------------------------------------------------ decode
 def run_decode(fa, q, k, v, seqlens_dev, scale):
     B, _, Hq, d = q.shape
