@@ -275,6 +275,7 @@ def run_product(args, rank, world, local_rank):
             out["prefill_long_context"] = run_long_context(fa, dev, peaks)
         out["decode_paged"] = run_decode_paged(fa, dec[0], dev, peaks)
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
+        out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
         out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
         print(json.dumps(out), flush=True)
@@ -308,6 +309,37 @@ def run_long_context(fa, dev, peaks):
     if rc != 0:
         raise SystemExit(f"device status {rc} at {where} block {blk}")
     return res
+
+
+def run_d64(fa, dev, peaks, small=False, iters=10):
+    """The short non-causal vision workload with head dimension 64 (197 tokens, 12 heads, batch
+    1024; batch 64 for the small debugging run), outside the timed steps.  With 99 FLOPs per byte
+    of q, k, v, o the shape sits under the HBM roof, so both rates are printed."""
+    cfg = synth.DEIT_B if not small else synth.PrefillConfig("DeiT-B-small", 64, 12, 12, 197, 197, d=64,
+                                                             dtype="fp16", causal=False, seed=1031)
+    q, k, v = synth.prefill_inputs(cfg, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+    for _ in range(3):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    tf = cfg.flops() / (ms * 1e-3) / 1e12
+    nbytes = 4.0 * q.numel() * 2 + lse.numel() * 4
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": f"{cfg.name}: non-causal B={cfg.B} H={cfg.Hq} S={cfg.Sq} d=64 fp16", "kernel": "fa_fwd_d64_kernel",
+            "ms": round(ms, 4), "tflops": round(tf, 1), "gbs": round(gbs, 1), "algorithmic_bytes": nbytes,
+            "bound": "hbm", "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
+            "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
 
 
 def run_varlen(fa, dev, peaks, small=False, iters=10):

@@ -45,7 +45,7 @@ extern "C" {
 #define FA_OK 0
 #define FA_ERR_NULL (-1)        /* a required pointer is NULL                                 */
 #define FA_ERR_SHAPE (-2)       /* negative dims, Hq % Hkv != 0, bad stride                  */
-#define FA_ERR_UNSUPPORTED (-3) /* d != 128, causal with Sq > Skv, unknown dtype             */
+#define FA_ERR_UNSUPPORTED (-3) /* head dimension, causal with Sq > Skv, unknown dtype        */
 #define FA_ERR_ALIGN (-4)       /* a pointer or stride is not 16-byte aligned                */
 #define FA_ERR_WORKSPACE (-5)   /* workspace missing or too small                            */
 #define FA_ERR_DEVICE (-6)      /* current device is not compute capability 10.x             */
@@ -59,7 +59,9 @@ extern "C" {
 /*
  * Prefill / general forward, fp16 inputs and output (Section 5.1 operator; Section 4.1 method).
  *   q [B,Sq,Hq,d], k,v [B,Skv,Hkv,d], o [B,Sq,Hq,d] fp16, contiguous; lse [B,Hq,Sq] float or NULL.
- *   d must be 128.  B == 0 or Sq == 0 is a successful no-op.  Skv == 0 gives O = 0, LSE = -inf.
+ *   d must be 128, or 64 (the short vision workload of the evaluation section; fa_forward,
+ *   fa_forward_bf16 and fa_forward_ex with variant 0 only; every other entry point wants 128).
+ *   B == 0 or Sq == 0 is a successful no-op.  Skv == 0 gives O = 0, LSE = -inf.
  *   o and lse must not alias the inputs.
  */
 int fa_forward(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,

@@ -13,6 +13,7 @@
 
 #include "decode.cuh"
 #include "prefill_pingpong.cuh"
+#include "prefill_d64.cuh"
 #include "prefill_pipelined.cuh"
 #include "prefill_simple.cuh"
 
@@ -44,16 +45,16 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// Tensor map over a [B, S, H, 128] 16-bit tensor with element strides (sb, ss, sh); a box is
-// box_rows sequence positions x 64 elements of d for one (batch, head), 128-byte swizzled.
+// Tensor map over a [B, S, H, d] 16-bit tensor (d = 128 or 64) with element strides (sb, ss, sh);
+// a box is box_rows sequence positions x 64 elements of d for one (batch, head), 128-byte swizzled.
 int encode_map(CUtensorMap* tm, const void* base, int B, int S, int H, int64_t sb, int64_t ss, int64_t sh,
-               int box_rows, bool bf16) {
+               int box_rows, bool bf16, int d = 128) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return FA_ERR_DEVICE;
-    cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)ss * 2, (cuuint64_t)sb * 2};
     // a dimension of extent 1 never advances; give it a harmless legal stride
-    if (H == 1) strides[0] = 256;
+    if (H == 1) strides[0] = (cuuint64_t)d * 2;
     if (S == 1) strides[1] = strides[0] * (cuuint64_t)H;
     if (B == 1) strides[2] = strides[1] * (cuuint64_t)S;
     cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
@@ -85,22 +86,22 @@ int check_device() {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-void default_strides(int64_t s[3], int S, int H) {
+void default_strides(int64_t s[3], int S, int H, int d = 128) {
     if (s[0] == 0 && s[1] == 0 && s[2] == 0) {
-        s[2] = 128;
-        s[1] = (int64_t)H * 128;
-        s[0] = (int64_t)S * H * 128;
+        s[2] = d;
+        s[1] = (int64_t)H * d;
+        s[0] = (int64_t)S * H * d;
     }
 }
 
-bool strides_ok(const int64_t s[3], int B, int S, int H) {
+bool strides_ok(const int64_t s[3], int B, int S, int H, int d = 128) {
     for (int i = 0; i < 3; ++i) {
         if (s[i] < 0 || (s[i] & 7)) return false;
         if (s[i] >= (1ll << 38)) return false;
     }
-    if (H > 1 && s[2] < 128) return false;
-    if (S > 1 && s[1] < 128) return false;
-    if (B > 1 && s[0] < 128) return false;
+    if (H > 1 && s[2] < d) return false;
+    if (S > 1 && s[1] < d) return false;
+    if (B > 1 && s[0] < d) return false;
     return true;
 }
 
@@ -129,7 +130,8 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     // ---- validation (no CUDA call before it passes)
     if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
     if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
-    if (p.d != 128) return FA_ERR_UNSUPPORTED;
+    if (p.d != 128 && p.d != 64) return FA_ERR_UNSUPPORTED;
+    if (p.d == 64 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // one kernel serves d = 64
     if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
     if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
@@ -138,12 +140,12 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (p.B == 0 || p.Sq == 0) return FA_OK;
     if (!p.q || !p.o) return FA_ERR_NULL;
     if (p.Skv > 0 && (!p.k || !p.v)) return FA_ERR_NULL;
-    default_strides(p.q_stride, p.Sq, p.Hq);
-    default_strides(p.k_stride, p.Skv, p.Hkv);
-    default_strides(p.v_stride, p.Skv, p.Hkv);
-    default_strides(p.o_stride, p.Sq, p.Hq);
-    if (!strides_ok(p.q_stride, p.B, p.Sq, p.Hq) || !strides_ok(p.k_stride, p.B, p.Skv, p.Hkv) ||
-        !strides_ok(p.v_stride, p.B, p.Skv, p.Hkv) || !strides_ok(p.o_stride, p.B, p.Sq, p.Hq))
+    default_strides(p.q_stride, p.Sq, p.Hq, p.d);
+    default_strides(p.k_stride, p.Skv, p.Hkv, p.d);
+    default_strides(p.v_stride, p.Skv, p.Hkv, p.d);
+    default_strides(p.o_stride, p.Sq, p.Hq, p.d);
+    if (!strides_ok(p.q_stride, p.B, p.Sq, p.Hq, p.d) || !strides_ok(p.k_stride, p.B, p.Skv, p.Hkv, p.d) ||
+        !strides_ok(p.v_stride, p.B, p.Skv, p.Hkv, p.d) || !strides_ok(p.o_stride, p.B, p.Sq, p.Hq, p.d))
         return FA_ERR_SHAPE;
     if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.o)) return FA_ERR_ALIGN;
     if (p.lse && (reinterpret_cast<uintptr_t>(p.lse) & 3u)) return FA_ERR_ALIGN;
@@ -173,6 +175,7 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.cu_q = nullptr;
     fp.cu_k = nullptr;
     fp.total_q = 0;
+    fp.d = p.d;
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
     const bool bf16 = p.dtype == FA_DTYPE_BF16;
@@ -187,12 +190,23 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     }
 
     CUtensorMap tq, tk, tv;
-    rc = encode_map(&tq, p.q, p.B, p.Sq, p.Hq, p.q_stride[0], p.q_stride[1], p.q_stride[2], 128, bf16);
+    rc = encode_map(&tq, p.q, p.B, p.Sq, p.Hq, p.q_stride[0], p.q_stride[1], p.q_stride[2], 128, bf16, p.d);
     if (rc) return rc;
-    rc = encode_map(&tk, p.k, p.B, p.Skv, p.Hkv, p.k_stride[0], p.k_stride[1], p.k_stride[2], 128, bf16);
+    rc = encode_map(&tk, p.k, p.B, p.Skv, p.Hkv, p.k_stride[0], p.k_stride[1], p.k_stride[2], 128, bf16, p.d);
     if (rc) return rc;
-    rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16);
+    rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16, p.d);
     if (rc) return rc;
+
+    if (p.d == 64) {  // head dimension 64: one CTA per (batch, head, query tile), two CTAs per SM
+        auto kern = bf16 ? fa::fa_fwd_d64_kernel<__nv_bfloat16> : fa::fa_fwd_d64_kernel<__half>;
+        int sm_count = 0;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64Smem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
+        dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
+        kern<<<grid, 128, fa::kD64Smem, st>>>(tq, tk, tv, fp);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
 
     // Default choice, from timings of both kernels on B200: the ping-pong kernel (one query tile
     // per CTA, Q K^T running ahead of the softmax) wins from 1024 keys on; the paired-tile kernel
@@ -338,6 +352,7 @@ int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, floa
     fp.cu_q = cu_seqlens_q;
     fp.cu_k = cu_seqlens_k;
     fp.total_q = total_q;
+    fp.d = 128;
 
     if (total_k == 0 || max_seqlen_k == 0) {
         // no keys anywhere: O = 0, LSE = -inf over the packed rows, seen as one sequence

@@ -58,6 +58,7 @@ struct FwdParams {
     const int* cu_q;
     const int* cu_k;
     int total_q;
+    int d;  // head dimension: 128, or 64 (its own kernel)
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim
@@ -476,7 +477,7 @@ __global__ void fa_fill_empty_kernel(const FwdParams p) {
         const int i = bi % p.Sq;
         const int b = bi / p.Sq;
         const long long obase = (long long)b * p.o_sb + (long long)i * p.o_ss + (long long)h * p.o_sh;
-        for (int t = 0; t < kTile; ++t) {
+        for (int t = 0; t < p.d; ++t) {
             if (p.o_fp32) static_cast<float*>(p.o)[obase + t] = 0.f;
             else static_cast<T*>(p.o)[obase + t] = T(0.f);
         }

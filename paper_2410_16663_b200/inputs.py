@@ -115,6 +115,8 @@ C3 = {s: PrefillConfig(f"C3-{s // 1024}K", 1, 32, 32, s, s, dtype="bf16", causal
       for i, s in enumerate((8192, 32768, 131072, 262144))}
 C4 = PrefillConfig("C4", 2, 64, 8, 8192, 8192, dtype="bf16", causal=True, seed=1010)
 C4_NC = PrefillConfig("C4-noncausal", 2, 64, 8, 1024, 8192, dtype="bf16", causal=False, seed=1011)
+# the short non-causal vision workload (DeiT-B dimensions: 197 tokens, 12 heads of 64), batch 1024
+DEIT_B = PrefillConfig("DeiT-B", 1024, 12, 12, 197, 197, d=64, dtype="fp16", causal=False, seed=1030)
 C5_MHA = DecodeConfig("C5-mha", 64, 32, 32, 32768, 1024, 32768, seed=1020)
 C5_GQA = DecodeConfig("C5-gqa", 64, 32, 8, 32768, 1024, 32768, seed=1021)
 

@@ -317,6 +317,54 @@ def test_c4_gqa_sampled(fa):
     assert sampled_case(fa, synth.C4_NC, 64) >= 256
 
 
+# ------------------------------------------------------------------ head dimension 64
+def full_case_d64(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed):
+    cfg = synth.PrefillConfig("t", B, Hq, Hkv, Sq, Skv, d=64, dtype=dtype, causal=causal, seed=seed)
+    q, k, v = synth.prefill_inputs(cfg, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, causal, cfg.scale)
+    absv = oracle.attention_full(q, k, v.abs(), causal, cfg.scale)[0] if dtype == "bf16" else None
+    what = f"d64 B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {dtype}"
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=what)
+    if dtype == "bf16":
+        o32, lse32 = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale, o_dtype=torch.float32)
+        assert_close_to_oracle(o32, lse32, o_ref, l_ref, p_absv=absv, what=what + " fp32-out")
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", [(1, 1), (127, 127), (128, 128), (129, 129), (197, 197), (256, 256), (257, 257),
+                                    (1, 129), (17, 1000), (100, 257), (300, 700)])
+def test_d64_shape_grid(fa, sq, skv, causal):
+    full_case_d64(fa, 2, 3, 3, sq, skv, causal, "fp16", seed=sq * 1000 + skv + 11)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_d64_gqa_and_both_types(fa, dtype):
+    full_case_d64(fa, 2, 8, 2, 333, 333, True, dtype, seed=71)
+    full_case_d64(fa, 1, 12, 12, 197, 197, False, dtype, seed=72)       # the vision shape, one image
+    full_case_d64(fa, 1, 4, 1, 130, 1500, False, dtype, seed=73)        # many kv tiles through the two-slot ring
+
+
+def test_d64_vision_batch_full_size_sampled(fa):
+    # the benchmark's batch of 1024 images: sampled rows against the oracle, everything finite
+    cfg = synth.DEIT_B
+    q, k, v = synth.prefill_inputs(cfg, DEV)
+    o, lse = run_forward(fa, q, k, v, cfg.causal, cfg.scale)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    rows = synth.sample_rows(cfg, 6, seed=5, pairs=[(0, 0), (0, 11), (511, 5), (1023, 0), (1023, 11)])
+    o_ref, l_ref = oracle_rows_for(q, k, v, rows, cfg.causal, cfg.scale)
+    idx = torch.tensor(rows)
+    o_s = o[idx[:, 0], idx[:, 2], idx[:, 1]].view(1, len(rows), 1, cfg.d)
+    l_s = lse[idx[:, 0], idx[:, 1], idx[:, 2]].view(1, 1, len(rows))
+    assert_close_to_oracle(o_s, l_s, o_ref.view(1, len(rows), 1, cfg.d), l_ref.view(1, 1, len(rows)), what="DeiT-B batch")
+
+
+def test_d64_is_refused_where_it_is_not_built(fa):
+    q = torch.zeros(1, 4, 2, 64, dtype=torch.float16, device=DEV)
+    o = torch.empty_like(q); lse = torch.empty(1, 2, 4, device=DEV)
+    assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=3, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------------ packed variable-length batches
 def varlen_case(fa, cfg, what):
     q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
