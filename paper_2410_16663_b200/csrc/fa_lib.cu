@@ -197,6 +197,17 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16, p.d);
     if (rc) return rc;
 
+    if (p.d == 64 && p.Skv > 128 && p.Skv <= 256) {
+        // short sequences: all keys are one 256-wide tile, one CTA per (batch, head, two query tiles)
+        auto kern = bf16 ? fa::fa_fwd_d64_short_kernel<__nv_bfloat16> : fa::fa_fwd_d64_short_kernel<__half>;
+        int sm_count = 0;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64ShortSmem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
+        dim3 grid((fp.n_qtiles + 1) / 2, fp.Hq, fp.B);
+        kern<<<grid, 128, fa::kD64ShortSmem, st>>>(tq, tk, tv, fp);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
     if (p.d == 64) {  // head dimension 64: one CTA per (batch, head, query tile), two CTAs per SM
         auto kern = bf16 ? fa::fa_fwd_d64_kernel<__nv_bfloat16> : fa::fa_fwd_d64_kernel<__half>;
         int sm_count = 0;

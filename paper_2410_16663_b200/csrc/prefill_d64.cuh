@@ -242,3 +242,217 @@ fa_fwd_d64_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 }
 
 }  // namespace fa
+
+namespace fa {
+
+// ---------------------------------------------------------------------------------------
+// Short sequences (128 < Skv <= 256, d = 64): the whole key range is one 256-wide tile, so the
+// softmax needs no running state.  One CTA per (batch, head, pair of query tiles): K and V are
+// loaded once for both query tiles; per query tile one N = 256 score MMA into tensor-memory
+// columns [0,256), a first pass over the row for its max, a second pass that writes
+// P = exp(S - max) packed over columns [0,128) (a chunk's P lands in columns the thread has
+// already read), then O = P V into columns [128,192), which the scores no longer need.
+// Chunks of 32 columns that lie entirely past the keys are skipped (their P is written as 0).
+// Two CTAs per SM (97 KiB of shared memory, 256 tensor-memory columns each).
+constexpr int kD64ShortSmem = 1024 + 6 * kD64TileBytes;
+
+template <typename T>
+__global__ void __launch_bounds__(128, 2)
+fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base;                  // 2 query tiles
+    const uint32_t sK = sQ + 2 * kD64TileBytes;     // keys 0..255: two boxes back to back
+    const uint32_t sV = sK + 2 * kD64TileBytes;
+    __shared__ __align__(8) uint64_t bars[8];
+    __shared__ uint32_t tmem_holder;
+    __shared__ volatile uint32_t abort_flag;
+
+    const uint32_t bar_q0 = smem_u32(&bars[0]);  // +8 for the second query tile
+    const uint32_t bar_k = smem_u32(&bars[2]);
+    const uint32_t bar_v = smem_u32(&bars[3]);
+    const uint32_t bar_s = smem_u32(&bars[4]);
+    const uint32_t bar_o = smem_u32(&bars[5]);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int h = blockIdx.y;
+    const int b = blockIdx.z;
+    const int hk = h / (p.Hq / p.Hkv);
+    const int qt0 = blockIdx.x * 2;                       // first query tile of this CTA
+    const int nq = min(2, p.n_qtiles - qt0);              // its query tiles
+    const int off = p.Skv - p.Sq;
+
+    if (tid == 0) {
+        for (int i = 0; i < 6; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&tmem_holder), 256);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t tS = tmem_base + lane_sel;        // columns [0,256): S; P packed in [0,128)
+    const uint32_t tO = tmem_base + lane_sel + 128;  // columns [128,192): O, once P is written
+
+    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    constexpr uint32_t idesc_qk = instr_desc_f16(kBf16, 128, 256, false, false);
+    constexpr uint32_t idesc_pv = instr_desc_f16(kBf16, 128, 64, false, true);
+
+    if (tid == 0) {
+        mbar_expect_tx(bar_q0, kD64TileBytes);
+        tma_load_4d(sQ, &tm_q, bar_q0, 0, h, qt0 * kTile, b);
+        mbar_expect_tx(bar_k, 2 * kD64TileBytes);   // rows past the keys arrive as zeros
+        tma_load_4d(sK, &tm_k, bar_k, 0, hk, 0, b);
+        tma_load_4d(sK + kD64TileBytes, &tm_k, bar_k, 0, hk, kTile, b);
+        if (nq > 1) {
+            mbar_expect_tx(bar_q0 + 8, kD64TileBytes);
+            tma_load_4d(sQ + kD64TileBytes, &tm_q, bar_q0 + 8, 0, h, (qt0 + 1) * kTile, b);
+        }
+        mbar_expect_tx(bar_v, 2 * kD64TileBytes);
+        tma_load_4d(sV, &tm_v, bar_v, 0, hk, 0, b);
+        tma_load_4d(sV + kD64TileBytes, &tm_v, bar_v, 0, hk, kTile, b);
+    }
+    __syncwarp();
+
+    const int n_chunks = (p.Skv + 31) / 32;   // chunks of 32 columns that hold keys (5..8)
+    bool ok = true;
+    for (int t = 0; t < nq && ok; ++t) {
+        const int q0 = (qt0 + t) * kTile;
+        const int row = q0 + tid;
+        // ---- S = Q K^T over all keys
+        if (tid == 0) {
+            ok = mbar_wait(bar_q0 + 8 * t, 0, &abort_flag, 51);
+            if (t == 0) ok = ok && mbar_wait(bar_k, 0, &abort_flag, 52);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ss(tmem_base, smem_desc_sw128(sQ + t * kD64TileBytes + ks * 32, 16, 1024),
+                           smem_desc_sw128(sK + ks * 32, 16, 1024), idesc_qk, ks > 0);
+                mma_commit(bar_s);
+            }
+        }
+        __syncwarp();
+        if (!mbar_wait(bar_s, t & 1, &abort_flag, 53)) { ok = false; break; }
+        tc_fence_after();
+
+        // columns >= lim are past the keys or above the diagonal; a row past the end of the
+        // queries (the ragged last tile) keeps nothing, which spares its exponentials
+        int lim = p.Skv;
+        if (p.causal) lim = min(lim, row + off + 1);
+        if (row >= p.Sq) lim = 0;
+        // ---- pass 1: row max
+        float m = -INFINITY;
+        // (a warp stops at the last chunk any of its rows can see)
+        const int my_chunks = min(n_chunks, (__reduce_max_sync(0xffffffffu, max(lim, 0)) + 31) / 32);
+        for (int c = 0; c < my_chunks; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tS + c * 32, r);
+            tmem_wait_ld();
+            const int live = lim - c * 32;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < live) m = fmaxf(m, __uint_as_float(r[i]));
+        }
+        const float m_use = (m == -INFINITY) ? 0.f : m;   // a row that sees nothing stays finite
+        const float neg_ms = -m_use * p.scale_log2;
+        // ---- pass 2: P = exp2(S * scale_log2 - max * scale_log2), row sum
+        float l = 0.f;
+        for (int c = 0; c < 8; ++c) {
+            uint32_t pk[16];
+            if (c < my_chunks) {
+                uint32_t r[32];
+                tmem_ld_x32(tS + c * 32, r);
+                tmem_wait_ld();
+                const int live = lim - c * 32;
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float e0 = (i < live) ? fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_ms)) : 0.f;
+                    const float e1 = (i + 1 < live) ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_ms)) : 0.f;
+                    l += e0 + e1;
+                    pk[i >> 1] = pack2<T>(e0, e1);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pk[i] = 0u;
+            }
+            tmem_st_x16(tS + c * 16, pk);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncthreads();
+        // ---- O = P V
+        if (tid == 0) {
+            if (t == 0) ok = mbar_wait(bar_v, 0, &abort_flag, 54);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 16; ++ks)  // 16 keys per step: 2048 bytes down the two V boxes
+                    mma_ts(tmem_base + 128, tmem_base + ks * 8, smem_desc_sw128(sV + ks * 2048, 16, 1024), idesc_pv,
+                           ks > 0);
+                mma_commit(bar_o);
+            }
+        }
+        __syncwarp();
+        if (!mbar_wait(bar_o, t & 1, &abort_flag, 55)) { ok = false; break; }
+        tc_fence_after();
+        // ---- epilogue: O / l, LSE = max * scale + ln l
+        const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+        const bool live_row = row < p.Sq;
+        const long long obase = (long long)b * p.o_sb + (long long)row * p.o_ss + (long long)h * p.o_sh;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tmem_ld_x32(tO + c * 32, r);
+            tmem_wait_ld();
+            if (live_row) {
+                if (p.o_fp32) {
+                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
+                                             __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
+                } else {
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.o) + obase + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 w;
+                        w.x = pack2<T>(__uint_as_float(r[8 * i]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
+                        w.y = pack2<T>(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
+                        w.z = pack2<T>(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
+                        w.w = pack2<T>(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                        dst[i] = w;
+                    }
+                }
+            }
+        }
+        if (live_row && p.lse != nullptr) {
+            const float lse = (l > 0.f) ? (m * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            p.lse[((long long)b * p.Hq + h) * p.Sq + row] = lse;
+        }
+        // the next query tile's scores overwrite the columns O was read from
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
+}  // namespace fa
