@@ -361,14 +361,27 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
             tmem_ld_x32(tS + c * 32, r);
             tmem_wait_ld();
             const int live = lim - c * 32;
+            if (__all_sync(0xffffffffu, live >= 32)) {
+                // every row of the warp sees the whole chunk: no selects
+                float m0 = m, m1 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (i < live) m = fmaxf(m, __uint_as_float(r[i]));
+                for (int i = 0; i < 32; i += 4) {
+                    m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                    m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                }
+                m = fmaxf(m0, m1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < live) m = fmaxf(m, __uint_as_float(r[i]));
+            }
         }
         const float m_use = (m == -INFINITY) ? 0.f : m;   // a row that sees nothing stays finite
         const float neg_ms = -m_use * p.scale_log2;
         // ---- pass 2: P = exp2(S * scale_log2 - max * scale_log2), row sum
         float l = 0.f;
+        const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
+        uint64_t l2 = f2_pack(0.f, 0.f);
         for (int c = 0; c < 8; ++c) {
             uint32_t pk[16];
             if (c < my_chunks) {
@@ -376,18 +389,34 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                 tmem_ld_x32(tS + c * 32, r);
                 tmem_wait_ld();
                 const int live = lim - c * 32;
+                if (__all_sync(0xffffffffu, live >= 32)) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float e0 = (i < live) ? fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_ms)) : 0.f;
-                    const float e1 = (i + 1 < live) ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_ms)) : 0.f;
-                    l += e0 + e1;
-                    pk[i >> 1] = pack2<T>(e0, e1);
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0, x1;
+                        f2_unpack(f2_fma(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2), x0, x1);
+                        const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
+                        l2 = f2_add(l2, f2_pack(e0, e1));
+                        pk[i >> 1] = pack2<T>(e0, e1);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float e0 = (i < live) ? fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_ms)) : 0.f;
+                        const float e1 = (i + 1 < live) ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_ms)) : 0.f;
+                        l += e0 + e1;
+                        pk[i >> 1] = pack2<T>(e0, e1);
+                    }
                 }
             } else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) pk[i] = 0u;
             }
             tmem_st_x16(tS + c * 16, pk);
+        }
+        {
+            float la, lb;
+            f2_unpack(l2, la, lb);
+            l += la + lb;
         }
         tmem_wait_st();
         tc_fence_before();

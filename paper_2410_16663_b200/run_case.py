@@ -24,6 +24,7 @@ def main():
     ap.add_argument("--S", type=int, default=8192)
     ap.add_argument("--Skv", type=int, default=0)
     ap.add_argument("--Smax", type=int, default=16384)
+    ap.add_argument("--d", type=int, default=128, choices=[64, 128], help="head dimension (prefill only)")
     ap.add_argument("--dtype", default="fp16", choices=["fp16", "bf16"])
     ap.add_argument("--noncausal", action="store_true")
     ap.add_argument("--variant", type=int, default=0)
@@ -33,7 +34,7 @@ def main():
     hkv = a.Hkv or a.H
     dev = "cuda"
     if a.kind == "prefill":
-        cfg = synth.PrefillConfig("case", a.B, a.H, hkv, a.S, a.Skv or a.S, dtype=a.dtype,
+        cfg = synth.PrefillConfig("case", a.B, a.H, hkv, a.S, a.Skv or a.S, d=a.d, dtype=a.dtype,
                                   causal=not a.noncausal, seed=7)
         q, k, v = synth.prefill_inputs(cfg, dev)
         o = torch.empty_like(q)
