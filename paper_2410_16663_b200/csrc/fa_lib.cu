@@ -131,7 +131,7 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
     if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
     if (p.d != 128 && p.d != 64) return FA_ERR_UNSUPPORTED;
-    if (p.d == 64 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // one kernel serves d = 64
+    if (p.d == 64 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // the shape picks the d = 64 kernel
     if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
     if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;

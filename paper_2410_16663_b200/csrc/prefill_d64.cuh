@@ -256,6 +256,110 @@ namespace fa {
 // Two CTAs per SM (97 KiB of shared memory, 256 tensor-memory columns each).
 constexpr int kD64ShortSmem = 1024 + 6 * kD64TileBytes;
 
+// One query row against up to 256 keys whose raw scores sit in tensor-memory columns [0,256) at
+// tS (this thread's lane): row max m (raw units), row sum l of P = exp2((S - m) * scale_log2),
+// and P written packed over columns [0,128).  Columns >= lim are hidden; n_chunks = chunks of 32
+// columns that hold keys.  Warp-collective (tensor-memory loads and stores).
+template <typename T>
+__device__ __forceinline__ void d64_row_softmax(uint32_t tS, int lim, int n_chunks, float scale_log2, float& m,
+                                                float& l) {
+    // ---- pass 1: row max
+    m = -INFINITY;
+    // (a warp stops at the last chunk any of its rows can see)
+    const int my_chunks = min(n_chunks, (__reduce_max_sync(0xffffffffu, max(lim, 0)) + 31) / 32);
+    for (int c = 0; c < my_chunks; ++c) {
+        uint32_t r[32];
+        tmem_ld_x32(tS + c * 32, r);
+        tmem_wait_ld();
+        const int live = lim - c * 32;
+        if (__all_sync(0xffffffffu, live >= 32)) {
+            // every row of the warp sees the whole chunk: no selects
+            float m0 = m, m1 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            }
+            m = fmaxf(m0, m1);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < live) m = fmaxf(m, __uint_as_float(r[i]));
+        }
+    }
+    const float m_use = (m == -INFINITY) ? 0.f : m;   // a row that sees nothing stays finite
+    const float neg_ms = -m_use * scale_log2;
+    // ---- pass 2: P = exp2(S * scale_log2 - max * scale_log2), row sum
+    l = 0.f;
+    const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
+    uint64_t l2 = f2_pack(0.f, 0.f);
+    for (int c = 0; c < 8; ++c) {
+        uint32_t pk[16];
+        if (c < my_chunks) {
+            uint32_t r[32];
+            tmem_ld_x32(tS + c * 32, r);
+            tmem_wait_ld();
+            const int live = lim - c * 32;
+            if (__all_sync(0xffffffffu, live >= 32)) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float x0, x1;
+                    f2_unpack(f2_fma(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2), x0, x1);
+                    const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
+                    l2 = f2_add(l2, f2_pack(e0, e1));
+                    pk[i >> 1] = pack2<T>(e0, e1);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float e0 = (i < live) ? fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, neg_ms)) : 0.f;
+                    const float e1 = (i + 1 < live) ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_ms)) : 0.f;
+                    l += e0 + e1;
+                    pk[i >> 1] = pack2<T>(e0, e1);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+        }
+        tmem_st_x16(tS + c * 16, pk);
+    }
+    {
+        float la, lb;
+        f2_unpack(l2, la, lb);
+        l += la + lb;
+    }
+}
+
+// This thread's row of O (64 fp32 columns in r0, r1) scaled by inv_l and stored.
+template <typename T>
+__device__ __forceinline__ void d64_store_row(const FwdParams& p, long long obase, const uint32_t (&r0)[32],
+                                              const uint32_t (&r1)[32], float inv_l) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const uint32_t(&r)[32] = c ? r1 : r0;
+        if (p.o_fp32) {
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
+                                     __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
+        } else {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.o) + obase + c * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 w;
+                w.x = pack2<T>(__uint_as_float(r[8 * i]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
+                w.y = pack2<T>(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
+                w.z = pack2<T>(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
+                w.w = pack2<T>(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                dst[i] = w;
+            }
+        }
+    }
+}
+
+
 template <typename T>
 __global__ void __launch_bounds__(128, 2)
 fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -352,72 +456,8 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         int lim = p.Skv;
         if (p.causal) lim = min(lim, row + off + 1);
         if (row >= p.Sq) lim = 0;
-        // ---- pass 1: row max
-        float m = -INFINITY;
-        // (a warp stops at the last chunk any of its rows can see)
-        const int my_chunks = min(n_chunks, (__reduce_max_sync(0xffffffffu, max(lim, 0)) + 31) / 32);
-        for (int c = 0; c < my_chunks; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32(tS + c * 32, r);
-            tmem_wait_ld();
-            const int live = lim - c * 32;
-            if (__all_sync(0xffffffffu, live >= 32)) {
-                // every row of the warp sees the whole chunk: no selects
-                float m0 = m, m1 = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                }
-                m = fmaxf(m0, m1);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (i < live) m = fmaxf(m, __uint_as_float(r[i]));
-            }
-        }
-        const float m_use = (m == -INFINITY) ? 0.f : m;   // a row that sees nothing stays finite
-        const float neg_ms = -m_use * p.scale_log2;
-        // ---- pass 2: P = exp2(S * scale_log2 - max * scale_log2), row sum
-        float l = 0.f;
-        const uint64_t sc2 = f2_pack(p.scale_log2, p.scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
-        uint64_t l2 = f2_pack(0.f, 0.f);
-        for (int c = 0; c < 8; ++c) {
-            uint32_t pk[16];
-            if (c < my_chunks) {
-                uint32_t r[32];
-                tmem_ld_x32(tS + c * 32, r);
-                tmem_wait_ld();
-                const int live = lim - c * 32;
-                if (__all_sync(0xffffffffu, live >= 32)) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float x0, x1;
-                        f2_unpack(f2_fma(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2), x0, x1);
-                        const float e0 = fast_exp2(x0), e1 = fast_exp2(x1);
-                        l2 = f2_add(l2, f2_pack(e0, e1));
-                        pk[i >> 1] = pack2<T>(e0, e1);
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float e0 = (i < live) ? fast_exp2(fmaf(__uint_as_float(r[i]), p.scale_log2, neg_ms)) : 0.f;
-                        const float e1 = (i + 1 < live) ? fast_exp2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, neg_ms)) : 0.f;
-                        l += e0 + e1;
-                        pk[i >> 1] = pack2<T>(e0, e1);
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) pk[i] = 0u;
-            }
-            tmem_st_x16(tS + c * 16, pk);
-        }
-        {
-            float la, lb;
-            f2_unpack(l2, la, lb);
-            l += la + lb;
-        }
+        float m, l;
+        d64_row_softmax<T>(tS, lim, n_chunks, p.scale_log2, m, l);
         tmem_wait_st();
         tc_fence_before();
         __syncthreads();

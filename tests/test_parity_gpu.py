@@ -318,16 +318,17 @@ def test_c4_gqa_sampled(fa):
 
 
 # ------------------------------------------------------------------ head dimension 64
-def full_case_d64(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed):
+def full_case_d64(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed, variant=0):
     cfg = synth.PrefillConfig("t", B, Hq, Hkv, Sq, Skv, d=64, dtype=dtype, causal=causal, seed=seed)
     q, k, v = synth.prefill_inputs(cfg, "cpu")
     o_ref, l_ref = oracle.attention_full(q, k, v, causal, cfg.scale)
     absv = oracle.attention_full(q, k, v.abs(), causal, cfg.scale)[0] if dtype == "bf16" else None
-    what = f"d64 B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {dtype}"
-    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale)
+    what = f"d64 B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {dtype} variant{variant}"
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale, variant=variant)
     assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=what)
     if dtype == "bf16":
-        o32, lse32 = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale, o_dtype=torch.float32)
+        o32, lse32 = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale, o_dtype=torch.float32,
+                                 variant=variant)
         assert_close_to_oracle(o32, lse32, o_ref, l_ref, p_absv=absv, what=what + " fp32-out")
 
 
@@ -336,6 +337,16 @@ def full_case_d64(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed):
                                     (1, 129), (17, 1000), (100, 257), (300, 700)])
 def test_d64_shape_grid(fa, sq, skv, causal):
     full_case_d64(fa, 2, 3, 3, sq, skv, causal, "fp16", seed=sq * 1000 + skv + 11)
+
+
+def test_d64_short_sequence_kernel(fa):
+    # 128 < Skv <= 256: all keys as one 256-wide tile.  More CTAs than fit at once, with one or
+    # two query tiles each, many query tiles over few keys, causal with fewer queries than keys
+    full_case_d64(fa, 30, 12, 12, 197, 197, False, "fp16", seed=81)
+    full_case_d64(fa, 40, 6, 2, 100, 130, False, "bf16", seed=82)
+    full_case_d64(fa, 3, 4, 4, 700, 256, False, "fp16", seed=83)
+    full_case_d64(fa, 5, 8, 8, 150, 255, True, "fp16", seed=84)
+    full_case_d64(fa, 2, 2, 1, 256, 256, True, "bf16", seed=85)
 
 
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
