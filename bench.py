@@ -274,6 +274,7 @@ def run_product(args, rank, world, local_rank):
         if not args.small:
             out["prefill_long_context"] = run_long_context(fa, dev, peaks)
         out["decode_paged"] = run_decode_paged(fa, dec[0], dev, peaks)
+        out["decode_fp8"] = run_decode_fp8(fa, dec[0], dev, peaks)
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
@@ -371,6 +372,32 @@ def run_varlen(fa, dev, peaks, small=False, iters=10):
                         f"(sum {int(q.shape[0])}), Hq=Hkv={cfg.Hq}, bf16, packed", "ms": round(ms, 4),
             "tflops": round(tf, 1), "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4),
             "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4)}
+
+
+def run_decode_fp8(fa, d, dev, peaks, iters=5):
+    """The first decode configuration once more with its cache stored as FP8 e4m3 (fa_decode_fp8),
+    outside the timed steps: the same keys in half the bytes.  `gbs` counts the 8-bit cache
+    bytes actually read; `fp16_equivalent_gbs` is the rate the fp16 cache would need for the same time."""
+    cfg = d["cfg"]
+    k8, v8 = synth.fp8_cache(d["k"], d["v"], d["sl_host"], 0.25, 0.125, poison=True)
+    for _ in range(3):
+        fa.fa_decode_fp8(d["q"], k8, v8, d["o"], d["lse"], d["sl"], cfg.scale, 0.25, 0.125, d["ws"])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_decode_fp8(d["q"], k8, v8, d["o"], d["lse"], d["sl"], cfg.scale, 0.25, 0.125, d["ws"])
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    nbytes = d["bytes"] / 2
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": f"{cfg.name} with the cache as FP8 e4m3 (one factor per tensor)", "ms": round(ms, 4),
+            "gbs": round(gbs, 1), "kv_bytes": nbytes, "fp16_equivalent_gbs": round(2 * gbs, 1),
+            "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4), "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
 
 
 def run_decode_paged(fa, d, dev, peaks, page_size=256, iters=5):

@@ -142,6 +142,22 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * Decode over an 8-bit cache (Appendix D.2 evaluates the operator with 8-bit operands; in the
+ * decode stage the cache dominates the traffic, so here it is the cached K and V that are 8-bit):
+ * the computation of fa_decode with K = k_scale * k_cache and V = v_scale * v_cache, where
+ * k_cache and v_cache [B,Skv_max,Hkv,d] hold FP8 e4m3 bit patterns (1 sign, 4 exponent, 3
+ * mantissa bits, bias 7, no infinities; one byte per element, contiguous, 16-byte aligned) and
+ * k_scale, v_scale are positive finite factors for the whole tensor.  q and o are fp16 and the
+ * probabilities are rounded to fp16 as in fa_decode; the widened cache values are exact in fp16.
+ * Rows beyond seqlens_k[b] may hold anything (the NaN patterns 0x7f / 0xff too).
+ * Everything else (lse, seqlens_k, workspace size and alignment, errors) as for fa_decode;
+ * FA_ERR_UNSUPPORTED also for a scale that is not positive and finite.
+ */
+int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                  const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
+                  float k_scale, float v_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Decode over a paged cache: the same computation as fa_decode (Appendix C), with the cached
  * keys and values of a sequence scattered over fixed-size pages of a pool shared by all
  * sequences, as serving systems keep them for batched decoding (the batch 8/16 serving runs of

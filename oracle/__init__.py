@@ -191,6 +191,37 @@ def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
     return O, LSE
 
 
+def e4m3_to_float64(bits):
+    """Value of FP8 e4m3 bit patterns (1 sign, 4 exponent, 3 mantissa bits, exponent bias 7, no
+    infinities; exponent 15 with mantissa 7 is NaN), written out from the format's definition.
+    ``bits``: uint8 tensor.  Returns float64 of the same shape."""
+    b = torch.as_tensor(bits).to(torch.int64)
+    sign = torch.where((b >> 7) & 1 == 1, -1.0, 1.0).to(torch.float64)
+    e = (b >> 3) & 0xF
+    mnt = (b & 0x7).to(torch.float64)
+    normal = torch.pow(torch.tensor(2.0, dtype=torch.float64), (e - 7).to(torch.float64)) * (1.0 + mnt / 8.0)
+    subnormal = (2.0 ** -6) * (mnt / 8.0)
+    val = sign * torch.where(e == 0, subnormal, normal)
+    nan = (e == 15) & ((b & 0x7) == 7)
+    return torch.where(nan, torch.full_like(val, float("nan")), val)
+
+
+def decode_fp8(q, k_bits, v_bits, seqlens, scale: float, k_scale: float, v_scale: float, nthreads: int = 0):
+    """Decode-stage attention over an FP8 e4m3 cache: ``decode`` on K = k_scale * value(k_bits),
+    V = v_scale * value(v_bits), evaluated in float64 (Appendix D.2 runs the operator on 8-bit
+    operands; the widening itself is exact).  ``k_bits``/``v_bits``: uint8 ``[B,Smax,Hkv,d]``.
+    Rows at or beyond ``seqlens[b]`` are replaced by zeros first (they may hold NaN patterns and
+    are never used)."""
+    q = torch.as_tensor(q).to(torch.float64)
+    k = e4m3_to_float64(k_bits) * float(k_scale)
+    v = e4m3_to_float64(v_bits) * float(v_scale)
+    sl = np.asarray(seqlens, dtype=np.int64).reshape(-1)
+    for b in range(k.shape[0]):
+        k[b, int(sl[b]):] = 0.0
+        v[b, int(sl[b]):] = 0.0
+    return decode(q, k.contiguous(), v.contiguous(), sl.astype(np.int32), scale, nthreads)
+
+
 def decode_paged(q, k_pages, v_pages, block_table, seqlens, scale: float, nthreads: int = 0):
     """Decode-stage attention over a paged cache (the decode computation of Appendix C; only
     the addressing differs): key j of sequence b is row ``j % page_size`` of page

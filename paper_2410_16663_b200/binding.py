@@ -47,6 +47,8 @@ lib.fa_decode_workspace_bytes.restype = _sz
 lib.fa_decode_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
 lib.fa_forward_varlen.restype = _i
 lib.fa_forward_varlen.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p]
+lib.fa_decode_fp8.restype = _i
+lib.fa_decode_fp8.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
 lib.fa_decode_paged.restype = _i
 lib.fa_decode_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_noalloc.restype = _i
@@ -65,7 +67,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -160,6 +162,18 @@ def fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace,
     rc = lib.fa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq,
                        Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode", raise_on_error)
+
+
+def fa_decode_fp8(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, k_scale: float, v_scale: float, workspace,
+                  raise_on_error: bool = True) -> int:
+    """``fa_decode_fp8``: q [B,1,Hq,d] fp16, caches [B,Smax,Hkv,d] of FP8 e4m3 (``torch.float8_e4m3fn`` or
+    uint8 bit patterns) with one factor each, seqlens_k int32 [B] on the device."""
+    B, _, Hq, d = q.shape
+    _, Smax, Hkv, _ = k_cache.shape
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_fp8(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq, Hkv,
+                           Smax, d, float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
+    return _check(rc, "fa_decode_fp8", raise_on_error)
 
 
 def fa_decode_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, workspace,

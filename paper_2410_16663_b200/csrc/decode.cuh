@@ -29,6 +29,7 @@ struct DecodeParams {
     // [pages, page_size, Hkv, 128] and page_size is a multiple of kDecTile
     const int* block_table;
     int page_size, table_stride;
+    float v_scale;        // 8-bit cache only: factor of the stored values
 };
 
 

@@ -14,6 +14,7 @@
 #include "decode.cuh"
 #include "prefill_pingpong.cuh"
 #include "prefill_d64.cuh"
+#include "decode_fp8.cuh"
 #include "prefill_pipelined.cuh"
 #include "prefill_simple.cuh"
 
@@ -62,6 +63,25 @@ int encode_map(CUtensorMap* tm, const void* base, int B, int S, int H, int64_t s
     CUresult r = fn(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        t_last_cuda_error = static_cast<int>(r);
+        return FA_ERR_CUDA;
+    }
+    return FA_OK;
+}
+
+// Tensor map over a [B, S, H, 128] one-byte tensor, contiguous: a box is box_rows sequence
+// positions x 128 bytes for one (batch, head), 128-byte swizzled.
+int encode_map_u8(CUtensorMap* tm, const void* base, int B, int S, int H, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return FA_ERR_DEVICE;
+    cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)S, (cuuint64_t)B};
+    cuuint64_t strides[3] = {128, (cuuint64_t)H * 128, (cuuint64_t)S * H * 128};
+    cuuint32_t box[4] = {128, 1, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         t_last_cuda_error = static_cast<int>(r);
@@ -433,6 +453,7 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.block_table = block_table;
     dp.page_size = block_table ? page_size : 1;
     dp.table_stride = table_stride;
+    dp.v_scale = 1.f;
     const int g = Hq / Hkv;
 
     if (Skv_max > 0) {
@@ -469,6 +490,61 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
               void* stream) {
     return decode_impl(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, workspace,
                        workspace_bytes, stream, nullptr, 0, 0, 0);
+}
+
+int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+                  int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale, float v_scale,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
+    if (!(k_scale > 0.f) || isinf(k_scale) || !(v_scale > 0.f) || isinf(v_scale)) return FA_ERR_UNSUPPORTED;
+    if (B > 65535 || Hq > 65535) return FA_ERR_UNSUPPORTED;
+    if (B == 0) return FA_OK;
+    if (!q || !o || !seqlens_k) return FA_ERR_NULL;
+    if (Skv_max > 0 && (!k_cache || !v_cache)) return FA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(workspace))
+        return FA_ERR_ALIGN;
+    const size_t need = fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return FA_ERR_WORKSPACE;
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    fa::DecodeParams dp;
+    dp.q = q;
+    dp.seqlens = seqlens_k;
+    dp.B = B; dp.Hq = Hq; dp.Hkv = Hkv; dp.Smax = Skv_max;
+    dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max) : 256;
+    dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
+    dp.o_part = static_cast<float*>(workspace);
+    dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
+    dp.scale_log2 = scale * k_scale * 1.4426950408889634f;   // the scores are q . (k_scale * k8)
+    dp.block_table = nullptr;
+    dp.page_size = 1;
+    dp.table_stride = 0;
+    dp.v_scale = v_scale;
+    const int g = Hq / Hkv;
+    if (Skv_max > 0) {
+        CUtensorMap tk, tv;
+        rc = encode_map_u8(&tk, k_cache, B, Skv_max, Hkv, fa::kDecTile);
+        if (rc) return rc;
+        rc = encode_map_u8(&tv, v_cache, B, Skv_max, Hkv, fa::kDecTile);
+        if (rc) return rc;
+        constexpr int smem = 1024 + 2 * fa::kDec8Stages * fa::kDec8TileBytes;
+        int sm_count = 0;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(fa::fa_decode_split_fp8_kernel), smem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
+        dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
+        fa::fa_decode_split_fp8_kernel<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
+        cudaError_t e = cudaGetLastError();
+        rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
+        if (rc) return rc;
+    }
+    fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
 int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,

@@ -194,6 +194,21 @@ def decode_inputs(cfg: DecodeConfig, device="cpu", poison: bool = True):
     return q, k, v, seqlens
 
 
+def fp8_cache(k, v, seqlens, k_scale: float, v_scale: float, poison: bool = True):
+    """The caches of ``decode_inputs`` as FP8 e4m3 bit patterns (uint8) for given factors: each
+    value divided by its factor and rounded to e4m3 by torch's conversion.  Rows at or beyond a
+    sequence's length hold the NaN pattern 0x7f when ``poison`` is set.  (An input generator: the
+    8-bit cache is what the decode stage is handed.)"""
+    k8 = (k.float() / k_scale).to(torch.float8_e4m3fn).view(torch.uint8)
+    v8 = (v.float() / v_scale).to(torch.float8_e4m3fn).view(torch.uint8)
+    for b in range(k.shape[0]):
+        n = int(seqlens[b])
+        if n < k.shape[1]:
+            k8[b, n:] = 0x7f if poison else 0
+            v8[b, n:] = 0x7f if poison else 0
+    return k8, v8
+
+
 def paged_cache(k, v, seqlens, page_size: int, seed: int, spare_pages: int = 3, poison: bool = True):
     """The caches of ``decode_inputs`` laid out in pages: returns ``(k_pages, v_pages, block_table)``.
 

@@ -130,6 +130,27 @@ def test_varlen_validation(fa):
     assert call(max_q=0) == fa.FA_OK
 
 
+def test_fp8_decode_validation(fa):
+    L = fa.lib
+    q, o = _t(2, 1, 8, 128), _t(2, 1, 8, 128)
+    kc = torch.zeros(2, 256, 2, 128, dtype=torch.uint8)
+    sl = torch.zeros(2, dtype=torch.int32)
+    ws = torch.zeros(1 << 16, dtype=torch.uint8)
+    P = lambda t: t.data_ptr()
+    need = fa.fa_decode_workspace_bytes(2, 8, 2, 256, 128)
+    call = lambda **kw: L.fa_decode_fp8(P(q), P(kc), P(kc), P(o), None, kw.get("sl", P(sl)), kw.get("B", 2), 8,
+                                        kw.get("Hkv", 2), 256, kw.get("d", 128), 0.1, kw.get("ks", 1.0), kw.get("vs", 1.0),
+                                        P(ws), kw.get("wbytes", need), None)
+    assert call(Hkv=3) == fa.FA_ERR_SHAPE
+    assert call(d=64) == fa.FA_ERR_UNSUPPORTED
+    assert call(ks=0.0) == fa.FA_ERR_UNSUPPORTED
+    assert call(vs=float("inf")) == fa.FA_ERR_UNSUPPORTED
+    assert call(ks=float("nan")) == fa.FA_ERR_UNSUPPORTED
+    assert call(sl=None) == fa.FA_ERR_NULL
+    assert call(wbytes=need - 1) == fa.FA_ERR_WORKSPACE
+    assert call(B=0) == fa.FA_OK
+
+
 def test_paged_decode_validation(fa):
     L = fa.lib
     q, pool, o = _t(2, 1, 8, 128), _t(6, 128, 2, 128), _t(2, 1, 8, 128)

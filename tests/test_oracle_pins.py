@@ -324,6 +324,38 @@ def test_varlen_attention_is_attention_of_each_sequence_alone():
         oracle.attention_varlen(qp, kp, vp, cq[:-1], ck[:-1], False, 0.3)   # sums do not reach the end
 
 
+def test_e4m3_values_and_fp8_decode():
+    # the format's landmarks: 0x38 = 1, 0x40 = 2, 0x01 = 2^-9 (smallest subnormal), 0x08 = 2^-6
+    # (smallest normal), 0x7e = 448 (largest), 0x7f / 0xff = NaN, sign bit; and all 256 patterns
+    # against torch's own conversion (a library routine the decoder does not use)
+    val = oracle.e4m3_to_float64(torch.tensor([0x38, 0x40, 0x01, 0x08, 0x7e, 0xb8, 0x00, 0x80, 0x3c], dtype=torch.uint8))
+    assert val.tolist() == [1.0, 2.0, 2.0 ** -9, 2.0 ** -6, 448.0, -1.0, 0.0, 0.0, 1.5]
+    assert torch.isnan(oracle.e4m3_to_float64(torch.tensor([0x7f, 0xff], dtype=torch.uint8))).all()
+    bits = torch.arange(256, dtype=torch.uint8)
+    mine, ref = oracle.e4m3_to_float64(bits), bits.view(torch.float8_e4m3fn).to(torch.float64)
+    assert ((mine == ref) | (torch.isnan(mine) & torch.isnan(ref))).all()
+    # fp8 decode = decode on the widened, scaled cache; NaN patterns past a sequence's end are ignored;
+    # doubling v_scale doubles O and leaves LSE, and k_scale is interchangeable with the softmax scale
+    B, Hq, Hkv, Smax, d = 2, 4, 2, 9, 8
+    q = rnd((B, 1, Hq, d), 70)
+    gen = torch.Generator().manual_seed(71)
+    k8 = torch.randint(0, 0x78, (B, Smax, Hkv, d), generator=gen, dtype=torch.uint8) | (torch.randint(0, 2, (B, Smax, Hkv, d), generator=gen, dtype=torch.uint8) << 7)
+    v8 = torch.randint(0, 0x78, (B, Smax, Hkv, d), generator=gen, dtype=torch.uint8)
+    seqlens = [9, 4]
+    k8[1, 4:] = 0x7f
+    v8[1, 4:] = 0xff
+    O, LSE = oracle.decode_fp8(q, k8, v8, seqlens, 0.3, 0.5, 0.25)
+    kf = k8.view(torch.float8_e4m3fn).to(torch.float64) * 0.5
+    vf = v8.view(torch.float8_e4m3fn).to(torch.float64) * 0.25
+    for b, n in enumerate(seqlens):
+        Ob, Lb = oracle.attention_full(q[b:b + 1], kf[b:b + 1, :n].contiguous(), vf[b:b + 1, :n].contiguous(), False, 0.3)
+        assert torch.equal(O[b], Ob[0, 0]) and torch.equal(LSE[b], Lb[0, :, 0])
+    O2, L2 = oracle.decode_fp8(q, k8, v8, seqlens, 0.3, 0.5, 0.5)
+    assert torch.allclose(O2, 2 * O, rtol=1e-14, atol=0) and torch.equal(L2, LSE)
+    O3, L3 = oracle.decode_fp8(q, k8, v8, seqlens, 0.15, 1.0, 0.25)
+    assert torch.allclose(O3, O, rtol=1e-12, atol=1e-14) and torch.allclose(L3, LSE, rtol=1e-12, atol=1e-14)
+
+
 def test_paged_decode_equals_decode_on_the_same_keys_wherever_the_pages_lie():
     # the paged form only changes where a key is stored: build the pools by hand (page p of
     # sequence b at a chosen pool slot), compare with decode on the contiguous caches, then move

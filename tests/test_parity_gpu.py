@@ -510,6 +510,78 @@ def test_c5_decode_full_size_sampled(fa, cfg):
                                    what=f"{cfg.name} b{b} h{h} n{n}")
 
 
+# ------------------------------------------------------------------ decode over an FP8 cache
+def run_decode_fp8(fa, q, k8, v8, seqlens_dev, scale, k_scale, v_scale):
+    B, _, Hq, d = q.shape
+    Smax, Hkv = k8.shape[1], k8.shape[2]
+    o, chk_o = guard_alloc((B, 1, Hq, d), torch.float16, DEV)
+    lse, chk_l = guard_alloc((B, Hq), torch.float32, DEV)
+    nbytes = fa.fa_decode_workspace_bytes(B, Hq, Hkv, Smax, d)
+    ws, chk_w = guard_alloc((max(nbytes // 4, 4),), torch.float32, DEV)
+    fa.fa_decode_fp8(q, k8, v8, o, lse, seqlens_dev, scale, k_scale, v_scale, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    return o, lse
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 2), (8, 1), (6, 2), (17, 1), (40, 2)])
+def test_decode_fp8_small_full(fa, hq, hkv):
+    # N(0,1) caches stored as e4m3 with factors 1/4 and 1/8 (so that the 8-bit grid is used over
+    # its range), NaN patterns past every sequence's end; lengths: full, empty, one key, ragged
+    cfg = synth.DecodeConfig("t", 5, hq, hkv, 1500, 1, 1500, seed=hq * 41 + hkv)
+    q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    sl[0], sl[1], sl[2] = 1500, 0, 1
+    k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+    o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, 0.25, 0.125)
+    o, lse = run_decode_fp8(fa, q.to(DEV), k8.to(DEV), v8.to(DEV), sl.to(DEV), cfg.scale, 0.25, 0.125)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what=f"fp8 decode {hq}/{hkv}")
+    assert float(o[1].abs().max()) == 0.0 and torch.isneginf(lse[1]).all()
+
+
+def test_decode_fp8_every_bit_pattern_in_every_position(fa):
+    # every finite e4m3 pattern in K and V (drawn uniformly over the bit patterns, so that
+    # subnormals, both signs and the largest values occur), lengths around tile and chunk
+    # boundaries; the factors keep the scores in a sane range
+    cfg = synth.DecodeConfig("t", 6, 8, 4, 4096, 1, 4096, seed=555)
+    q, _, _, _ = synth.decode_inputs(cfg, "cpu", poison=False)
+    gen = torch.Generator().manual_seed(556)
+    shape = (cfg.B, cfg.Smax, cfg.Hkv, cfg.d)
+    mag = torch.randint(0, 0x7f, shape, generator=gen, dtype=torch.uint8)       # 0x00 .. 0x7e
+    sgn = torch.randint(0, 2, shape, generator=gen, dtype=torch.uint8) << 7
+    k8, v8 = mag | sgn, torch.randint(0, 0x7f, shape, generator=gen, dtype=torch.uint8) | sgn
+    sl = torch.tensor([127, 128, 129, 2047, 2049, 4096], dtype=torch.int32)
+    for b in range(cfg.B):
+        k8[b, int(sl[b]):] = 0xff
+        v8[b, int(sl[b]):] = 0x7f
+    ks, vs = 1.0 / 256, 1.0 / 64
+    o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, ks, vs)
+    o, lse = run_decode_fp8(fa, q.to(DEV), k8.to(DEV), v8.to(DEV), sl.to(DEV), cfg.scale, ks, vs)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what="fp8 decode, all patterns")
+
+
+@pytest.mark.parametrize("cfg", [synth.C5_MHA, synth.C5_GQA], ids=["mha", "gqa"])
+def test_c5_decode_fp8_full_size_sampled(fa, cfg):
+    q, k, v, sl = synth.decode_inputs(cfg, DEV, poison=False)
+    k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+    del k, v
+    o, lse = run_decode_fp8(fa, q, k8, v8, sl.to(DEV), cfg.scale, 0.25, 0.125)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    g = cfg.Hq // cfg.Hkv
+    gen = torch.Generator().manual_seed(cfg.seed + 6)
+    order = torch.argsort(sl)
+    seqs = {int(order[0]), int(order[-1]), 0, cfg.B - 1}
+    seqs.update(int(x) for x in torch.randint(0, cfg.B, (4,), generator=gen))
+    for b in sorted(seqs):
+        n = int(sl[b])
+        for h in sorted({0, g - 1, cfg.Hq - 1, int(torch.randint(0, cfg.Hq, (1,), generator=gen))}):
+            hk = h // g
+            o_ref, l_ref = oracle.decode_fp8(q[b:b + 1, :, h:h + 1].cpu(), k8[b:b + 1, :n, hk:hk + 1].contiguous().cpu(),
+                                             v8[b:b + 1, :n, hk:hk + 1].contiguous().cpu(), [n], cfg.scale, 0.25, 0.125)
+            assert_close_to_oracle(o[b, 0, h].view(1, 1, -1), lse[b, h].view(1, 1), o_ref, l_ref,
+                                   what=f"{cfg.name} fp8 b{b} h{h} n{n}")
+
+
 # ------------------------------------------------------------------ decode over a paged cache
 def run_decode_paged(fa, q, kp, vp, table_dev, seqlens_dev, scale, max_pages=None):
     B, _, Hq, d = q.shape
