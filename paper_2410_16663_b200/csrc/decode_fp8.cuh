@@ -13,6 +13,16 @@ namespace fa {
 
 constexpr int kDec8Stages = 4;
 constexpr int kDec8TileBytes = 16384;   // 128 keys x 128 one-byte elements
+#ifndef FA_DEC8_WARPS
+#define FA_DEC8_WARPS 4
+#endif
+// Consumer warps: each owns kDec8KeysPerWarp keys of every tile.  Four warps of 32 keys as in the
+// fp16 kernel; eight warps of 16 keys (two per scheduler) were 5 % slower: the kernel is bound
+// by the throughput of the conversions and the warp-level MMAs, not by their latency.
+constexpr int kDec8Warps = FA_DEC8_WARPS;
+constexpr int kDec8KeysPerWarp = kDecTile / kDec8Warps;
+constexpr int kDec8Threads = (kDec8Warps + 1) * 32;
+static_assert(kDec8KeysPerWarp == 16 || kDec8KeysPerWarp == 32, "a warp owns one or two MMA k-steps of keys");
 
 // Four e4m3 bytes -> two fp16 pairs: (byte 0, byte 1) and (byte 2, byte 3).  (Widening on the
 // integer pipe instead -- the byte moved into the upper half of a halfword with its low seven
@@ -25,7 +35,7 @@ __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t in, uint32_t& lo, uin
 }
 
 // grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
-__global__ void __launch_bounds__(kDecMmaThreads, 1)
+__global__ void __launch_bounds__(kDec8Threads, 1)
 fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -55,13 +65,13 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     if (tid == 0) {
         for (int i = 0; i < 2 * kDec8Stages; ++i) mbar_init(smem_u32(&bars[i]), 1);
-        for (int i = 0; i < kDec8Stages; ++i) mbar_init(smem_u32(&bars[2 * kDec8Stages + i]), 4);  // one arrival per consumer warp
+        for (int i = 0; i < kDec8Stages; ++i) mbar_init(smem_u32(&bars[2 * kDec8Stages + i]), kDec8Warps);  // one arrival per consumer warp
         abort_flag = 0;
         fence_mbar_init();
     }
     __syncthreads();
 
-    if (warp == 4) {
+    if (warp == kDec8Warps) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
             // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
@@ -110,7 +120,7 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 #pragma unroll
         for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
         float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;  // rows g and g + 8
-        const int key_w = warp * 32;  // this warp's keys inside a tile
+        const int key_w = warp * kDec8KeysPerWarp;  // this warp's keys inside a tile
         bool ok = true;
 
         for (int t = 0; t < n_tiles; ++t) {
@@ -120,12 +130,12 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             ok = mbar_wait(smem_u32(&bars[st]), parity, &abort_flag, 20);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            float sc[4][4];
+            float sc[kDec8KeysPerWarp / 8][4];
             if (valid > 0) {
                 // ---- S = Q K^T for this warp's four blocks of 8 keys
                 const uint32_t kt = sK + st * kDec8TileBytes;
 #pragma unroll
-                for (int nb = 0; nb < 4; ++nb) {
+                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
                     sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
                     const int key = key_w + nb * 8 + (lane & 7);
 #pragma unroll
@@ -145,7 +155,7 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 // ---- mask, running max, probabilities
                 float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-                for (int nb = 0; nb < 4; ++nb) {
+                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
                     const int k0 = nb * 8 + 2 * t4;
                     if (k0 >= valid) sc[nb][0] = sc[nb][2] = -INFINITY;
                     if (k0 + 1 >= valid) sc[nb][1] = sc[nb][3] = -INFINITY;
@@ -164,7 +174,7 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 const float nm_lo = -mn_lo * p.scale_log2, nm_hi = -mn_hi * p.scale_log2;
                 float s_lo = 0.f, s_hi = 0.f;
 #pragma unroll
-                for (int nb = 0; nb < 4; ++nb) {
+                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
                     const int k0 = nb * 8 + 2 * t4;
                     sc[nb][0] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][0], p.scale_log2, nm_lo)) : 0.f;
                     sc[nb][1] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][1], p.scale_log2, nm_lo)) : 0.f;
@@ -188,9 +198,9 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             if (!ok) break;
             if (valid > 0) {
                 const uint32_t vt = sV + st * kDec8TileBytes;
-                if (valid < 32) {
+                if (valid < kDec8KeysPerWarp) {
                     // rows past the sequence may hold NaN bits: zero them (0 * NaN would poison O)
-                    for (int i = lane; i < (32 - valid) * 8; i += 32) {
+                    for (int i = lane; i < (kDec8KeysPerWarp - valid) * 8; i += 32) {
                         const int key = key_w + valid + (i >> 3), ch = i & 7;
                         const uint32_t addr = vt + key * 128 + ((ch ^ (key & 7)) << 4);
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
@@ -199,7 +209,7 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 }
                 // ---- O += P V: two k-steps of 16 keys, sixteen blocks of 8 output columns
 #pragma unroll
-                for (int k2 = 0; k2 < 2; ++k2) {
+                for (int k2 = 0; k2 < kDec8KeysPerWarp / 16; ++k2) {
                     uint32_t pa[4];
                     {
                         __half2 h0 = __floats2half2_rn(sc[2 * k2][0], sc[2 * k2][1]);
@@ -249,8 +259,8 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
         float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][128]
-        float* ml = mo + 4 * 16 * 128;                                                       // [4][16][2]: m, l
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        float* ml = mo + kDec8Warps * 16 * 128;                                                       // [4][16][2]: m, l
+        asm volatile("bar.sync 1, %0;" ::"n"(kDec8Warps * 32) : "memory");
         if (ok) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
@@ -268,23 +278,24 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 ml[(warp * 16 + g + 8) * 2 + 1] = l_hi;
             }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kDec8Warps * 32) : "memory");
         if (ok) {
-            for (int r = 0; r < G; ++r) {  // thread `tid` owns output column `tid` of every row
+            const int col = tid & 127;   // a thread owns one output column of every second (or fourth ...) row
+            for (int r = tid >> 7; r < G; r += kDec8Warps / 4) {
                 float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) M = fmaxf(M, ml[(w * 16 + r) * 2]);
+                for (int w = 0; w < kDec8Warps; ++w) M = fmaxf(M, ml[(w * 16 + r) * 2]);
                 float l = 0.f, acc = 0.f;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
+                for (int w = 0; w < kDec8Warps; ++w) {
                     const float mw = ml[(w * 16 + r) * 2];
                     const float sw = (mw == -INFINITY) ? 0.f : fast_exp2((mw - M) * p.scale_log2);
                     l += sw * ml[(w * 16 + r) * 2 + 1];
-                    acc += sw * mo[(w * 16 + r) * 128 + tid];
+                    acc += sw * mo[(w * 16 + r) * 128 + col];
                 }
                 const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;
-                p.o_part[slot * 128 + tid] = acc / l * p.v_scale;
-                if (tid == 0) p.lse_part[slot] = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
+                p.o_part[slot * 128 + col] = acc / l * p.v_scale;
+                if (col == 0) p.lse_part[slot] = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
             }
         }
     }

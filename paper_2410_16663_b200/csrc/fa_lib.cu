@@ -537,7 +537,7 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(fa::fa_decode_split_fp8_kernel), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
-        fa::fa_decode_split_fp8_kernel<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
+        fa::fa_decode_split_fp8_kernel<<<grid, fa::kDec8Threads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
