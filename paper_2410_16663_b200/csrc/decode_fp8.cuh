@@ -1,9 +1,10 @@
 // Decode-stage attention over an 8-bit cache (Appendix D.2 runs the operator with 8-bit operands;
 // here the cached K and V are FP8 e4m3 with one scale each, the queries and the probabilities
-// stay fp16): the split kernel of decode.cuh with half the cache bytes per key.  K and V tiles of
-// 128 keys x 128 bytes arrive through TMA (one 128-byte-swizzled box each); the 8-bit rows go
-// through ldmatrix as if they were 16-bit elements and are widened to fp16 pairs in registers
-// (cvt.rn.f16x2.e4m3x2) on their way into the same warp-level m16n8k16 MMAs.  The key scale is
+// stay fp16): the structure of the split kernel of decode.cuh with half the cache bytes per key.
+// K and V tiles of 128 keys x 128 bytes arrive through TMA (one 128-byte-swizzled box each); the
+// 8-bit rows go through ldmatrix as if they were 16-bit elements and are widened to fp16 pairs in
+// registers (cvt.rn.f16x2.e4m3x2) on their way into warp-level m16n8k16 MMAs, whose rows are keys
+// and whose columns are query heads (the products are taken transposed).  The key scale is
 // folded into the softmax scale, the value scale into the partial output.
 #pragma once
 
@@ -13,16 +14,8 @@ namespace fa {
 
 constexpr int kDec8Stages = 4;
 constexpr int kDec8TileBytes = 16384;   // 128 keys x 128 one-byte elements
-#ifndef FA_DEC8_WARPS
-#define FA_DEC8_WARPS 4
-#endif
-// Consumer warps: each owns kDec8KeysPerWarp keys of every tile.  Four warps of 32 keys as in the
-// fp16 kernel; eight warps of 16 keys (two per scheduler) were 5 % slower: the kernel is bound
-// by the throughput of the conversions and the warp-level MMAs, not by their latency.
-constexpr int kDec8Warps = FA_DEC8_WARPS;
-constexpr int kDec8KeysPerWarp = kDecTile / kDec8Warps;
+constexpr int kDec8Warps = 4;            // consumer warps, 32 keys of every tile each (as in the fp16 kernel)
 constexpr int kDec8Threads = (kDec8Warps + 1) * 32;
-static_assert(kDec8KeysPerWarp == 16 || kDec8KeysPerWarp == 32, "a warp owns one or two MMA k-steps of keys");
 
 // Four e4m3 bytes -> two fp16 pairs: (byte 0, byte 1) and (byte 2, byte 3).  (Widening on the
 // integer pipe instead -- the byte moved into the upper half of a halfword with its low seven
@@ -35,6 +28,7 @@ __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t in, uint32_t& lo, uin
 }
 
 // grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
+template <int NB>
 __global__ void __launch_bounds__(kDec8Threads, 1)
 fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
@@ -98,29 +92,42 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         __syncwarp();
     } else {
         // ---------------------------------------------------------------- consumers
-        const int g = lane >> 2, t4 = lane & 3;  // fragment row (query head g and g + 8) and column pair
-        // Q as A fragments for the eight k-steps of d = 128 (rows >= G are zero).  A k-step
-        // covers 16 consecutive d, but in the order the 8-bit K rows come out of ldmatrix: a
-        // thread's four bytes of a 16-byte chunk are d = 4 t4 .. 4 t4 + 3, which become the
-        // k-step's columns (2 t4, 2 t4 + 1) and (2 t4 + 8, 2 t4 + 9).  The dot product over d does
-        // not care about the order as long as Q uses the same one.
-        uint32_t qa[8][4];
+        // The products are taken transposed, S^T = K q^T and O^T = V^T P^T: the 16 rows of an
+        // MMA are keys (or output columns) and its 8 columns are query heads, so that a group of
+        // up to 8 heads costs half the MMAs of the head-major form (NB = 1; NB = 2 for 9..16 heads).
+        const int g = lane >> 2, t4 = lane & 3;
+        // q^T as B fragments: column g = head 8 nbk + g; a k-step's rows (2 t4, 2 t4 + 1) and
+        // (2 t4 + 8, 2 t4 + 9) are d = 16 ks + 4 t4 .. + 3, the order in which a thread receives a
+        // key's bytes from ldmatrix (the dot product over d does not care about the order)
+        uint32_t qb[NB][8][2];
         {
-            const __half* qb = static_cast<const __half*>(p.q) + ((long long)b * p.Hq + h0) * 128;
+            const __half* qp = static_cast<const __half*>(p.q) + ((long long)b * p.Hq + h0) * 128;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const int k0 = ks * 16 + 4 * t4;
-                qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0) : 0u;
-                qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0) : 0u;
-                qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0 + 2) : 0u;
-                qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0 + 2) : 0u;
+            for (int nbk = 0; nbk < NB; ++nbk) {
+                const int head = nbk * 8 + g;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const int d0 = ks * 16 + 4 * t4;
+                    qb[nbk][ks][0] = (head < G) ? *reinterpret_cast<const uint32_t*>(qp + head * 128 + d0) : 0u;
+                    qb[nbk][ks][1] = (head < G) ? *reinterpret_cast<const uint32_t*>(qp + head * 128 + d0 + 2) : 0u;
+                }
             }
         }
-        float o[16][4];
+        // O^T: block c holds output columns 16 c .. 16 c + 15 as MMA rows (row g = column
+        // 16 c + 2 g, row g + 8 = column 16 c + 2 g + 1) for heads 8 nbk + 2 t4 and + 1
+        float o[8][NB][4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-        float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;  // rows g and g + 8
-        const int key_w = warp * kDec8KeysPerWarp;  // this warp's keys inside a tile
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int nbk = 0; nbk < NB; ++nbk) o[i][nbk][0] = o[i][nbk][1] = o[i][nbk][2] = o[i][nbk][3] = 0.f;
+        // running max and (per-thread partial) sum for heads 8 nbk + 2 t4 (index 0) and + 1 (index 1)
+        float m_run[NB][2], l_run[NB][2];
+#pragma unroll
+        for (int nbk = 0; nbk < NB; ++nbk) {
+            m_run[nbk][0] = m_run[nbk][1] = -INFINITY;
+            l_run[nbk][0] = l_run[nbk][1] = 0.f;
+        }
+        const int key_w = warp * 32;  // this warp's keys inside a tile
         bool ok = true;
 
         for (int t = 0; t < n_tiles; ++t) {
@@ -130,67 +137,82 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             ok = mbar_wait(smem_u32(&bars[st]), parity, &abort_flag, 20);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            float sc[kDec8KeysPerWarp / 8][4];
+            uint32_t pt[2][NB][2];   // P^T as B fragments per 16-key step
             if (valid > 0) {
-                // ---- S = Q K^T for this warp's four blocks of 8 keys
+                // ---- S^T = K q^T: two blocks of 16 keys
+                float sc[2][NB][4];  // (key 16 mb + g, heads 2 t4, 2 t4 + 1), (key 16 mb + g + 8, same heads)
                 const uint32_t kt = sK + st * kDec8TileBytes;
 #pragma unroll
-                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
-                    sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
-                    const int key = key_w + nb * 8 + (lane & 7);
+                for (int mb = 0; mb < 2; ++mb) {
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {  // 4 chunks of 16 bytes per ldmatrix.x4 = four k-steps
-                        const int chunk = hf * 4 + (lane >> 3);
+                    for (int nbk = 0; nbk < NB; ++nbk) sc[mb][nbk][0] = sc[mb][nbk][1] = sc[mb][nbk][2] = sc[mb][nbk][3] = 0.f;
+                    const int key = key_w + mb * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {  // two 16-byte chunks (two k-steps) per ldmatrix.x4
+                        const int chunk = cc * 2 + (lane >> 4);
                         const uint32_t addr = kt + key * 128 + ((chunk ^ (key & 7)) << 4);
+                        // matrices: (keys 0-7, chunk 2 cc), (keys 8-15, chunk 2 cc), (keys 0-7, chunk 2 cc + 1), (keys 8-15, ...)
                         uint32_t w[4];
                         ldsm_x4(addr, w[0], w[1], w[2], w[3]);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint32_t b0, b1;   // d = 4 t4, 4 t4 + 1 and 4 t4 + 2, 4 t4 + 3 of the chunk, as fp16 pairs
-                            e4m3x4_to_f16x2x2(w[j], b0, b1);
-                            mma_16816(sc[nb], qa[hf * 4 + j], b0, b1);
+                        for (int j = 0; j < 2; ++j) {
+                            uint32_t a[4];
+                            e4m3x4_to_f16x2x2(w[2 * j], a[0], a[2]);      // keys g: d 4 t4, +1 | +2, +3
+                            e4m3x4_to_f16x2x2(w[2 * j + 1], a[1], a[3]);  // keys g + 8
+#pragma unroll
+                            for (int nbk = 0; nbk < NB; ++nbk)
+                                mma_16816(sc[mb][nbk], a, qb[nbk][cc * 2 + j][0], qb[nbk][cc * 2 + j][1]);
                         }
                     }
                 }
                 // ---- mask, running max, probabilities
-                float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
-                    const int k0 = nb * 8 + 2 * t4;
-                    if (k0 >= valid) sc[nb][0] = sc[nb][2] = -INFINITY;
-                    if (k0 + 1 >= valid) sc[nb][1] = sc[nb][3] = -INFINITY;
-                    mx_lo = fmaxf(mx_lo, fmaxf(sc[nb][0], sc[nb][1]));
-                    mx_hi = fmaxf(mx_hi, fmaxf(sc[nb][2], sc[nb][3]));
-                }
-                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-                mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-                mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);  // finite: key 0 of the warp is valid
-                const float a_lo = (m_lo == -INFINITY) ? 0.f : fast_exp2((m_lo - mn_lo) * p.scale_log2);
-                const float a_hi = (m_hi == -INFINITY) ? 0.f : fast_exp2((m_hi - mn_hi) * p.scale_log2);
-                m_lo = mn_lo;
-                m_hi = mn_hi;
-                const float nm_lo = -mn_lo * p.scale_log2, nm_hi = -mn_hi * p.scale_log2;
-                float s_lo = 0.f, s_hi = 0.f;
+                for (int nbk = 0; nbk < NB; ++nbk) {
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-                for (int nb = 0; nb < kDec8KeysPerWarp / 8; ++nb) {
-                    const int k0 = nb * 8 + 2 * t4;
-                    sc[nb][0] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][0], p.scale_log2, nm_lo)) : 0.f;
-                    sc[nb][1] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][1], p.scale_log2, nm_lo)) : 0.f;
-                    sc[nb][2] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][2], p.scale_log2, nm_hi)) : 0.f;
-                    sc[nb][3] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][3], p.scale_log2, nm_hi)) : 0.f;
-                    s_lo += sc[nb][0] + sc[nb][1];
-                    s_hi += sc[nb][2] + sc[nb][3];
-                }
-                l_lo = l_lo * a_lo + s_lo;  // per-thread partial of the row sum (the quad is summed at the end)
-                l_hi = l_hi * a_hi + s_hi;
+                    for (int mb = 0; mb < 2; ++mb) {
+                        const int k_lo = mb * 16 + g;
+                        if (k_lo >= valid) sc[mb][nbk][0] = sc[mb][nbk][1] = -INFINITY;
+                        if (k_lo + 8 >= valid) sc[mb][nbk][2] = sc[mb][nbk][3] = -INFINITY;
+                        mx0 = fmaxf(mx0, fmaxf(sc[mb][nbk][0], sc[mb][nbk][2]));
+                        mx1 = fmaxf(mx1, fmaxf(sc[mb][nbk][1], sc[mb][nbk][3]));
+                    }
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    o[i][0] *= a_lo;
-                    o[i][1] *= a_lo;
-                    o[i][2] *= a_hi;
-                    o[i][3] *= a_hi;
+                    for (int sh = 4; sh <= 16; sh <<= 1) {  // over the lanes that hold other keys of the same heads
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+                    }
+                    const float mn0 = fmaxf(m_run[nbk][0], mx0), mn1 = fmaxf(m_run[nbk][1], mx1);  // finite: key 0 of the warp is valid
+                    const float a0 = (m_run[nbk][0] == -INFINITY) ? 0.f : fast_exp2((m_run[nbk][0] - mn0) * p.scale_log2);
+                    const float a1 = (m_run[nbk][1] == -INFINITY) ? 0.f : fast_exp2((m_run[nbk][1] - mn1) * p.scale_log2);
+                    m_run[nbk][0] = mn0;
+                    m_run[nbk][1] = mn1;
+                    const float nm0 = -mn0 * p.scale_log2, nm1 = -mn1 * p.scale_log2;
+                    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                    for (int mb = 0; mb < 2; ++mb) {
+                        const int k_lo = mb * 16 + g;
+                        float* e = sc[mb][nbk];
+                        e[0] = (k_lo < valid) ? fast_exp2(fmaf(e[0], p.scale_log2, nm0)) : 0.f;
+                        e[1] = (k_lo < valid) ? fast_exp2(fmaf(e[1], p.scale_log2, nm1)) : 0.f;
+                        e[2] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[2], p.scale_log2, nm0)) : 0.f;
+                        e[3] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[3], p.scale_log2, nm1)) : 0.f;
+                        s0 += e[0] + e[2];
+                        s1 += e[1] + e[3];
+                        // (keys g | heads 2 t4, 2 t4 + 1) -> transposed: (head g | keys 2 t4, 2 t4 + 1), the B fragment
+                        __half2 lo = __floats2half2_rn(e[0], e[1]), hi = __floats2half2_rn(e[2], e[3]);
+                        asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pt[mb][nbk][0]) : "r"(*reinterpret_cast<uint32_t*>(&lo)));
+                        asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pt[mb][nbk][1]) : "r"(*reinterpret_cast<uint32_t*>(&hi)));
+                    }
+                    l_run[nbk][0] = l_run[nbk][0] * a0 + s0;  // per-thread partial of the sum over keys (reduced at the end)
+                    l_run[nbk][1] = l_run[nbk][1] * a1 + s1;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        o[i][nbk][0] *= a0;
+                        o[i][nbk][1] *= a1;
+                        o[i][nbk][2] *= a0;
+                        o[i][nbk][3] *= a1;
+                    }
                 }
             }
             ok = mbar_wait(smem_u32(&bars[kDec8Stages + st]), parity, &abort_flag, 21);
@@ -198,52 +220,43 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             if (!ok) break;
             if (valid > 0) {
                 const uint32_t vt = sV + st * kDec8TileBytes;
-                if (valid < kDec8KeysPerWarp) {
+                if (valid < 32) {
                     // rows past the sequence may hold NaN bits: zero them (0 * NaN would poison O)
-                    for (int i = lane; i < (kDec8KeysPerWarp - valid) * 8; i += 32) {
+                    for (int i = lane; i < (32 - valid) * 8; i += 32) {
                         const int key = key_w + valid + (i >> 3), ch = i & 7;
                         const uint32_t addr = vt + key * 128 + ((ch ^ (key & 7)) << 4);
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                     __syncwarp();
                 }
-                // ---- O += P V: two k-steps of 16 keys, sixteen blocks of 8 output columns
+                // ---- O^T += V^T P^T: two k-steps of 16 keys, eight blocks of 16 output columns
 #pragma unroll
-                for (int k2 = 0; k2 < kDec8KeysPerWarp / 16; ++k2) {
-                    uint32_t pa[4];
-                    {
-                        __half2 h0 = __floats2half2_rn(sc[2 * k2][0], sc[2 * k2][1]);
-                        __half2 h1 = __floats2half2_rn(sc[2 * k2][2], sc[2 * k2][3]);
-                        __half2 h2 = __floats2half2_rn(sc[2 * k2 + 1][0], sc[2 * k2 + 1][1]);
-                        __half2 h3 = __floats2half2_rn(sc[2 * k2 + 1][2], sc[2 * k2 + 1][3]);
-                        pa[0] = *reinterpret_cast<uint32_t*>(&h0);
-                        pa[1] = *reinterpret_cast<uint32_t*>(&h1);
-                        pa[2] = *reinterpret_cast<uint32_t*>(&h2);
-                        pa[3] = *reinterpret_cast<uint32_t*>(&h3);
-                    }
+                for (int k2 = 0; k2 < 2; ++k2) {
                     const int key = key_w + k2 * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {  // two 16-byte chunks (32 output columns) per ldmatrix.x4.trans
+                    for (int q4 = 0; q4 < 4; ++q4) {  // two 16-byte chunks per ldmatrix.x4.trans
                         const int ch = q4 * 2 + (lane >> 4);
                         const uint32_t addr = vt + key * 128 + ((ch ^ (key & 7)) << 4);
                         // matrices: (keys 0-7, chunk 2 q4), (keys 8-15, chunk 2 q4), (keys 0-7, chunk 2 q4 + 1), (keys 8-15, ...)
                         uint32_t w[4];
                         ldsm_x4_trans(addr, w[0], w[1], w[2], w[3]);
-                        // a transposed 16-bit element is the byte pair (2g, 2g + 1) of one key; the register
-                        // holds it for keys 2 t4 and 2 t4 + 1.  Regrouped by byte: the even column of both
-                        // keys, then the odd column of both keys, each converted to an fp16 pair.
+                        // a transposed 16-bit element is the byte pair (2g, 2g + 1) of one key, held for keys
+                        // 2 t4 and 2 t4 + 1; regrouped by byte: column 2g of both keys, then column 2g + 1
                         uint32_t ev[4], od[4];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            uint32_t t;
-                            asm("prmt.b32 %0, %1, %1, 0x3120;" : "=r"(t) : "r"(w[j]));
-                            e4m3x4_to_f16x2x2(t, ev[j], od[j]);
+                            uint32_t tw;
+                            asm("prmt.b32 %0, %1, %1, 0x3120;" : "=r"(tw) : "r"(w[j]));
+                            e4m3x4_to_f16x2x2(tw, ev[j], od[j]);
                         }
-                        // accumulator block 2c + parity holds output columns 16c + 2n + parity, n = the MMA's column
-                        mma_16816(o[4 * q4], pa, ev[0], ev[1]);
-                        mma_16816(o[4 * q4 + 1], pa, od[0], od[1]);
-                        mma_16816(o[4 * q4 + 2], pa, ev[2], ev[3]);
-                        mma_16816(o[4 * q4 + 3], pa, od[2], od[3]);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            // rows g: even columns, rows g + 8: odd columns; k: keys 2 t4.. | keys 2 t4 + 8..
+                            const uint32_t a[4] = {ev[2 * j], od[2 * j], ev[2 * j + 1], od[2 * j + 1]};
+#pragma unroll
+                            for (int nbk = 0; nbk < NB; ++nbk)
+                                mma_16816(o[q4 * 2 + j][nbk], a, pt[k2][nbk][0], pt[k2][nbk][1]);
+                        }
                     }
                 }
             }
@@ -251,36 +264,41 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kDec8Stages + st]));
         }
 
-        // ---- merge the four warps' states and write this chunk's partial result
-        // (all tiles this CTA requested have been consumed by every warp before the barrier below,
-        // so the ring can be reused as the merge buffer)
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][128]
-        float* ml = mo + kDec8Warps * 16 * 128;                                                       // [4][16][2]: m, l
+        // ---- merge the warps' states and write this chunk's partial result (the ring is free:
+        // every warp has consumed all tiles this CTA requested before the barrier below)
+#pragma unroll
+        for (int nbk = 0; nbk < NB; ++nbk)
+#pragma unroll
+            for (int sh = 4; sh <= 16; sh <<= 1) {
+                l_run[nbk][0] += __shfl_xor_sync(0xffffffffu, l_run[nbk][0], sh);
+                l_run[nbk][1] += __shfl_xor_sync(0xffffffffu, l_run[nbk][1], sh);
+            }
+        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [warps][16 heads][128]
+        float* ml = mo + kDec8Warps * 16 * 128;                                              // [warps][16][2]: m, l
         asm volatile("bar.sync 1, %0;" ::"n"(kDec8Warps * 32) : "memory");
         if (ok) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                // block i = 2c + parity: MMA columns 2 t4 and 2 t4 + 1 are output columns 16c + 4 t4 + parity and + 2
-                const int col = (i >> 1) * 16 + 4 * t4 + (i & 1);
-                mo[(warp * 16 + g) * 128 + col] = o[i][0];
-                mo[(warp * 16 + g) * 128 + col + 2] = o[i][1];
-                mo[(warp * 16 + g + 8) * 128 + col] = o[i][2];
-                mo[(warp * 16 + g + 8) * 128 + col + 2] = o[i][3];
-            }
-            if (t4 == 0) {
-                ml[(warp * 16 + g) * 2] = m_lo;
-                ml[(warp * 16 + g) * 2 + 1] = l_lo;
-                ml[(warp * 16 + g + 8) * 2] = m_hi;
-                ml[(warp * 16 + g + 8) * 2 + 1] = l_hi;
+            for (int nbk = 0; nbk < NB; ++nbk) {
+                const int head = nbk * 8 + 2 * t4;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int col = i * 16 + 2 * g;
+                    mo[(warp * 16 + head) * 128 + col] = o[i][nbk][0];
+                    mo[(warp * 16 + head + 1) * 128 + col] = o[i][nbk][1];
+                    mo[(warp * 16 + head) * 128 + col + 1] = o[i][nbk][2];
+                    mo[(warp * 16 + head + 1) * 128 + col + 1] = o[i][nbk][3];
+                }
+                if (g == 0) {
+                    ml[(warp * 16 + head) * 2] = m_run[nbk][0];
+                    ml[(warp * 16 + head) * 2 + 1] = l_run[nbk][0];
+                    ml[(warp * 16 + head + 1) * 2] = m_run[nbk][1];
+                    ml[(warp * 16 + head + 1) * 2 + 1] = l_run[nbk][1];
+                }
             }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(kDec8Warps * 32) : "memory");
         if (ok) {
-            const int col = tid & 127;   // a thread owns one output column of every second (or fourth ...) row
+            const int col = tid & 127;   // a thread owns one output column
             for (int r = tid >> 7; r < G; r += kDec8Warps / 4) {
                 float M = -INFINITY;
 #pragma unroll

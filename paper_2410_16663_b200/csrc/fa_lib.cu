@@ -534,10 +534,12 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDec8Stages * fa::kDec8TileBytes;
         int sm_count = 0;
-        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(fa::fa_decode_split_fp8_kernel), smem, &sm_count))
+        // keys as the MMA's rows and up to 8 query heads as its columns (two column blocks for 9..16 heads)
+        auto kern = (g > 8) ? fa::fa_decode_split_fp8_kernel<2> : fa::fa_decode_split_fp8_kernel<1>;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
-        fa::fa_decode_split_fp8_kernel<<<grid, fa::kDec8Threads, smem, st>>>(tk, tv, dp);
+        kern<<<grid, fa::kDec8Threads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
