@@ -157,6 +157,13 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
                   const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
                   float k_scale, float v_scale, void* workspace, size_t workspace_bytes, void* stream);
 
+/* fa_decode_fp8 over a paged cache: k_pages, v_pages [num_pages, page_size, Hkv, d] of e4m3 bytes;
+ * block_table, page_size, max_pages, table_stride as for fa_decode_paged, scales as for fa_decode_fp8. */
+int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                        void* o, float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages,
+                        int page_size, int max_pages, int table_stride, int d, float scale, float k_scale,
+                        float v_scale, void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * Decode over a paged cache: the same computation as fa_decode (Appendix C), with the cached
  * keys and values of a sequence scattered over fixed-size pages of a pool shared by all

@@ -49,6 +49,8 @@ lib.fa_forward_varlen.restype = _i
 lib.fa_forward_varlen.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p]
 lib.fa_decode_fp8.restype = _i
 lib.fa_decode_fp8.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
+lib.fa_decode_fp8_paged.restype = _i
+lib.fa_decode_fp8_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
 lib.fa_decode_paged.restype = _i
 lib.fa_decode_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_noalloc.restype = _i
@@ -67,7 +69,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -174,6 +176,21 @@ def fa_decode_fp8(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, k_scale:
     rc = lib.fa_decode_fp8(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq, Hkv,
                            Smax, d, float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode_fp8", raise_on_error)
+
+
+def fa_decode_fp8_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, k_scale: float,
+                        v_scale: float, workspace, max_pages: int = None, raise_on_error: bool = True) -> int:
+    """``fa_decode_fp8_paged``: as ``fa_decode_paged`` with pools of FP8 e4m3 bytes and one factor per tensor."""
+    B, _, Hq, d = q.shape
+    num_pages, page_size, Hkv, _ = k_pages.shape
+    stride = block_table.stride(0) if block_table.dim() == 2 else block_table.numel() // max(1, B)
+    if max_pages is None:
+        max_pages = block_table.shape[1]
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_fp8_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(o), _ptr(lse),
+                                 _ptr(seqlens_k), B, Hq, Hkv, num_pages, page_size, int(max_pages), int(stride), d,
+                                 float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
+    return _check(rc, "fa_decode_fp8_paged", raise_on_error)
 
 
 def fa_decode_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, workspace,

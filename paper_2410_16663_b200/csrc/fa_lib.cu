@@ -492,9 +492,11 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
                        workspace_bytes, stream, nullptr, 0, 0, 0);
 }
 
-int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
-                  int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale, float v_scale,
-                  void* workspace, size_t workspace_bytes, void* stream) {
+// FP8 cache, contiguous (block_table == nullptr) or in pages (Skv_max = max_pages * page_size).
+static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                           const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale,
+                           float v_scale, void* workspace, size_t workspace_bytes, void* stream, const int* block_table,
+                           int num_pages, int page_size, int table_stride) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
     if (Hq % Hkv) return FA_ERR_SHAPE;
     if (d != 128) return FA_ERR_UNSUPPORTED;
@@ -521,16 +523,18 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
     dp.o_part = static_cast<float*>(workspace);
     dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
     dp.scale_log2 = scale * k_scale * 1.4426950408889634f;   // the scores are q . (k_scale * k8)
-    dp.block_table = nullptr;
-    dp.page_size = 1;
-    dp.table_stride = 0;
+    dp.block_table = block_table;
+    dp.page_size = block_table ? page_size : 1;
+    dp.table_stride = table_stride;
     dp.v_scale = v_scale;
     const int g = Hq / Hkv;
     if (Skv_max > 0) {
         CUtensorMap tk, tv;
-        rc = encode_map_u8(&tk, k_cache, B, Skv_max, Hkv, fa::kDecTile);
+        const int slabs = block_table ? num_pages : B;          // outermost dimension: the sequence, or the page
+        const int slab_rows = block_table ? page_size : Skv_max;
+        rc = encode_map_u8(&tk, k_cache, slabs, slab_rows, Hkv, fa::kDecTile);
         if (rc) return rc;
-        rc = encode_map_u8(&tv, v_cache, B, Skv_max, Hkv, fa::kDecTile);
+        rc = encode_map_u8(&tv, v_cache, slabs, slab_rows, Hkv, fa::kDecTile);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDec8Stages * fa::kDec8TileBytes;
         int sm_count = 0;
@@ -547,6 +551,27 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+                  int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale, float v_scale,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_fp8_impl(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, k_scale, v_scale,
+                           workspace, workspace_bytes, stream, nullptr, 0, 0, 0);
+}
+
+int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+                        float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
+                        int max_pages, int table_stride, int d, float scale, float k_scale, float v_scale,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (num_pages < 0 || page_size <= 0 || max_pages < 0 || page_size % fa::kDecTile) return FA_ERR_SHAPE;
+    if (table_stride < max_pages) return FA_ERR_SHAPE;
+    if ((long long)max_pages * page_size > 0x7fffffffll) return FA_ERR_SHAPE;
+    if (B > 0 && max_pages > 0 && !block_table) return FA_ERR_NULL;
+    if (max_pages > 0 && num_pages == 0) return FA_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(block_table) & 3u) return FA_ERR_ALIGN;
+    return decode_fp8_impl(q, k_pages, v_pages, o, lse, seqlens_k, B, Hq, Hkv, max_pages * page_size, d, scale, k_scale,
+                           v_scale, workspace, workspace_bytes, stream, block_table, num_pages, page_size, table_stride);
 }
 
 int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
