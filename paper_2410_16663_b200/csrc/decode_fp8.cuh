@@ -12,7 +12,7 @@
 
 namespace fa {
 
-constexpr int kDec8Stages = 4;
+constexpr int kDec8Stages = 3;            // ring slots of one K and one V tile: 97 KiB per CTA, two CTAs per SM
 constexpr int kDec8TileBytes = 16384;   // 128 keys x 128 one-byte elements
 constexpr int kDec8Warps = 4;            // consumer warps, 32 keys of every tile each (as in the fp16 kernel)
 constexpr int kDec8Threads = (kDec8Warps + 1) * 32;
@@ -29,7 +29,7 @@ __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t in, uint32_t& lo, uin
 
 // grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
 template <int NB>
-__global__ void __launch_bounds__(kDec8Threads, 1)
+__global__ void __launch_bounds__(kDec8Threads, 2)
 fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
     extern __shared__ uint8_t smem_raw[];

@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--d", type=int, default=128, choices=[64, 128], help="head dimension (prefill only)")
     ap.add_argument("--dtype", default="fp16", choices=["fp16", "bf16"])
     ap.add_argument("--noncausal", action="store_true")
+    ap.add_argument("--fp8", action="store_true", help="decode: the cache as FP8 e4m3 (factors 1/4 and 1/8)")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
@@ -49,8 +50,13 @@ def main():
         ws = torch.empty(max(16, fa.fa_decode_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Smax, cfg.d)),
                          dtype=torch.uint8, device=dev)
         sld = sl.to(dev)
-        run = lambda: fa.fa_decode(q, k, v, o, lse, sld, cfg.scale, ws)
-        work, unit = float(sl.sum()) * cfg.Hkv * cfg.d * 4 / 1e9, "GB/s"
+        if a.fp8:
+            k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+            del k, v
+            run = lambda: fa.fa_decode_fp8(q, k8, v8, o, lse, sld, cfg.scale, 0.25, 0.125, ws)
+        else:
+            run = lambda: fa.fa_decode(q, k, v, o, lse, sld, cfg.scale, ws)
+        work, unit = float(sl.sum()) * cfg.Hkv * cfg.d * (2 if a.fp8 else 4) / 1e9, "GB/s"
     for _ in range(a.warmup):
         run()
     torch.cuda.synchronize()
