@@ -171,7 +171,8 @@ int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages,
  * the evaluation section).  Key j of sequence b is row (j mod page_size) of page
  * block_table[b * table_stride + j / page_size].
  *   k_pages, v_pages [num_pages, page_size, Hkv, d] fp16 on the device, 16-byte aligned;
- *   page_size a positive multiple of 128 (a 128-key tile never straddles two pages);
+ *   page_size a positive multiple of 128, or 16, 32 or 64 (a 128-key tile is then one box of a
+ *   page or several whole pages; other sizes are refused);
  *   block_table int32 on the DEVICE, table_stride >= max_pages entries per sequence; only the
  *   entries that cover keys [0, seqlens_k[b]) are read and they must lie in [0, num_pages)
  *   (a page index outside that range reads as zeros and never faults); rows of a page past the
@@ -179,7 +180,7 @@ int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages,
  *   seqlens_k [B] int32 on the DEVICE, clamped to [0, max_pages * page_size];
  *   q, o, lse, scale, stream as for fa_decode; workspace of at least
  *   fa_decode_workspace_bytes(B, Hq, Hkv, max_pages * page_size, d) bytes.
- * Errors: FA_ERR_SHAPE for page_size not a multiple of 128 or table_stride < max_pages;
+ * Errors: FA_ERR_SHAPE for a page_size other than those or table_stride < max_pages;
  * otherwise as fa_decode.
  */
 int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,

@@ -26,7 +26,8 @@ struct DecodeParams {
     float scale_log2;
     // paged cache (block_table != nullptr): key j of sequence b is row j % page_size of page
     // block_table[b * table_stride + j / page_size]; the tensor maps then run over
-    // [pages, page_size, Hkv, 128] and page_size is a multiple of kDecTile
+    // [pages, page_size, Hkv, 128]; page_size is a multiple of kDecTile, or 16, 32 or 64 (then a
+    // tile is several pages and the TMA box is one page high)
     const int* block_table;
     int page_size, table_stride;
     float v_scale;        // 8-bit cache only: factor of the stored values
@@ -107,6 +108,44 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
             // the table read is not on the path that refills a freed slot
             const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
+            if (table && p.page_size < kDecTile) {
+                // pages of 16, 32 or 64 keys: a tile is several pages, each its own TMA box (rows past
+                // the sequence's last page are not loaded: their scores are masked and their V rows
+                // zeroed by the consumers).  The pages of a tile are looked up one tile ahead.
+                const int ps = p.page_size, n_sub = kDecTile / ps;
+                int pg[8];
+                auto lookup = [&](int first_key) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int key = first_key + i * ps;
+                        pg[i] = (i < n_sub && key < k_end) ? table[key / ps] : -1;
+                    }
+                };
+                lookup(k_begin);
+                for (int t = 0; t < n_tiles; ++t) {
+                    const int st = t % kDecStages;
+                    const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                    const int row0 = k_begin + t * kDecTile;
+                    int cur[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) cur[i] = pg[i];
+                    if (t + 1 < n_tiles) lookup(row0 + kDecTile);
+                    if (!mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22)) break;
+                    const int live = min(n_sub, (k_end - row0 + ps - 1) / ps);   // pages of this tile that hold keys
+                    mbar_expect_tx(bk, (uint32_t)(live * ps) * 256u);
+                    mbar_expect_tx(bv, (uint32_t)(live * ps) * 256u);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (i < live) {
+                            const uint32_t offs = (uint32_t)(i * ps) * 128u;
+                            tma_load_4d(sK + st * kDecTileBytes + offs, &tm_k, bk, 0, hk, 0, cur[i]);
+                            tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur[i]);
+                            tma_load_4d(sV + st * kDecTileBytes + offs, &tm_v, bv, 0, hk, 0, cur[i]);
+                            tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur[i]);
+                        }
+                }
+            } else
+            {
             int page_next = table ? table[k_begin / p.page_size] : 0;
             for (int t = 0; t < n_tiles; ++t) {
                 const int st = t % kDecStages;
@@ -125,6 +164,7 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 mbar_expect_tx(bv, kDecTileBytes);
                 tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, slab);
                 tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
+            }
             }
         }
         __syncwarp();

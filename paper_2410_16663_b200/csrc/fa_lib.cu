@@ -90,6 +90,9 @@ int encode_map_u8(CUtensorMap* tm, const void* base, int B, int S, int H, int bo
     return FA_OK;
 }
 
+// a page holds a multiple of the 128-key tile, or 16, 32 or 64 keys (several pages per tile)
+bool page_size_ok(int ps) { return ps > 0 && (ps % fa::kDecTile == 0 || ps == 16 || ps == 32 || ps == 64); }
+
 int check_device() {
     static thread_local int cached_dev = -1, cached_rc = FA_OK;
     int dev = 0;
@@ -461,11 +464,12 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
         const int slabs = block_table ? num_pages : B;
         const int slab_rows = block_table ? page_size : Skv_max;
         CUtensorMap tk, tv;
+        const int box_rows = (block_table && page_size < fa::kDecTile) ? page_size : fa::kDecTile;
         rc = encode_map(&tk, k_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        fa::kDecTile, false);
+                        box_rows, false);
         if (rc) return rc;
         rc = encode_map(&tv, v_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        fa::kDecTile, false);
+                        box_rows, false);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
         int sm_count = 0;
@@ -532,9 +536,10 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
         CUtensorMap tk, tv;
         const int slabs = block_table ? num_pages : B;          // outermost dimension: the sequence, or the page
         const int slab_rows = block_table ? page_size : Skv_max;
-        rc = encode_map_u8(&tk, k_cache, slabs, slab_rows, Hkv, fa::kDecTile);
+        const int box_rows = (block_table && page_size < fa::kDecTile) ? page_size : fa::kDecTile;
+        rc = encode_map_u8(&tk, k_cache, slabs, slab_rows, Hkv, box_rows);
         if (rc) return rc;
-        rc = encode_map_u8(&tv, v_cache, slabs, slab_rows, Hkv, fa::kDecTile);
+        rc = encode_map_u8(&tv, v_cache, slabs, slab_rows, Hkv, box_rows);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDec8Stages * fa::kDec8TileBytes;
         int sm_count = 0;
@@ -564,7 +569,7 @@ int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages,
                         float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
                         int max_pages, int table_stride, int d, float scale, float k_scale, float v_scale,
                         void* workspace, size_t workspace_bytes, void* stream) {
-    if (num_pages < 0 || page_size <= 0 || max_pages < 0 || page_size % fa::kDecTile) return FA_ERR_SHAPE;
+    if (num_pages < 0 || max_pages < 0 || !page_size_ok(page_size)) return FA_ERR_SHAPE;
     if (table_stride < max_pages) return FA_ERR_SHAPE;
     if ((long long)max_pages * page_size > 0x7fffffffll) return FA_ERR_SHAPE;
     if (B > 0 && max_pages > 0 && !block_table) return FA_ERR_NULL;
@@ -578,7 +583,7 @@ int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, con
                     float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
                     int max_pages, int table_stride, int d, float scale, void* workspace, size_t workspace_bytes,
                     void* stream) {
-    if (num_pages < 0 || page_size <= 0 || max_pages < 0 || page_size % fa::kDecTile) return FA_ERR_SHAPE;
+    if (num_pages < 0 || max_pages < 0 || !page_size_ok(page_size)) return FA_ERR_SHAPE;
     if (table_stride < max_pages) return FA_ERR_SHAPE;
     if ((long long)max_pages * page_size > 0x7fffffffll) return FA_ERR_SHAPE;
     if (B > 0 && max_pages > 0 && !block_table) return FA_ERR_NULL;

@@ -163,7 +163,8 @@ def test_paged_decode_validation(fa):
         P(q), P(pool), P(pool), kw.get("table", P(table)), P(o), None, P(sl), kw.get("B", 2), 8, kw.get("Hkv", 2),
         kw.get("num_pages", 6), kw.get("page_size", 128), kw.get("max_pages", 3), kw.get("stride", 3), 128, 0.1,
         P(ws), kw.get("wbytes", need), None)
-    assert call(page_size=64) == fa.FA_ERR_SHAPE        # not a multiple of the 128-key tile
+    assert call(page_size=48) == fa.FA_ERR_SHAPE        # neither a multiple of the 128-key tile nor 16, 32, 64
+    assert call(page_size=8) == fa.FA_ERR_SHAPE
     assert call(page_size=192) == fa.FA_ERR_SHAPE
     assert call(page_size=0) == fa.FA_ERR_SHAPE
     assert call(stride=2) == fa.FA_ERR_SHAPE            # rows of the table overlap

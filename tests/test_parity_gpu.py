@@ -582,7 +582,8 @@ def test_c5_decode_fp8_full_size_sampled(fa, cfg):
                                    what=f"{cfg.name} fp8 b{b} h{h} n{n}")
 
 
-def test_decode_fp8_paged_equals_contiguous_fp8_decode(fa):
+@pytest.mark.parametrize("page", [256, 16, 64])
+def test_decode_fp8_paged_equals_contiguous_fp8_decode(fa, page):
     # the 8-bit cache in pages: bit for bit what fa_decode_fp8 gives on the same keys stored
     # contiguously (which the tests above check against the oracle), pages in random order, NaN
     # patterns in every unused row and page
@@ -591,21 +592,21 @@ def test_decode_fp8_paged_equals_contiguous_fp8_decode(fa):
     sl[0], sl[1], sl[2], sl[3] = 2048, 0, 1, 257
     k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
     o1, lse1 = run_decode_fp8(fa, q.to(DEV), k8.to(DEV), v8.to(DEV), sl.to(DEV), cfg.scale, 0.25, 0.125)
-    kp, vp, table = synth.paged_cache(k8, v8, sl, 256, seed=7, spare_pages=3, poison=False)
-    used = torch.zeros(kp.shape[0], 256, dtype=torch.bool)
+    kp, vp, table = synth.paged_cache(k8, v8, sl, page, seed=7, spare_pages=3, poison=False)
+    used = torch.zeros(kp.shape[0], page, dtype=torch.bool)
     for b in range(cfg.B):
         for j in range(int(sl[b])):
-            used[int(table[b, j // 256]), j % 256] = True
+            used[int(table[b, j // page]), j % page] = True
     kp[~used] = 0x7f
     vp[~used] = 0xff
     B, _, Hq, d = q.shape
     o2 = torch.full((B, 1, Hq, d), float("nan"), dtype=torch.float16, device=DEV)
     lse2 = torch.full((B, Hq), float("nan"), device=DEV)
-    ws = torch.empty(fa.fa_decode_workspace_bytes(B, Hq, cfg.Hkv, table.shape[1] * 256, d), dtype=torch.uint8, device=DEV)
+    ws = torch.empty(fa.fa_decode_workspace_bytes(B, Hq, cfg.Hkv, table.shape[1] * page, d), dtype=torch.uint8, device=DEV)
     fa.fa_decode_fp8_paged(q.to(DEV), kp.to(DEV), vp.to(DEV), table.to(DEV), o2, lse2, sl.to(DEV), cfg.scale, 0.25, 0.125, ws)
     torch.cuda.synchronize()
     check_status(fa)
-    assert table.shape[1] * 256 == cfg.Smax
+    assert table.shape[1] * page == cfg.Smax
     assert torch.equal(o1, o2) and torch.equal(lse1, lse2)
     o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, 0.25, 0.125)
     assert_close_to_oracle(o2[:, 0], lse2, o_ref, l_ref, what="fp8 paged decode")
@@ -627,7 +628,8 @@ def run_decode_paged(fa, q, kp, vp, table_dev, seqlens_dev, scale, max_pages=Non
     return o, lse
 
 
-@pytest.mark.parametrize("hq,hkv,page", [(4, 4, 128), (8, 2, 128), (8, 2, 256), (17, 1, 384), (40, 2, 512)])
+@pytest.mark.parametrize("hq,hkv,page", [(4, 4, 128), (8, 2, 128), (8, 2, 256), (17, 1, 384), (40, 2, 512),
+                                         (4, 4, 16), (8, 2, 32), (8, 1, 64), (17, 1, 16)])
 def test_decode_paged_small_full(fa, hq, hkv, page):
     # pages handed out in random order from a pool with unused pages; NaN in every row no key
     # lives in; lengths: several pages, none, one key, exactly one page, one past a page
