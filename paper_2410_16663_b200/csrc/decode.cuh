@@ -104,48 +104,43 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     if (warp == 4) {
         // ---------------------------------------------------------------- producer
-        if (lane == 0) {
-            // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
-            // the table read is not on the path that refills a freed slot
-            const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
-            if (table && p.page_size < kDecTile) {
-                // pages of 16, 32 or 64 keys: a tile is several pages, each its own TMA box (rows past
-                // the sequence's last page are not loaded: their scores are masked and their V rows
-                // zeroed by the consumers).  The pages of a tile are looked up one tile ahead.
-                const int ps = p.page_size, n_sub = kDecTile / ps;
-                int pg[8];
-                auto lookup = [&](int first_key) {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int key = first_key + i * ps;
-                        pg[i] = (i < n_sub && key < k_end) ? table[key / ps] : -1;
-                    }
-                };
-                lookup(k_begin);
-                for (int t = 0; t < n_tiles; ++t) {
-                    const int st = t % kDecStages;
-                    const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
-                    const int row0 = k_begin + t * kDecTile;
-                    int cur[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) cur[i] = pg[i];
-                    if (t + 1 < n_tiles) lookup(row0 + kDecTile);
-                    if (!mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22)) break;
-                    const int live = min(n_sub, (k_end - row0 + ps - 1) / ps);   // pages of this tile that hold keys
+        // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
+        // the table read is not on the path that refills a freed slot
+        const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
+        if (table && p.page_size < kDecTile) {
+            // pages of 16, 32 or 64 keys: a tile is several pages, each its own TMA box (pages past
+            // the sequence's last are not loaded: their scores are masked and their V rows zeroed
+            // by the consumers).  Lane i of the warp looks up and loads page i of every tile.
+            const int ps = p.page_size, n_sub = kDecTile / ps;
+            auto lookup = [&](int first_key) {
+                const int key = first_key + lane * ps;
+                return (lane < n_sub && key < k_end) ? table[key / ps] : -1;
+            };
+            int pg_next = lookup(k_begin);
+            for (int t = 0; t < n_tiles; ++t) {
+                const int st = t % kDecStages;
+                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                const int row0 = k_begin + t * kDecTile;
+                const int cur = pg_next;
+                if (t + 1 < n_tiles) pg_next = lookup(row0 + kDecTile);
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22);
+                if (!__shfl_sync(0xffffffffu, ok, 0)) break;
+                const int live = min(n_sub, (k_end - row0 + ps - 1) / ps);   // pages of this tile that hold keys
+                if (lane == 0) {
                     mbar_expect_tx(bk, (uint32_t)(live * ps) * 256u);
                     mbar_expect_tx(bv, (uint32_t)(live * ps) * 256u);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (i < live) {
-                            const uint32_t offs = (uint32_t)(i * ps) * 128u;
-                            tma_load_4d(sK + st * kDecTileBytes + offs, &tm_k, bk, 0, hk, 0, cur[i]);
-                            tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur[i]);
-                            tma_load_4d(sV + st * kDecTileBytes + offs, &tm_v, bv, 0, hk, 0, cur[i]);
-                            tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur[i]);
-                        }
                 }
-            } else
-            {
+                __syncwarp();
+                if (lane < live) {
+                    const uint32_t offs = (uint32_t)(lane * ps) * 128u;
+                    tma_load_4d(sK + st * kDecTileBytes + offs, &tm_k, bk, 0, hk, 0, cur);
+                    tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur);
+                    tma_load_4d(sV + st * kDecTileBytes + offs, &tm_v, bv, 0, hk, 0, cur);
+                    tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur);
+                }
+            }
+        } else if (lane == 0) {
             int page_next = table ? table[k_begin / p.page_size] : 0;
             for (int t = 0; t < n_tiles; ++t) {
                 const int st = t % kDecStages;
@@ -164,7 +159,6 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 mbar_expect_tx(bv, kDecTileBytes);
                 tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, slab);
                 tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
-            }
             }
         }
         __syncwarp();
