@@ -672,6 +672,45 @@ def test_c5_decode_paged_full_size_equals_contiguous_decode(fa, cfg):
     assert torch.equal(o1, o2) and torch.equal(lse1, lse2)
 
 
+# ------------------------------------------------------------------ stream capture
+def test_calls_can_be_captured_in_a_cuda_graph_and_replayed(fa):
+    # the entry points only launch kernels on the caller's stream (no allocation, no
+    # synchronisation), so after one warm-up call each they can be recorded in a CUDA graph;
+    # the replay on new inputs (same buffers) must give what a direct call gives
+    pc = synth.PrefillConfig("t", 2, 4, 2, 300, 1300, dtype="fp16", causal=True, seed=950)
+    dc = synth.DecodeConfig("t", 4, 8, 2, 3000, 1, 3000, seed=951)
+    q, k, v = synth.prefill_inputs(pc, DEV)
+    o = torch.empty_like(q); lse = torch.empty(pc.B, pc.Hq, pc.Sq, device=DEV)
+    dq, dk, dv, sl = synth.decode_inputs(dc, DEV, poison=True)
+    sld = sl.to(DEV)
+    do = torch.empty_like(dq); dl = torch.empty(dc.B, dc.Hq, device=DEV)
+    ws = torch.empty(fa.fa_decode_workspace_bytes(dc.B, dc.Hq, dc.Hkv, dc.Smax, dc.d), dtype=torch.uint8, device=DEV)
+
+    def both():
+        fa.fa_forward(q, k, v, o, lse, pc.causal, pc.scale)
+        fa.fa_decode(dq, dk, dv, do, dl, sld, dc.scale, ws)
+
+    both()                                  # first use of each kernel outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            both()
+    torch.cuda.synchronize()
+    q.copy_(torch.flip(q, dims=[1]))        # new inputs in the same buffers
+    dq.mul_(-1.0)
+    both()
+    torch.cuda.synchronize()
+    o_direct, lse_direct, do_direct, dl_direct = o.clone(), lse.clone(), do.clone(), dl.clone()
+    o.fill_(float("nan")); lse.fill_(float("nan")); do.fill_(float("nan")); dl.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert torch.equal(o, o_direct) and torch.equal(lse, lse_direct)
+    assert torch.equal(do, do_direct) and torch.equal(dl, dl_direct)
+
+
 # ------------------------------------------------------------------ host-buffer entry point
 def test_forward_host_entry(fa):
     c = synth.C1
