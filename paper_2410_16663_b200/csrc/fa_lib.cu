@@ -231,13 +231,13 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? FA_OK : cuda_fail(e);
     }
-    if (p.d == 64) {  // head dimension 64: one CTA per (batch, head, query tile), two CTAs per SM
-        auto kern = bf16 ? fa::fa_fwd_d64_kernel<__nv_bfloat16> : fa::fa_fwd_d64_kernel<__half>;
+    if (p.d == 64) {  // one CTA per (batch, head, query tile), four CTAs per SM
+        auto kern = bf16 ? fa::fa_fwd_d64_slim_kernel<__nv_bfloat16> : fa::fa_fwd_d64_slim_kernel<__half>;
         int sm_count = 0;
-        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64Smem, &sm_count))
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64SlimSmem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
-        kern<<<grid, 128, fa::kD64Smem, st>>>(tq, tk, tv, fp);
+        kern<<<grid, 128, fa::kD64SlimSmem, st>>>(tq, tk, tv, fp);
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? FA_OK : cuda_fail(e);
     }
