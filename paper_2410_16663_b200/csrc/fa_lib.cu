@@ -316,11 +316,18 @@ int forward_plain(const void* q, const void* k, const void* v, void* o, float* l
 
 // ---- decode helpers
 int decode_chunk(int B, int Hkv, int Smax) {
-    // Largest chunk that still leaves several waves of work items for 148 SMs; multiples of the tile.
-    const long long target = 4ll * 148;
-    int chunk = 2048;
-    while (chunk > 256 && (long long)B * Hkv * ((Smax + chunk - 1) / chunk) < target) chunk >>= 1;
-    return chunk;
+    // Keys per work item (multiples of the tile).  A CTA costs a few microseconds on top of its
+    // tiles (launch, the first loads' latency, the merge), so chunks are as long as the number of
+    // work items allows: 2048 keys when that still gives four waves on 148 SMs (sequences of
+    // different lengths then balance well); otherwise the longest chunk, up to 4096 keys, that
+    // keeps about one work item per SM (timed on one to sixteen sequences of 4K to 128K keys: e.g.
+    // one sequence of 32K keys with 8 kv heads takes 32 us with 2048-key chunks against 61 us with
+    // 256-key chunks); 256 keys when even that leaves SMs without work.
+    auto items = [&](int chunk) { return (long long)B * Hkv * ((Smax + chunk - 1) / chunk); };
+    if (items(2048) >= 4ll * 148) return 2048;
+    for (int chunk = 4096; chunk > 256; chunk >>= 1)
+        if (items(chunk) >= 120) return chunk;
+    return 256;
 }
 
 }  // namespace

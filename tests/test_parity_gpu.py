@@ -479,7 +479,8 @@ def test_decode_chunked_lengths_and_clamping(fa):
     # lengths on both sides of chunk and tile boundaries; a length beyond Smax is clamped
     cfg = synth.DecodeConfig("t", 8, 8, 8, 4096, 1, 4096, seed=321)
     q, k, v, _ = synth.decode_inputs(cfg, "cpu", poison=False)
-    sl = torch.tensor([127, 128, 129, 255, 256, 257, 4096, 99999], dtype=torch.int32)
+    # (the chunk length depends on the problem size: 256 to 4096 keys; the lengths straddle each candidate)
+    sl = torch.tensor([127, 129, 257, 511, 1025, 2047, 2049, 99999], dtype=torch.int32)
     o_ref, l_ref = oracle.decode(q, k, v, sl.clamp(max=4096), cfg.scale)
     o, lse = run_decode(fa, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), cfg.scale)
     assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what="decode boundaries")
