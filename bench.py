@@ -275,6 +275,7 @@ def run_product(args, rank, world, local_rank):
             out["prefill_long_context"] = run_long_context(fa, dev, peaks)
         out["decode_paged"] = run_decode_paged(fa, dec[0], dev, peaks)
         out["decode_fp8"] = run_decode_fp8(fa, dec[0], dev, peaks)
+        out["decode_append"] = run_decode_append(fa, dec[-1], dev, peaks)
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
@@ -372,6 +373,37 @@ def run_varlen(fa, dev, peaks, small=False, iters=10):
                         f"(sum {int(q.shape[0])}), Hq=Hkv={cfg.Hq}, bf16, packed", "ms": round(ms, 4),
             "tflops": round(tf, 1), "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4),
             "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4)}
+
+
+def run_decode_append(fa, d, dev, peaks, Sq=4, iters=5):
+    """The GQA decode configuration with four new tokens per sequence instead of one
+    (fa_decode_append: the queries of the last four cache positions, causal among themselves),
+    outside the timed steps.  The cache is read once, as in plain decode."""
+    cfg = d["cfg"]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + 21)
+    q = torch.randn(cfg.B, Sq, cfg.Hq, cfg.d, generator=gen, device=dev).to(torch.float16)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, Sq, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(16, fa.fa_decode_append_workspace_bytes(cfg.B, Sq, cfg.Hq, cfg.Hkv, cfg.Smax, cfg.d)),
+                     dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        fa.fa_decode_append(q, d["k"], d["v"], o, lse, d["sl"], cfg.scale, ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_decode_append(q, d["k"], d["v"], o, lse, d["sl"], cfg.scale, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    gbs = d["bytes"] / (ms * 1e-3) / 1e9
+    return {"workload": f"{cfg.name} with {Sq} new tokens per sequence", "ms": round(ms, 4), "gbs": round(gbs, 1),
+            "kv_bytes": d["bytes"], "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
+            "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
 
 
 def run_decode_fp8(fa, d, dev, peaks, iters=5):

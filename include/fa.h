@@ -142,6 +142,25 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * Decode after several tokens were appended (Appendix C with Sq > 1 new tokens per sequence, as
+ * in chunked or speculative decoding): the Sq query rows of sequence b are the LAST Sq positions
+ * of its cache, so query t (0 <= t < Sq) sees the keys 0 .. seqlens_k[b] - Sq + t -- the
+ * bottom-right aligned causal mask of fa_forward, computed by the split-KV decode kernels
+ * instead of the prefill kernel, which for a few query rows over a long cache would leave
+ * most of the GPU idle.
+ *   q, o [B,Sq,Hq,d] fp16 contiguous, lse [B,Hq,Sq] float or NULL; 1 <= Sq <= 64; caches,
+ *   seqlens_k (the lengths INCLUDING the Sq new tokens), scale, stream as for fa_decode.
+ *   A query that sees no key (seqlens_k[b] < Sq - t) gives O = 0 and LSE = -inf.
+ *   workspace: at least fa_decode_append_workspace_bytes(...) bytes, 16-byte aligned.
+ * Errors: as fa_decode; FA_ERR_UNSUPPORTED also for Sq > 64 or Sq > Skv_max.
+ */
+int fa_decode_append(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                     const int* seqlens_k, int B, int Sq, int Hq, int Hkv, int Skv_max, int d, float scale,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+size_t fa_decode_append_workspace_bytes(int B, int Sq, int Hq, int Hkv, int Skv_max, int d);
+
+/*
  * Decode over an 8-bit cache (Appendix D.2 evaluates the operator with 8-bit operands; in the
  * decode stage the cache dominates the traffic, so here it is the cached K and V that are 8-bit):
  * the computation of fa_decode with K = k_scale * k_cache and V = v_scale * v_cache, where

@@ -191,6 +191,31 @@ def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
     return O, LSE
 
 
+def decode_append(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
+    """Decode after ``Sq`` tokens were appended: q ``[B,Sq,Hq,d]`` holds the queries of the LAST
+    ``Sq`` positions of every sequence, whose cache ``[B,Smax,Hkv,d]`` has ``seqlens[b]`` valid
+    rows including those positions.  Per sequence this is ``attention_full`` with the causal,
+    bottom-right aligned mask over the valid prefix.  Returns ``(O [B,Sq,Hq,d], LSE [B,Hq,Sq])``
+    float64; a query that sees no key gives O = 0, LSE = -inf."""
+    q = torch.as_tensor(q)
+    k = torch.as_tensor(k_cache)
+    v = torch.as_tensor(v_cache)
+    B, Sq, Hq, d = q.shape
+    sl = np.asarray(seqlens, dtype=np.int64).reshape(-1)
+    O = torch.zeros(B, Sq, Hq, d, dtype=torch.float64)
+    LSE = torch.full((B, Hq, Sq), float("-inf"), dtype=torch.float64)
+    for b in range(B):
+        n = int(sl[b])
+        if n == 0:
+            continue
+        lo = max(0, Sq - n)                  # queries before position 0 see nothing
+        Ob, Lb = attention_full(q[b:b + 1, lo:].contiguous(), k[b:b + 1, :n].contiguous(), v[b:b + 1, :n].contiguous(),
+                                True, scale, nthreads)
+        O[b, lo:] = Ob[0]
+        LSE[b, :, lo:] = Lb[0]
+    return O, LSE
+
+
 def e4m3_to_float64(bits):
     """Value of FP8 e4m3 bit patterns (1 sign, 4 exponent, 3 mantissa bits, exponent bias 7, no
     infinities; exponent 15 with mantissa 7 is NaN), written out from the format's definition.

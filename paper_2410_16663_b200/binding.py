@@ -47,6 +47,10 @@ lib.fa_decode_workspace_bytes.restype = _sz
 lib.fa_decode_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
 lib.fa_forward_varlen.restype = _i
 lib.fa_forward_varlen.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p]
+lib.fa_decode_append.restype = _i
+lib.fa_decode_append.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
+lib.fa_decode_append_workspace_bytes.restype = _sz
+lib.fa_decode_append_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 lib.fa_decode_fp8.restype = _i
 lib.fa_decode_fp8.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
 lib.fa_decode_fp8_paged.restype = _i
@@ -69,7 +73,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -164,6 +168,21 @@ def fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace,
     rc = lib.fa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq,
                        Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode", raise_on_error)
+
+
+def fa_decode_append_workspace_bytes(B: int, Sq: int, Hq: int, Hkv: int, Skv_max: int, d: int) -> int:
+    return int(lib.fa_decode_append_workspace_bytes(B, Sq, Hq, Hkv, Skv_max, d))
+
+
+def fa_decode_append(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace, raise_on_error: bool = True) -> int:
+    """``fa_decode_append``: q, o [B,Sq,Hq,d] (the last Sq positions of every sequence), lse [B,Hq,Sq],
+    caches [B,Smax,Hkv,d], seqlens_k int32 [B] on the device (lengths including the Sq new tokens)."""
+    B, Sq, Hq, d = q.shape
+    _, Smax, Hkv, _ = k_cache.shape
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_append(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Sq, Hq,
+                              Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
+    return _check(rc, "fa_decode_append", raise_on_error)
 
 
 def fa_decode_fp8(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, k_scale: float, v_scale: float, workspace,

@@ -31,6 +31,7 @@ struct DecodeParams {
     const int* block_table;
     int page_size, table_stride;
     float v_scale;        // 8-bit cache only: factor of the stored values
+    int Sq;               // query rows per sequence (1; more for the append form of the fp16 kernel)
 };
 
 
@@ -65,7 +66,12 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
+// kMulti: Sq > 1 query rows per sequence, the last Sq positions of its cache (decoding after
+// several tokens were appended, Appendix C with more than one new token): the 16 MMA rows of a
+// CTA are then (token, head) pairs of one kv head, and query token t sees the keys up to
+// position len - Sq + t.  q is [B,Sq,Hq,128], the partials [B,Sq,Hq,NC,...].
+// grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
+template <bool kMulti>
 __global__ void __launch_bounds__(kDecMmaThreads, 1)
 fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
@@ -81,11 +87,19 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     const int c = blockIdx.x;
     const int b = blockIdx.z;
     const int g_all = p.Hq / p.Hkv;
-    const int n_sub = (g_all + 15) / 16;           // CTAs per kv head when more than 16 heads share it
+    const int Sq = kMulti ? p.Sq : 1;
+    const int rows_all = g_all * Sq;               // (token, head) rows that share a kv head
+    const int n_sub = (rows_all + 15) / 16;        // CTAs per kv head when there are more than 16
     const int hk = blockIdx.y / n_sub;
     const int sub = blockIdx.y % n_sub;
-    const int h0 = hk * g_all + sub * 16;          // first query head of this CTA
-    const int G = min(16, g_all - sub * 16);       // its number of query heads
+    const int G = min(16, rows_all - sub * 16);    // rows of this CTA
+    // row r of the CTA: token and head, and its row in q and in the partial results
+    auto row_token = [&](int r) { return kMulti ? (sub * 16 + r) / g_all : 0; };
+    auto row_index = [&](int r) -> long long {
+        const int R = sub * 16 + r;
+        const int hh = kMulti ? R % g_all : R;
+        return ((long long)b * Sq + row_token(r)) * p.Hq + hk * g_all + hh;
+    };
 
     int len = p.seqlens[b];
     len = max(0, min(len, p.Smax));
@@ -168,16 +182,20 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         // Q as A fragments for the eight k-steps of d = 128 (rows >= G are zero)
         uint32_t qa[8][4];
         {
-            const __half* qb = static_cast<const __half*>(p.q) + ((long long)b * p.Hq + h0) * 128;
+            const __half* q_lo = static_cast<const __half*>(p.q) + row_index(g) * 128;
+            const __half* q_hi = static_cast<const __half*>(p.q) + row_index(g + 8) * 128;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const int k0 = ks * 16 + 2 * t4;
-                qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0) : 0u;
-                qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0) : 0u;
-                qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(qb + g * 128 + k0 + 8) : 0u;
-                qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(qb + (g + 8) * 128 + k0 + 8) : 0u;
+                qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_lo + k0) : 0u;
+                qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q_hi + k0) : 0u;
+                qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_lo + k0 + 8) : 0u;
+                qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q_hi + k0 + 8) : 0u;
             }
         }
+        // keys an earlier query token must not see: the last Sq - 1 - t of the sequence
+        const int hide_lo = kMulti ? Sq - 1 - row_token(g) : 0;
+        const int hide_hi = kMulti ? Sq - 1 - row_token(min(g + 8, G - 1)) : 0;
         float o[16][4];
 #pragma unroll
         for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
@@ -211,12 +229,18 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     }
                 }
                 // ---- mask, running max, probabilities
+                // keys of this warp's 32 that the row may see: all valid ones, minus (several query
+                // rows) those among the sequence's last that came after the row's token
+                const int seen_lo = kMulti ? min(valid, len - hide_lo - (k_begin + t * kDecTile) - key_w) : valid;
+                const int seen_hi = kMulti ? min(valid, len - hide_hi - (k_begin + t * kDecTile) - key_w) : valid;
                 float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
                 for (int nb = 0; nb < 4; ++nb) {
                     const int k0 = nb * 8 + 2 * t4;
-                    if (k0 >= valid) sc[nb][0] = sc[nb][2] = -INFINITY;
-                    if (k0 + 1 >= valid) sc[nb][1] = sc[nb][3] = -INFINITY;
+                    if (k0 >= seen_lo) sc[nb][0] = -INFINITY;
+                    if (k0 + 1 >= seen_lo) sc[nb][1] = -INFINITY;
+                    if (k0 >= seen_hi) sc[nb][2] = -INFINITY;
+                    if (k0 + 1 >= seen_hi) sc[nb][3] = -INFINITY;
                     mx_lo = fmaxf(mx_lo, fmaxf(sc[nb][0], sc[nb][1]));
                     mx_hi = fmaxf(mx_hi, fmaxf(sc[nb][2], sc[nb][3]));
                 }
@@ -224,20 +248,23 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
                 mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
                 mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);  // finite: key 0 of the warp is valid
+                // finite when key 0 of the warp is visible (always with one query row; an earlier
+                // token of several may see none of the warp's keys: its state then stays empty)
+                const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
                 const float a_lo = (m_lo == -INFINITY) ? 0.f : fast_exp2((m_lo - mn_lo) * p.scale_log2);
                 const float a_hi = (m_hi == -INFINITY) ? 0.f : fast_exp2((m_hi - mn_hi) * p.scale_log2);
                 m_lo = mn_lo;
                 m_hi = mn_hi;
-                const float nm_lo = -mn_lo * p.scale_log2, nm_hi = -mn_hi * p.scale_log2;
+                const float nm_lo = (mn_lo == -INFINITY) ? 0.f : -mn_lo * p.scale_log2;
+                const float nm_hi = (mn_hi == -INFINITY) ? 0.f : -mn_hi * p.scale_log2;
                 float s_lo = 0.f, s_hi = 0.f;
 #pragma unroll
                 for (int nb = 0; nb < 4; ++nb) {
                     const int k0 = nb * 8 + 2 * t4;
-                    sc[nb][0] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][0], p.scale_log2, nm_lo)) : 0.f;
-                    sc[nb][1] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][1], p.scale_log2, nm_lo)) : 0.f;
-                    sc[nb][2] = (k0 < valid) ? fast_exp2(fmaf(sc[nb][2], p.scale_log2, nm_hi)) : 0.f;
-                    sc[nb][3] = (k0 + 1 < valid) ? fast_exp2(fmaf(sc[nb][3], p.scale_log2, nm_hi)) : 0.f;
+                    sc[nb][0] = (k0 < seen_lo) ? fast_exp2(fmaf(sc[nb][0], p.scale_log2, nm_lo)) : 0.f;
+                    sc[nb][1] = (k0 + 1 < seen_lo) ? fast_exp2(fmaf(sc[nb][1], p.scale_log2, nm_lo)) : 0.f;
+                    sc[nb][2] = (k0 < seen_hi) ? fast_exp2(fmaf(sc[nb][2], p.scale_log2, nm_hi)) : 0.f;
+                    sc[nb][3] = (k0 + 1 < seen_hi) ? fast_exp2(fmaf(sc[nb][3], p.scale_log2, nm_hi)) : 0.f;
                     s_lo += sc[nb][0] + sc[nb][1];
                     s_hi += sc[nb][2] + sc[nb][3];
                 }
@@ -333,9 +360,10 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     l += sw * ml[(w * 16 + r) * 2 + 1];
                     acc += sw * mo[(w * 16 + r) * 128 + tid];
                 }
-                const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;
-                p.o_part[slot * 128 + tid] = acc / l;
-                if (tid == 0) p.lse_part[slot] = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
+                const long long slot = row_index(r) * p.n_chunks + c;
+                // (l == 0: a query token that sees none of this chunk's keys)
+                p.o_part[slot * 128 + tid] = (l > 0.f) ? acc / l : 0.f;
+                if (tid == 0) p.lse_part[slot] = (l > 0.f) ? (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
             }
         }
     }
@@ -343,25 +371,27 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
 // Merge of the per-chunk partials (rowmax/rowsum recurrence applied across chunks):
 //   M = max_c LSE_c, w_c = exp(LSE_c - M), O = sum_c w_c O_c / sum_c w_c, LSE = M + ln sum_c w_c.
-// grid: B * Hq blocks of 128 threads, thread t owns output dim t.
+// grid: B * Sq * Hq blocks of 128 threads (row = (b, token, head)), thread t owns output dim t.
 template <typename T>
 __global__ void __launch_bounds__(128)
 fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
     const int bh = blockIdx.x;
-    const int b = bh / p.Hq;
+    const int b = bh / (p.Hq * p.Sq);
+    // lse is [B,Hq,Sq]
+    const long long lse_at = ((long long)b * p.Hq + bh % p.Hq) * p.Sq + (bh / p.Hq) % p.Sq;
     const int tid = threadIdx.x;
     int len = p.seqlens[b];
     len = max(0, min(len, p.Smax));
     const int nc = (len + p.chunk - 1) / p.chunk;
     const float* lp = p.lse_part + (long long)bh * p.n_chunks;
     const float* op = p.o_part + (long long)bh * p.n_chunks * 128;
-    if (nc == 0) {
-        o[(long long)bh * 128 + tid] = T(0.f);
-        if (lse && tid == 0) lse[bh] = -INFINITY;
-        return;
-    }
     float M = -INFINITY;
     for (int c = 0; c < nc; ++c) M = fmaxf(M, lp[c]);
+    if (nc == 0 || M == -INFINITY) {   // no keys, or (several query rows) a token that sees none
+        o[(long long)bh * 128 + tid] = T(0.f);
+        if (lse && tid == 0) lse[lse_at] = -INFINITY;
+        return;
+    }
     float wsum = 0.f, acc = 0.f;
     for (int c = 0; c < nc; ++c) {
         const float w = __expf(lp[c] - M);
@@ -369,7 +399,7 @@ fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
         acc = fmaf(w, op[(long long)c * 128 + tid], acc);
     }
     o[(long long)bh * 128 + tid] = T(acc / wsum);
-    if (lse && tid == 0) lse[bh] = M + logf(wsum);
+    if (lse && tid == 0) lse[lse_at] = M + logf(wsum);
 }
 
 }  // namespace fa

@@ -427,6 +427,11 @@ size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {
     return (size_t)B * Hq * nc * (128 + 1) * sizeof(float);
 }
 
+size_t fa_decode_append_workspace_bytes(int B, int Sq, int Hq, int Hkv, int Skv_max, int d) {
+    if (Sq <= 0) return 0;
+    return (size_t)Sq * fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d);
+}
+
 }  // extern "C"
 
 namespace {
@@ -434,8 +439,9 @@ namespace {
 // or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
 int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
                 int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
-                void* stream, const int* block_table, int num_pages, int page_size, int table_stride) {
-    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
+                void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0 || Sq < 1) return FA_ERR_SHAPE;
+    if (Sq > 64 || Sq > Skv_max) return FA_ERR_UNSUPPORTED;   // several query rows are the LAST rows of the cache
     if (Hq % Hkv) return FA_ERR_SHAPE;
     if (d != 128) return FA_ERR_UNSUPPORTED;
     if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
@@ -445,7 +451,7 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     if (Skv_max > 0 && (!k_cache || !v_cache)) return FA_ERR_NULL;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(workspace))
         return FA_ERR_ALIGN;
-    const size_t need = fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d);
+    const size_t need = fa_decode_append_workspace_bytes(B, Sq, Hq, Hkv, Skv_max, d);
     if (need > 0 && (!workspace || workspace_bytes < need)) return FA_ERR_WORKSPACE;
     int rc = check_device();
     if (rc) return rc;
@@ -455,10 +461,11 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.q = q;
     dp.seqlens = seqlens_k;
     dp.B = B; dp.Hq = Hq; dp.Hkv = Hkv; dp.Smax = Skv_max;
+    dp.Sq = Sq;
     dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max) : 256;
     dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
     dp.o_part = static_cast<float*>(workspace);
-    dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
+    dp.lse_part = dp.o_part + (size_t)B * Sq * Hq * dp.n_chunks * 128;
     dp.scale_log2 = scale * 1.4426950408889634f;
     dp.block_table = block_table;
     dp.page_size = block_table ? page_size : 1;
@@ -480,15 +487,16 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
         int sm_count = 0;
-        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(fa::fa_decode_split_mma_kernel), smem, &sm_count))
+        auto kern = (Sq > 1) ? fa::fa_decode_split_mma_kernel<true> : fa::fa_decode_split_mma_kernel<false>;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
-        dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
-        fa::fa_decode_split_mma_kernel<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
+        dim3 grid(dp.n_chunks, Hkv * ((g * Sq + 15) / 16), B);   // 16 (token, head) rows per CTA
+        kern<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
     }
-    fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    fa::fa_decode_combine_kernel<__half><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
@@ -538,6 +546,7 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     dp.page_size = block_table ? page_size : 1;
     dp.table_stride = table_stride;
     dp.v_scale = v_scale;
+    dp.Sq = 1;
     const int g = Hq / Hkv;
     if (Skv_max > 0) {
         CUtensorMap tk, tv;
@@ -563,6 +572,13 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+int fa_decode_append(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                     const int* seqlens_k, int B, int Sq, int Hq, int Hkv, int Skv_max, int d, float scale,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_impl(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, workspace,
+                       workspace_bytes, stream, nullptr, 0, 0, 0, Sq);
 }
 
 int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,

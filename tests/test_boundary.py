@@ -130,6 +130,24 @@ def test_varlen_validation(fa):
     assert call(max_q=0) == fa.FA_OK
 
 
+def test_decode_append_validation(fa):
+    L = fa.lib
+    q, kc, o = _t(2, 4, 8, 128), _t(2, 256, 2, 128), _t(2, 4, 8, 128)
+    sl = torch.zeros(2, dtype=torch.int32)
+    ws = torch.zeros(1 << 18, dtype=torch.uint8)
+    P = lambda t: t.data_ptr()
+    need = fa.fa_decode_append_workspace_bytes(2, 4, 8, 2, 256, 128)
+    assert need == 4 * fa.fa_decode_workspace_bytes(2, 8, 2, 256, 128)
+    call = lambda **kw: L.fa_decode_append(P(q), P(kc), P(kc), P(o), None, P(sl), kw.get("B", 2), kw.get("Sq", 4), 8,
+                                           kw.get("Hkv", 2), kw.get("Smax", 256), 128, 0.1, P(ws), kw.get("wbytes", need), None)
+    assert call(Sq=0) == fa.FA_ERR_SHAPE
+    assert call(Sq=65) == fa.FA_ERR_UNSUPPORTED
+    assert call(Sq=4, Smax=3) == fa.FA_ERR_UNSUPPORTED
+    assert call(Hkv=3) == fa.FA_ERR_SHAPE
+    assert call(wbytes=need - 1) == fa.FA_ERR_WORKSPACE
+    assert call(B=0) == fa.FA_OK
+
+
 def test_fp8_decode_validation(fa):
     L = fa.lib
     q, o = _t(2, 1, 8, 128), _t(2, 1, 8, 128)

@@ -324,6 +324,28 @@ def test_varlen_attention_is_attention_of_each_sequence_alone():
         oracle.attention_varlen(qp, kp, vp, cq[:-1], ck[:-1], False, 0.3)   # sums do not reach the end
 
 
+def test_decode_append_is_one_decode_per_new_token_on_the_cache_as_it_stood_then():
+    # query t of the last Sq positions must come out as plain decode over the cache truncated
+    # to what existed when that token was appended; with Sq = 1 it is decode itself; a sequence
+    # shorter than Sq leaves its first queries without keys
+    B, Sq, Hq, Hkv, Smax, d = 3, 4, 4, 2, 12, 4
+    q, k, v = rnd((B, Sq, Hq, d), 80), rnd((B, Smax, Hkv, d), 81), rnd((B, Smax, Hkv, d), 82)
+    seqlens = [12, 5, 2]
+    kp, vp = k.clone(), v.clone()
+    for b, n in enumerate(seqlens):
+        kp[b, n:] = float("nan")
+        vp[b, n:] = float("nan")
+    O, LSE = oracle.decode_append(q, kp, vp, seqlens, 0.4)
+    for t in range(Sq):
+        then = [max(0, n - (Sq - 1 - t)) for n in seqlens]
+        Ot, Lt = oracle.decode(q[:, t:t + 1].contiguous(), k, v, then, 0.4)
+        assert torch.equal(O[:, t], Ot) and torch.equal(LSE[:, :, t], Lt)
+    assert float(O[2, :2].abs().max()) == 0.0 and torch.isneginf(LSE[2, :, :2]).all()   # 2 keys, 4 queries
+    O1, L1 = oracle.decode_append(q[:, 3:4].contiguous(), kp, vp, seqlens, 0.4)
+    Od, Ld = oracle.decode(q[:, 3:4].contiguous(), kp, vp, seqlens, 0.4)
+    assert torch.equal(O1[:, 0], Od) and torch.equal(L1[:, :, 0], Ld)
+
+
 def test_e4m3_values_and_fp8_decode():
     # the format's landmarks: 0x38 = 1, 0x40 = 2, 0x01 = 2^-9 (smallest subnormal), 0x08 = 2^-6
     # (smallest normal), 0x7e = 448 (largest), 0x7f / 0xff = NaN, sign bit; and all 256 patterns

@@ -511,6 +511,65 @@ def test_c5_decode_full_size_sampled(fa, cfg):
                                    what=f"{cfg.name} b{b} h{h} n{n}")
 
 
+# ------------------------------------------------------------------ decode after several appended tokens
+def run_decode_append(fa, q, k, v, seqlens_dev, scale):
+    B, Sq, Hq, d = q.shape
+    Smax, Hkv = k.shape[1], k.shape[2]
+    o, chk_o = guard_alloc((B, Sq, Hq, d), torch.float16, DEV)
+    lse, chk_l = guard_alloc((B, Hq, Sq), torch.float32, DEV)
+    nbytes = fa.fa_decode_append_workspace_bytes(B, Sq, Hq, Hkv, Smax, d)
+    ws, chk_w = guard_alloc((max(nbytes // 4, 4),), torch.float32, DEV)
+    fa.fa_decode_append(q, k, v, o, lse, seqlens_dev, scale, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    return o, lse
+
+
+@pytest.mark.parametrize("sq,hq,hkv", [(2, 4, 4), (4, 8, 2), (5, 8, 1), (8, 8, 8), (16, 4, 1), (17, 6, 2), (3, 40, 2), (64, 2, 1)])
+def test_decode_append_small_full(fa, sq, hq, hkv):
+    # sq query rows = the last sq positions of each cache; lengths: long, exactly sq, shorter than
+    # sq (its first queries see nothing), sq + 1, around a tile and a chunk boundary; NaN past the end
+    cfg = synth.DecodeConfig("t", 7, hq, hkv, 3000, 1, 3000, seed=sq * 53 + hq + hkv)
+    _, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    sl[:] = torch.tensor([3000, sq, max(1, sq - 2), sq + 1, 129, 2049, 1500], dtype=torch.int32)
+    for b in range(cfg.B):
+        k[b, int(sl[b]):] = float("nan")
+        v[b, int(sl[b]):] = float("nan")
+    gen = torch.Generator().manual_seed(cfg.seed + 3)
+    q = torch.randn(cfg.B, sq, hq, 128, generator=gen).half()
+    o_ref, l_ref = oracle.decode_append(q, k, v, sl, cfg.scale)
+    o, lse = run_decode_append(fa, q.to(DEV), k.to(DEV), v.to(DEV), sl.to(DEV), cfg.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what=f"append decode sq{sq} {hq}/{hkv}")
+
+
+def test_decode_append_of_one_token_is_decode(fa):
+    cfg = synth.DecodeConfig("t", 4, 8, 2, 2500, 1, 2500, seed=977)
+    q, k, v, sl = synth.decode_inputs(cfg, DEV, poison=True)
+    o1, l1 = run_decode(fa, q, k, v, sl.to(DEV), cfg.scale)
+    o2, l2 = run_decode_append(fa, q, k, v, sl.to(DEV), cfg.scale)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2.view(cfg.B, cfg.Hq))
+
+
+def test_decode_append_full_size_sampled(fa):
+    # four new tokens per sequence on the GQA decode configuration (64 sequences, up to 32K keys)
+    cfg = synth.C5_GQA
+    _, k, v, sl = synth.decode_inputs(cfg, DEV, poison=True)
+    gen = torch.Generator(device=DEV).manual_seed(cfg.seed + 9)
+    q = torch.randn(cfg.B, 4, cfg.Hq, cfg.d, generator=gen, device=DEV).half()
+    o, lse = run_decode_append(fa, q, k, v, sl.to(DEV), cfg.scale)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    g = cfg.Hq // cfg.Hkv
+    order = torch.argsort(sl)
+    for b in sorted({int(order[0]), int(order[-1]), 0, 17, cfg.B - 1}):
+        n = int(sl[b])
+        for h in (0, g - 1, cfg.Hq - 1):
+            hk = h // g
+            o_ref, l_ref = oracle.decode_append(q[b:b + 1, :, h:h + 1].cpu(), k[b:b + 1, :n, hk:hk + 1].contiguous().cpu(),
+                                                v[b:b + 1, :n, hk:hk + 1].contiguous().cpu(), [n], cfg.scale)
+            assert_close_to_oracle(o[b:b + 1, :, h:h + 1], lse[b:b + 1, h:h + 1], o_ref, l_ref, what=f"append b{b} h{h} n{n}")
+
+
 # ------------------------------------------------------------------ decode over an FP8 cache
 def run_decode_fp8(fa, q, k8, v8, seqlens_dev, scale, k_scale, v_scale):
     B, _, Hq, d = q.shape
