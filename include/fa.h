@@ -142,6 +142,31 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * The general form of the 16-bit decode: fp16 or bf16 (q, caches and o share the type), one or
+ * several query rows per sequence (Sq <= 0 means 1; see fa_decode_append), contiguous cache
+ * (block_table == NULL: k, v [B,Skv_max,Hkv,d]) or paged (k, v [num_pages,page_size,Hkv,d];
+ * Skv_max is then ignored and max_pages * page_size takes its place; see fa_decode_paged).
+ * workspace: fa_decode_append_workspace_bytes(B, Sq, Hq, Hkv, Skv_max or max_pages * page_size, d).
+ * Everything else as documented for fa_decode, fa_decode_append and fa_decode_paged.
+ */
+typedef struct fa_decode_params {
+    const void* q;          /* [B,Sq,Hq,d] */
+    const void* k;          /* cache or page pool */
+    const void* v;
+    void* o;                /* [B,Sq,Hq,d] */
+    float* lse;             /* [B,Hq,Sq] or NULL */
+    const int* seqlens_k;   /* [B], device */
+    const int* block_table; /* NULL, or [B,table_stride] on the device */
+    int B, Sq, Hq, Hkv, Skv_max, d;
+    int dtype;              /* FA_DTYPE_FP16 or FA_DTYPE_BF16 */
+    int num_pages, page_size, max_pages, table_stride;
+    float scale;
+    void* workspace;
+    size_t workspace_bytes;
+} fa_decode_params;
+int fa_decode_ex(const fa_decode_params* p, void* stream);
+
+/*
  * Decode after several tokens were appended (Appendix C with Sq > 1 new tokens per sequence, as
  * in chunked or speculative decoding): the Sq query rows of sequence b are the LAST Sq positions
  * of its cache, so query t (0 <= t < Sq) sees the keys 0 .. seqlens_k[b] - Sq + t -- the

@@ -47,6 +47,15 @@ lib.fa_decode_workspace_bytes.restype = _sz
 lib.fa_decode_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
 lib.fa_forward_varlen.restype = _i
 lib.fa_forward_varlen.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _p]
+class fa_decode_params(ctypes.Structure):
+    _fields_ = [("q", _p), ("k", _p), ("v", _p), ("o", _p), ("lse", _p), ("seqlens_k", _p), ("block_table", _p),
+                ("B", _i), ("Sq", _i), ("Hq", _i), ("Hkv", _i), ("Skv_max", _i), ("d", _i), ("dtype", _i),
+                ("num_pages", _i), ("page_size", _i), ("max_pages", _i), ("table_stride", _i), ("scale", _f),
+                ("workspace", _p), ("workspace_bytes", _sz)]
+
+
+lib.fa_decode_ex.restype = _i
+lib.fa_decode_ex.argtypes = [ctypes.POINTER(fa_decode_params), _p]
 lib.fa_decode_append.restype = _i
 lib.fa_decode_append.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_append_workspace_bytes.restype = _sz
@@ -73,7 +82,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -168,6 +177,29 @@ def fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace,
     rc = lib.fa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq,
                        Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode", raise_on_error)
+
+
+def fa_decode_ex(q, k, v, o, lse, seqlens_k, scale: float, workspace, block_table=None, max_pages: int = None,
+                 raise_on_error: bool = True) -> int:
+    """``fa_decode_ex``: fp16 or bf16 (from q's dtype); q, o [B,Sq,Hq,d]; k, v the caches [B,Smax,Hkv,d] or, with a
+    block table, the page pools [num_pages,page_size,Hkv,d]."""
+    p = fa_decode_params()
+    p.q, p.k, p.v, p.o, p.lse = _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse)
+    p.seqlens_k, p.block_table = _ptr(seqlens_k), _ptr(block_table)
+    p.B, p.Sq, p.Hq, p.d = q.shape
+    p.Hkv = k.shape[2]
+    p.dtype = FA_DTYPE_BF16 if q.dtype == torch.bfloat16 else FA_DTYPE_FP16
+    if block_table is None:
+        p.Skv_max = k.shape[1]
+    else:
+        p.num_pages, p.page_size = k.shape[0], k.shape[1]
+        p.max_pages = block_table.shape[1] if max_pages is None else int(max_pages)
+        p.table_stride = block_table.stride(0)
+    p.scale = float(scale)
+    p.workspace = _ptr(workspace)
+    p.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_ex(ctypes.byref(p), _stream())
+    return _check(rc, "fa_decode_ex", raise_on_error)
 
 
 def fa_decode_append_workspace_bytes(B: int, Sq: int, Hq: int, Hkv: int, Skv_max: int, d: int) -> int:

@@ -6,6 +6,8 @@
 // exactly once and nothing but the partials is written.
 #pragma once
 
+#include <type_traits>
+
 #include "sm100_ptx.cuh"
 
 namespace fa {
@@ -58,6 +60,13 @@ __device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t& r0, uint3
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                  : "r"(addr));
 }
+__device__ __forceinline__ void mma_16816_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
@@ -71,7 +80,8 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // CTA are then (token, head) pairs of one kv head, and query token t sees the keys up to
 // position len - Sq + t.  q is [B,Sq,Hq,128], the partials [B,Sq,Hq,NC,...].
 // grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
-template <bool kMulti>
+// T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
+template <bool kMulti, typename T = __half>
 __global__ void __launch_bounds__(kDecMmaThreads, 1)
 fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
@@ -224,8 +234,13 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                         const uint32_t addr = kt + (chunk >> 3) * kDecHalfBytes + key * 128 + (((chunk & 7) ^ (key & 7)) << 4);
                         uint32_t b0, b1, b2, b3;
                         ldsm_x4(addr, b0, b1, b2, b3);
-                        mma_16816(sc[nb], qa[2 * c4], b0, b1);
-                        mma_16816(sc[nb], qa[2 * c4 + 1], b2, b3);
+                        if (std::is_same<T, __nv_bfloat16>::value) {
+                            mma_16816_bf16(sc[nb], qa[2 * c4], b0, b1);
+                            mma_16816_bf16(sc[nb], qa[2 * c4 + 1], b2, b3);
+                        } else {
+                            mma_16816(sc[nb], qa[2 * c4], b0, b1);
+                            mma_16816(sc[nb], qa[2 * c4 + 1], b2, b3);
+                        }
                     }
                 }
                 // ---- mask, running max, probabilities
@@ -296,16 +311,10 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 #pragma unroll
                 for (int k2 = 0; k2 < 2; ++k2) {
                     uint32_t pa[4];
-                    {
-                        __half2 h0 = __floats2half2_rn(sc[2 * k2][0], sc[2 * k2][1]);
-                        __half2 h1 = __floats2half2_rn(sc[2 * k2][2], sc[2 * k2][3]);
-                        __half2 h2 = __floats2half2_rn(sc[2 * k2 + 1][0], sc[2 * k2 + 1][1]);
-                        __half2 h3 = __floats2half2_rn(sc[2 * k2 + 1][2], sc[2 * k2 + 1][3]);
-                        pa[0] = *reinterpret_cast<uint32_t*>(&h0);
-                        pa[1] = *reinterpret_cast<uint32_t*>(&h1);
-                        pa[2] = *reinterpret_cast<uint32_t*>(&h2);
-                        pa[3] = *reinterpret_cast<uint32_t*>(&h3);
-                    }
+                    pa[0] = pack2<T>(sc[2 * k2][0], sc[2 * k2][1]);
+                    pa[1] = pack2<T>(sc[2 * k2][2], sc[2 * k2][3]);
+                    pa[2] = pack2<T>(sc[2 * k2 + 1][0], sc[2 * k2 + 1][1]);
+                    pa[3] = pack2<T>(sc[2 * k2 + 1][2], sc[2 * k2 + 1][3]);
                     const int key = key_w + k2 * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
                     for (int n2 = 0; n2 < 8; ++n2) {  // two output blocks per ldmatrix.x4.trans
@@ -313,8 +322,13 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                         const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
                         uint32_t b0, b1, b2, b3;
                         ldsm_x4_trans(addr, b0, b1, b2, b3);
-                        mma_16816(o[2 * n2], pa, b0, b1);
-                        mma_16816(o[2 * n2 + 1], pa, b2, b3);
+                        if (std::is_same<T, __nv_bfloat16>::value) {
+                            mma_16816_bf16(o[2 * n2], pa, b0, b1);
+                            mma_16816_bf16(o[2 * n2 + 1], pa, b2, b3);
+                        } else {
+                            mma_16816(o[2 * n2], pa, b0, b1);
+                            mma_16816(o[2 * n2 + 1], pa, b2, b3);
+                        }
                     }
                 }
             }

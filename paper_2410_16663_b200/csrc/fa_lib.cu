@@ -439,7 +439,8 @@ namespace {
 // or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
 int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
                 int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
-                void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1) {
+                void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1,
+                bool bf16 = false) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0 || Sq < 1) return FA_ERR_SHAPE;
     if (Sq > 64 || Sq > Skv_max) return FA_ERR_UNSUPPORTED;   // several query rows are the LAST rows of the cache
     if (Hq % Hkv) return FA_ERR_SHAPE;
@@ -480,14 +481,16 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
         CUtensorMap tk, tv;
         const int box_rows = (block_table && page_size < fa::kDecTile) ? page_size : fa::kDecTile;
         rc = encode_map(&tk, k_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        box_rows, false);
+                        box_rows, bf16);
         if (rc) return rc;
         rc = encode_map(&tv, v_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        box_rows, false);
+                        box_rows, bf16);
         if (rc) return rc;
         constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
         int sm_count = 0;
-        auto kern = (Sq > 1) ? fa::fa_decode_split_mma_kernel<true> : fa::fa_decode_split_mma_kernel<false>;
+        auto kern = bf16 ? ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __nv_bfloat16>
+                                     : fa::fa_decode_split_mma_kernel<false, __nv_bfloat16>)
+                         : ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __half> : fa::fa_decode_split_mma_kernel<false, __half>);
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(dp.n_chunks, Hkv * ((g * Sq + 15) / 16), B);   // 16 (token, head) rows per CTA
@@ -496,7 +499,8 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
     }
-    fa::fa_decode_combine_kernel<__half><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
+    else fa::fa_decode_combine_kernel<__half><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
@@ -572,6 +576,24 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+int fa_decode_ex(const fa_decode_params* p, void* stream) {
+    if (!p) return FA_ERR_NULL;
+    if (p->dtype != FA_DTYPE_FP16 && p->dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    const int Sq = p->Sq > 0 ? p->Sq : 1;
+    if (p->block_table) {
+        if (p->num_pages < 0 || p->max_pages < 0 || !page_size_ok(p->page_size)) return FA_ERR_SHAPE;
+        if (p->table_stride < p->max_pages) return FA_ERR_SHAPE;
+        if ((long long)p->max_pages * p->page_size > 0x7fffffffll) return FA_ERR_SHAPE;
+        if (p->max_pages > 0 && p->num_pages == 0) return FA_ERR_SHAPE;
+        if (reinterpret_cast<uintptr_t>(p->block_table) & 3u) return FA_ERR_ALIGN;
+        return decode_impl(p->q, p->k, p->v, p->o, p->lse, p->seqlens_k, p->B, p->Hq, p->Hkv, p->max_pages * p->page_size,
+                           p->d, p->scale, p->workspace, p->workspace_bytes, stream, p->block_table, p->num_pages,
+                           p->page_size, p->table_stride, Sq, p->dtype == FA_DTYPE_BF16);
+    }
+    return decode_impl(p->q, p->k, p->v, p->o, p->lse, p->seqlens_k, p->B, p->Hq, p->Hkv, p->Skv_max, p->d, p->scale,
+                       p->workspace, p->workspace_bytes, stream, nullptr, 0, 0, 0, Sq, p->dtype == FA_DTYPE_BF16);
 }
 
 int fa_decode_append(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,

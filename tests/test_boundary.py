@@ -130,6 +130,32 @@ def test_varlen_validation(fa):
     assert call(max_q=0) == fa.FA_OK
 
 
+def test_decode_ex_validation(fa):
+    q, kc, o = _t(2, 1, 8, 128), _t(2, 256, 2, 128), _t(2, 1, 8, 128)
+    sl = torch.zeros(2, dtype=torch.int32)
+    table = torch.zeros(2, 2, dtype=torch.int32)
+    ws = torch.zeros(1 << 16, dtype=torch.uint8)
+    assert fa.lib.fa_decode_ex(None, None) == fa.FA_ERR_NULL
+
+    def call(**kw):
+        p = fa.fa_decode_params()
+        p.q, p.k, p.v, p.o, p.seqlens_k = q.data_ptr(), kc.data_ptr(), kc.data_ptr(), o.data_ptr(), sl.data_ptr()
+        p.B, p.Sq, p.Hq, p.Hkv, p.Skv_max, p.d = 2, 1, 8, 2, 256, 128
+        p.dtype, p.scale = fa.FA_DTYPE_FP16, 0.1
+        p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel()
+        for key, val in kw.items():
+            setattr(p, key, val)
+        return fa.lib.fa_decode_ex(ctypes.byref(p), None)
+
+    assert call(dtype=fa.FA_DTYPE_FP32) == fa.FA_ERR_UNSUPPORTED
+    assert call(Hkv=3) == fa.FA_ERR_SHAPE
+    assert call(Sq=65) == fa.FA_ERR_UNSUPPORTED
+    assert call(workspace_bytes=8) == fa.FA_ERR_WORKSPACE
+    assert call(block_table=table.data_ptr(), num_pages=4, page_size=48, max_pages=2, table_stride=2) == fa.FA_ERR_SHAPE
+    assert call(block_table=table.data_ptr(), num_pages=4, page_size=128, max_pages=2, table_stride=1) == fa.FA_ERR_SHAPE
+    assert call(B=0) == fa.FA_OK
+
+
 def test_decode_append_validation(fa):
     L = fa.lib
     q, kc, o = _t(2, 4, 8, 128), _t(2, 256, 2, 128), _t(2, 4, 8, 128)

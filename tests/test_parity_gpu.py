@@ -570,6 +570,41 @@ def test_decode_append_full_size_sampled(fa):
             assert_close_to_oracle(o[b:b + 1, :, h:h + 1], lse[b:b + 1, h:h + 1], o_ref, l_ref, what=f"append b{b} h{h} n{n}")
 
 
+# ------------------------------------------------------------------ the general decode entry, bf16
+@pytest.mark.parametrize("form", ["plain", "append", "paged", "paged-append"])
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+def test_decode_ex_both_types_all_forms(fa, form, dtype):
+    # fa_decode_ex: fp16 and bf16, one or five query rows per sequence, contiguous or paged cache.
+    # bf16 is gated like the bf16 prefill: 2e-3 plus the exact bounds of the bf16 probabilities
+    # and of the stored bf16 output, both computed from the oracle
+    sq = 5 if "append" in form else 1
+    cfg = synth.DecodeConfig("t", 5, 8, 2, 2600, 1, 2600, dtype=dtype, seed=1200 + sq)
+    _, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    sl[:] = torch.tensor([2600, 3, 129, 2049, 700], dtype=torch.int32)
+    gen = torch.Generator().manual_seed(cfg.seed + 1)
+    q = torch.randn(cfg.B, sq, cfg.Hq, 128, generator=gen).to(k.dtype)
+    o_ref, l_ref = oracle.decode_append(q, k, v, sl, cfg.scale)
+    absv = oracle.decode_append(q, k, v.abs(), sl, cfg.scale)[0] if dtype == "bf16" else None
+    o, chk_o = guard_alloc((cfg.B, sq, cfg.Hq, 128), k.dtype, DEV)
+    lse, chk_l = guard_alloc((cfg.B, cfg.Hq, sq), torch.float32, DEV)
+    if "paged" in form:
+        kd, vd, table = synth.paged_cache(k, v, sl, 128, seed=9, spare_pages=2, poison=True)
+        table = table.to(DEV)
+        smax = table.shape[1] * 128
+    else:
+        kd, vd, table, smax = k.clone(), v.clone(), None, cfg.Smax
+        for b in range(cfg.B):
+            kd[b, int(sl[b]):] = float("nan")
+            vd[b, int(sl[b]):] = float("nan")
+    ws, chk_w = guard_alloc((max(fa.fa_decode_append_workspace_bytes(cfg.B, sq, cfg.Hq, cfg.Hkv, smax, 128) // 4, 4),),
+                            torch.float32, DEV)
+    fa.fa_decode_ex(q.to(DEV), kd.to(DEV), vd.to(DEV), o, lse, sl.to(DEV), cfg.scale, ws, block_table=table)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=f"decode_ex {form} {dtype}")
+
+
 # ------------------------------------------------------------------ decode over an FP8 cache
 def run_decode_fp8(fa, q, k8, v8, seqlens_dev, scale, k_scale, v_scale):
     B, _, Hq, d = q.shape
