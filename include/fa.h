@@ -142,6 +142,25 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
 
 /*
+ * fa_forward_varlen over a paged K/V cache (chunked prefill of a batch of requests whose
+ * earlier keys already sit in a serving system's page pool): q, o, lse, cu_seqlens_q as for
+ * fa_forward_varlen; sequence b has seqlens_k[b] keys (int32 [B] on the DEVICE), key j in row
+ * j mod page_size of page block_table[b * table_stride + j / page_size] of the pools k_pages,
+ * v_pages [num_pages, page_size, Hkv, d]; page_size a positive multiple of 128; max_seqlen_k an
+ * upper bound of seqlens_k, at most max_pages * page_size.  The causal mask is aligned
+ * bottom-right per sequence (the queries are the sequence's LAST rows).  Only the table entries
+ * that cover keys [0, seqlens_k[b]) are read.  Rows of a page past the end of its sequence are
+ * multiplied by exact zeros: they must hold finite values (zeros, or stale keys and values).
+ * Errors: as fa_forward_varlen; FA_ERR_SHAPE also for a page_size that is not a multiple of 128,
+ * table_stride < max_pages or max_seqlen_k > max_pages * page_size.
+ */
+int fa_forward_varlen_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                            void* o, float* lse, const int* cu_seqlens_q, const int* seqlens_k, int B, int Hq,
+                            int Hkv, int total_q, int num_pages, int page_size, int max_pages, int table_stride,
+                            int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, int dtype,
+                            void* stream);
+
+/*
  * The general form of the 16-bit decode: fp16 or bf16 (q, caches and o share the type), one or
  * several query rows per sequence (Sq <= 0 means 1; see fa_decode_append), contiguous cache
  * (block_table == NULL: k, v [B,Skv_max,Hkv,d]) or paged (k, v [num_pages,page_size,Hkv,d];

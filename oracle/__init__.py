@@ -172,6 +172,30 @@ def attention_varlen(q, k, v, cu_seqlens_q, cu_seqlens_k, causal: bool, scale: f
     return O, LSE
 
 
+def attention_varlen_paged(q, k_pages, v_pages, block_table, cu_seqlens_q, seqlens_k, causal: bool, scale: float,
+                           nthreads: int = 0):
+    """``attention_varlen`` with the keys and values of every sequence read out of page pools
+    ``[num_pages, page_size, Hkv, d]``: key j of sequence b is row ``j % page_size`` of page
+    ``block_table[b][j // page_size]``.  The keys are first collected, position by position,
+    into packed tensors; the result is ``attention_varlen`` on those."""
+    k_pages = torch.as_tensor(k_pages)
+    v_pages = torch.as_tensor(v_pages)
+    table = np.asarray(block_table, dtype=np.int64)
+    sk = np.asarray(seqlens_k, dtype=np.int64).reshape(-1)
+    num_pages, page_size, Hkv, d = k_pages.shape
+    cu_k = np.concatenate([[0], np.cumsum(sk)])
+    k = torch.zeros(int(cu_k[-1]), Hkv, d, dtype=k_pages.dtype)
+    v = torch.zeros(int(cu_k[-1]), Hkv, d, dtype=v_pages.dtype)
+    for b in range(sk.shape[0]):
+        for j in range(int(sk[b])):
+            page = int(table[b, j // page_size])
+            if not 0 <= page < num_pages:
+                raise ValueError(f"sequence {b}: key {j} maps to page {page} outside the pool")
+            k[int(cu_k[b]) + j] = k_pages[page, j % page_size]
+            v[int(cu_k[b]) + j] = v_pages[page, j % page_size]
+    return attention_varlen(q, k, v, cu_seqlens_q, cu_k, causal, scale, nthreads)
+
+
 def decode(q, k_cache, v_cache, seqlens, scale: float, nthreads: int = 0):
     """Decode-stage attention: q ``[B,1,Hq,d]`` over the first ``seqlens[b]`` rows of
     the ``[B,Smax,Hkv,d]`` caches.  Returns ``(O [B,Hq,d], LSE [B,Hq])`` float64."""

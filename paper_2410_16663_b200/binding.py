@@ -64,6 +64,9 @@ lib.fa_decode_fp8.restype = _i
 lib.fa_decode_fp8.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
 lib.fa_decode_fp8_paged.restype = _i
 lib.fa_decode_fp8_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
+lib.fa_forward_varlen_paged.restype = _i
+lib.fa_forward_varlen_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f,
+                                        _i, _p]
 lib.fa_decode_paged.restype = _i
 lib.fa_decode_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_noalloc.restype = _i
@@ -82,7 +85,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -177,6 +180,21 @@ def fa_decode(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, workspace,
     rc = lib.fa_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq,
                        Hkv, Smax, d, float(scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode", raise_on_error)
+
+
+def fa_forward_varlen_paged(q, k_pages, v_pages, block_table, o, lse, cu_seqlens_q, seqlens_k, max_seqlen_q: int,
+                            max_seqlen_k: int, causal: bool, scale: float, raise_on_error: bool = True) -> int:
+    """``fa_forward_varlen_paged``: q, o [total_q,Hq,d] packed, K and V in page pools [num_pages,page_size,Hkv,d]
+    behind block_table int32 [B,stride]; cu_seqlens_q int32 [B+1] and seqlens_k int32 [B] on the device."""
+    total_q, Hq, d = q.shape
+    num_pages, page_size, Hkv, _ = k_pages.shape
+    B = cu_seqlens_q.numel() - 1
+    dt = FA_DTYPE_BF16 if q.dtype == torch.bfloat16 else FA_DTYPE_FP16
+    rc = lib.fa_forward_varlen_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(o), _ptr(lse),
+                                     _ptr(cu_seqlens_q), _ptr(seqlens_k), B, Hq, Hkv, total_q, num_pages, page_size,
+                                     block_table.shape[1], block_table.stride(0), int(max_seqlen_q), int(max_seqlen_k), d,
+                                     int(bool(causal)), float(scale), dt, _stream())
+    return _check(rc, "fa_forward_varlen_paged", raise_on_error)
 
 
 def fa_decode_ex(q, k, v, o, lse, seqlens_k, scale: float, workspace, block_table=None, max_pages: int = None,

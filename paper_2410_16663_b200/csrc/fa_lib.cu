@@ -198,6 +198,10 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.cu_q = nullptr;
     fp.cu_k = nullptr;
     fp.total_q = 0;
+    fp.block_table = nullptr;
+    fp.seqlens_k = nullptr;
+    fp.table_stride = 0;
+    fp.page_size = 1;
     fp.d = p.d;
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
@@ -349,13 +353,16 @@ int fa_forward_ex(const fa_params* p, void* stream) {
     return forward_impl(*p, static_cast<cudaStream_t>(stream));
 }
 
-int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens_q,
-                      const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q, int total_k, int max_seqlen_q,
-                      int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream) {
+// Packed batch; K and V packed too (block_table == nullptr: k, v [total_k,Hkv,128], cu_seqlens_k) or in
+// pages (k, v [num_pages,page_size,Hkv,128], seqlens_k and the block table; total_k = num_pages * page_size).
+static int varlen_impl(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens_q,
+                       const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q, int total_k, int max_seqlen_q,
+                       int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream,
+                       const int* block_table, int num_pages, int page_size, int table_stride) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || total_q < 0 || total_k < 0 || max_seqlen_q < 0 || max_seqlen_k < 0 || d <= 0)
         return FA_ERR_SHAPE;
     if (Hq % Hkv) return FA_ERR_SHAPE;
-    if (max_seqlen_q > total_q || max_seqlen_k > total_k) return FA_ERR_SHAPE;
+    if (max_seqlen_q > total_q || (!block_table && max_seqlen_k > total_k)) return FA_ERR_SHAPE;
     if (d != 128) return FA_ERR_UNSUPPORTED;
     if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
@@ -394,6 +401,10 @@ int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, floa
     fp.cu_k = cu_seqlens_k;
     fp.total_q = total_q;
     fp.d = 128;
+    fp.block_table = block_table;
+    fp.seqlens_k = block_table ? cu_seqlens_k : nullptr;   // per-sequence key counts in the paged form
+    fp.table_stride = table_stride;
+    fp.page_size = block_table ? page_size : 1;
 
     if (total_k == 0 || max_seqlen_k == 0) {
         // no keys anywhere: O = 0, LSE = -inf over the packed rows, seen as one sequence
@@ -410,14 +421,39 @@ int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, floa
     CUtensorMap tq, tk, tv, to;
     rc = encode_map(&tq, q, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 128, bf16);
     if (rc) return rc;
-    rc = encode_map(&tk, k, 1, total_k, Hkv, (int64_t)total_k * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    // K and V: one batch entry with every sequence back to back, or one entry per page
+    const int slabs = block_table ? num_pages : 1, slab_rows = block_table ? page_size : total_k;
+    rc = encode_map(&tk, k, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
     if (rc) return rc;
-    rc = encode_map(&tv, v, 1, total_k, Hkv, (int64_t)total_k * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    rc = encode_map(&tv, v, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
     if (rc) return rc;
     rc = encode_map(&to, o, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 32, bf16);
     if (rc) return rc;
     return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
                 : fa::launch_pingpong<__half>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
+}
+
+int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens_q,
+                      const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q, int total_k, int max_seqlen_q,
+                      int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream) {
+    return varlen_impl(q, k, v, o, lse, cu_seqlens_q, cu_seqlens_k, B, Hq, Hkv, total_q, total_k, max_seqlen_q,
+                       max_seqlen_k, d, causal, scale, dtype, stream, nullptr, 0, 0, 0);
+}
+
+int fa_forward_varlen_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+                            float* lse, const int* cu_seqlens_q, const int* seqlens_k, int B, int Hq, int Hkv,
+                            int total_q, int num_pages, int page_size, int max_pages, int table_stride,
+                            int max_seqlen_q, int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream) {
+    if (num_pages < 0 || max_pages < 0 || page_size <= 0 || page_size % fa::kTile) return FA_ERR_SHAPE;
+    if (table_stride < max_pages) return FA_ERR_SHAPE;
+    if ((long long)num_pages * page_size > 0x7fffffffll) return FA_ERR_SHAPE;
+    if (max_seqlen_k > (long long)max_pages * page_size) return FA_ERR_SHAPE;
+    if (B > 0 && max_pages > 0 && !block_table) return FA_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(block_table) & 3u) return FA_ERR_ALIGN;
+    if (num_pages == 0) max_seqlen_k = 0;
+    return varlen_impl(q, k_pages, v_pages, o, lse, cu_seqlens_q, seqlens_k, B, Hq, Hkv, total_q, num_pages * page_size,
+                       max_seqlen_q, max_seqlen_k, d, causal, scale, dtype, stream, block_table, num_pages, page_size,
+                       table_stride);
 }
 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {

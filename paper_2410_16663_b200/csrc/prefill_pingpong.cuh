@@ -113,9 +113,14 @@ __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
     it.q0 = qt * kTile;
     if (kVarlen) {
         it.q_base = p.cu_q[it.b];
-        it.k_base = p.cu_k[it.b];
         it.Sq = p.cu_q[it.b + 1] - it.q_base;
-        it.Skv = p.cu_k[it.b + 1] - it.k_base;
+        if (p.block_table) {   // paged K/V: the keys are reached through the table
+            it.k_base = 0;
+            it.Skv = p.seqlens_k[it.b];
+        } else {
+            it.k_base = p.cu_k[it.b];
+            it.Skv = p.cu_k[it.b + 1] - it.k_base;
+        }
         it.n = (it.q0 < it.Sq) ? max(1, kv_tiles_for(it.q0, kTile, it.Sq, it.Skv, p.causal)) : 0;
     } else {
         it.n = kv_tiles_for(it.q0, kTile, p.Sq, p.Skv, p.causal);
@@ -268,6 +273,18 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
     }
 }
 
+// Paged K/V (packed batches only): kv tile j of sequence b lies in one page; its coordinates
+// become (row inside the page, page).  The loaders run two to three steps ahead of the MMAs,
+// which covers the table read.
+template <bool kVarlen>
+__device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int b, int j, int& row, int& slab) {
+    if (kVarlen && p.block_table != nullptr) {
+        const int key0 = j * kTile;
+        slab = p.block_table[(long long)b * p.table_stride + key0 / p.page_size];
+        row = key0 % p.page_size;
+    }
+}
+
 // The thread that loads Q of every item and K of every step.  (Packed batches: the tensor maps
 // have one batch entry that holds every sequence back to back.)
 template <bool kVarlen>
@@ -291,8 +308,9 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
-            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk,
-                           kVarlen ? it.k_base + j * kTile : j * kTile, kVarlen ? 0 : it.b, pol_kv);
+            int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
+            pp_paged_tile<kVarlen>(p, it.b, j, row, slab);
+            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }
@@ -311,8 +329,9 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
         for (int j = 0; j < it.n; ++j, ring.next()) {
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
-            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk,
-                           kVarlen ? it.k_base + j * kTile : j * kTile, kVarlen ? 0 : it.b, pol_kv);
+            int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
+            pp_paged_tile<kVarlen>(p, it.b, j, row, slab);
+            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }

@@ -58,6 +58,12 @@ struct FwdParams {
     const int* cu_q;
     const int* cu_k;
     int total_q;
+    // packed batch over a paged K/V cache (block_table != nullptr; cu_k unused): sequence b has
+    // seqlens_k[b] keys, key j in row j % page_size of page block_table[b * table_stride + j / page_size];
+    // page_size is a multiple of the 128-key tile and the K/V tensor maps run over the pages
+    const int* block_table;
+    const int* seqlens_k;
+    int table_stride, page_size;
     int d;  // head dimension: 128, or 64 (its own kernel)
 };
 

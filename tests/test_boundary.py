@@ -195,6 +195,23 @@ def test_fp8_decode_validation(fa):
     assert call(B=0) == fa.FA_OK
 
 
+def test_varlen_paged_validation(fa):
+    L = fa.lib
+    q, pool, o = _t(20, 4, 128), _t(6, 128, 2, 128), _t(20, 4, 128)
+    cu = torch.zeros(3, dtype=torch.int32)
+    sk = torch.zeros(2, dtype=torch.int32)
+    table = torch.zeros(2, 3, dtype=torch.int32)
+    P = lambda t: t.data_ptr()
+    call = lambda **kw: L.fa_forward_varlen_paged(
+        P(q), P(pool), P(pool), kw.get("table", P(table)), P(o), None, P(cu), P(sk), kw.get("B", 2), 4, 2, 20, 6,
+        kw.get("page_size", 128), 3, kw.get("stride", 3), 12, kw.get("max_k", 300), 128, 1, 0.1, fa.FA_DTYPE_FP16, None)
+    assert call(page_size=64) == fa.FA_ERR_SHAPE
+    assert call(stride=2) == fa.FA_ERR_SHAPE
+    assert call(max_k=3 * 128 + 1) == fa.FA_ERR_SHAPE
+    assert call(table=None) == fa.FA_ERR_NULL
+    assert call(B=0) == fa.FA_OK
+
+
 def test_paged_decode_validation(fa):
     L = fa.lib
     q, pool, o = _t(2, 1, 8, 128), _t(6, 128, 2, 128), _t(2, 1, 8, 128)

@@ -378,6 +378,30 @@ def test_e4m3_values_and_fp8_decode():
     assert torch.allclose(O3, O, rtol=1e-12, atol=1e-14) and torch.allclose(L3, LSE, rtol=1e-12, atol=1e-14)
 
 
+def test_paged_packed_batch_equals_the_packed_batch_on_the_same_keys():
+    # pools filled by hand, page by page in a scrambled order; NaN wherever no key lives
+    Hq, Hkv, d, ps = 4, 2, 4, 4
+    lens_q, lens_k = [3, 2, 5], [9, 2, 5]
+    cq, ck = np.concatenate([[0], np.cumsum(lens_q)]), np.concatenate([[0], np.cumsum(lens_k)])
+    q, k, v = rnd((int(cq[-1]), Hq, d), 90), rnd((int(ck[-1]), Hkv, d), 91), rnd((int(ck[-1]), Hkv, d), 92)
+    order = [4, 0, 6, 2, 5, 1, 3]
+    kp = torch.full((7, ps, Hkv, d), float("nan"), dtype=k.dtype)
+    vp = torch.full((7, ps, Hkv, d), float("nan"), dtype=v.dtype)
+    table = -np.ones((3, 3), dtype=np.int32)
+    nxt = 0
+    for b, n in enumerate(lens_k):
+        for p_ in range((n + ps - 1) // ps):
+            slot = order[nxt]; nxt += 1
+            table[b, p_] = slot
+            for r in range(min(ps, n - p_ * ps)):
+                kp[slot, r] = k[int(ck[b]) + p_ * ps + r]
+                vp[slot, r] = v[int(ck[b]) + p_ * ps + r]
+    for causal in (False, True):
+        O1, L1 = oracle.attention_varlen(q, k, v, cq, ck, causal, 0.3)
+        O2, L2 = oracle.attention_varlen_paged(q, kp, vp, table, cq, lens_k, causal, 0.3)
+        assert torch.equal(O1, O2) and torch.equal(L1, L2)
+
+
 def test_paged_decode_equals_decode_on_the_same_keys_wherever_the_pages_lie():
     # the paged form only changes where a key is stored: build the pools by hand (page p of
     # sequence b at a chosen pool slot), compare with decode on the contiguous caches, then move

@@ -433,6 +433,45 @@ def test_varlen_equal_lengths_match_the_batched_call_bit_for_bit(fa):
     assert torch.equal(l1, l2.view(c.Hq, c.B, c.Sq).permute(1, 0, 2))
 
 
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_varlen_over_a_paged_cache(fa, causal, dtype):
+    # chunked prefill against a page pool: each sequence's queries are its last rows, its keys sit
+    # in 128- or 256-key pages handed out in random order; unused pages hold NaN (a wrong page
+    # would show), the unused rows of a last page zeros (the contract: finite).  Lengths: a key
+    # count that ends exactly on a page, one key, more pages than queries, queries = keys
+    lq = (70, 1, 130, 300, 128, 5)
+    lk = (700, 1, 130, 1000, 256, 1500)
+    for page in (128, 256):
+        cfg = synth.VarlenConfig("t", 4, 2, lq, lk, dtype=dtype, causal=causal, seed=700 + page)
+        q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
+        B = len(lq)
+        kc = torch.zeros(B, max(lk), cfg.Hkv, 128, dtype=k.dtype); vc = torch.zeros_like(kc)
+        for b in range(B):
+            kc[b, :lk[b]] = k[int(cu_k[b]):int(cu_k[b + 1])]
+            vc[b, :lk[b]] = v[int(cu_k[b]):int(cu_k[b + 1])]
+        sk = torch.tensor(lk, dtype=torch.int32)
+        kp, vp, table = synth.paged_cache(kc, vc, sk, page, seed=cfg.seed, spare_pages=3, poison=True)
+        for b in range(B):      # the rows of a sequence's last page past its end: finite
+            last = (lk[b] - 1) // page
+            kp[int(table[b, last]), lk[b] - last * page:] = 0
+            vp[int(table[b, last]), lk[b] - last * page:] = 0
+        o_ref, l_ref = oracle.attention_varlen_paged(q, kp, vp, table, cu_q, sk, causal, cfg.scale)
+        o_chk, l_chk = oracle.attention_varlen(q, k, v, cu_q, cu_k, causal, cfg.scale)
+        assert torch.equal(o_ref, o_chk) and torch.equal(l_ref, l_chk)
+        absv = oracle.attention_varlen(q, k, v.abs(), cu_q, cu_k, causal, cfg.scale)[0] if dtype == "bf16" else None
+        o, chk_o = guard_alloc(tuple(q.shape), q.dtype, DEV)
+        lse, chk_l = guard_alloc((cfg.Hq, q.shape[0]), torch.float32, DEV)
+        fa.fa_forward_varlen_paged(q.to(DEV), kp.to(DEV), vp.to(DEV), table.to(DEV), o, lse, cu_q.to(DEV), sk.to(DEV),
+                                   max(lq), max(lk), causal, cfg.scale)
+        torch.cuda.synchronize()
+        check_status(fa)
+        chk_o(); chk_l()
+        assert_close_to_oracle(o.unsqueeze(0), lse.unsqueeze(0), o_ref.unsqueeze(0), l_ref.unsqueeze(0),
+                               stored_bf16=(dtype == "bf16"), p_absv=None if absv is None else absv.unsqueeze(0),
+                               what=f"varlen paged page{page} causal{int(causal)} {dtype}")
+
+
 def test_varlen_without_any_keys(fa):
     cfg = synth.VarlenConfig("t", 2, 2, (5, 130), (0, 0), dtype="fp16", causal=False, seed=612)
     q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, DEV)
