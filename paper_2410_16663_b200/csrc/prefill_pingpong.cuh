@@ -274,14 +274,25 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
 }
 
 // Paged K/V (packed batches only): kv tile j of sequence b lies in one page; its coordinates
-// become (row inside the page, page).  The loaders run two to three steps ahead of the MMAs,
-// which covers the table read.
+// become (row inside the page, page).  The page of tile j + 1 is looked up before the loader
+// waits for tile j's ring slot, so that the table read is off the path that refills a slot.
 template <bool kVarlen>
-__device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int b, int j, int& row, int& slab) {
+__device__ __forceinline__ int pp_page_of(const FwdParams& p, int b, int j, int n) {
+    if (kVarlen && p.block_table != nullptr && j < n) {
+        // (volatile: issued here, ahead of the wait that follows, not where the value is used)
+        int page;
+        asm volatile("ld.global.nc.s32 %0, [%1];"
+                     : "=r"(page)
+                     : "l"(p.block_table + (long long)b * p.table_stride + (j * kTile) / p.page_size));
+        return page;
+    }
+    return 0;
+}
+template <bool kVarlen>
+__device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int page, int j, int& row, int& slab) {
     if (kVarlen && p.block_table != nullptr) {
-        const int key0 = j * kTile;
-        slab = p.block_table[(long long)b * p.table_stride + key0 / p.page_size];
-        row = key0 % p.page_size;
+        slab = page;
+        row = (j * kTile) % p.page_size;
     }
 }
 
@@ -305,11 +316,14 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
         load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
                        kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
+        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n);
         for (int j = 0; j < it.n; ++j, ring.next()) {
+            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n);
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
-            pp_paged_tile<kVarlen>(p, it.b, j, row, slab);
+            pp_paged_tile<kVarlen>(p, page, j, row, slab);
+            page = page_next;
             load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
@@ -326,11 +340,14 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
     while (items.next(p, total_items)) {
         const int ord = items.ord;
         const PpItem& it = items.it;
+        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n);
         for (int j = 0; j < it.n; ++j, ring.next()) {
+            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n);
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
-            pp_paged_tile<kVarlen>(p, it.b, j, row, slab);
+            pp_paged_tile<kVarlen>(p, page, j, row, slab);
+            page = page_next;
             load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
