@@ -34,6 +34,10 @@ struct DecodeParams {
     int page_size, table_stride;
     float v_scale;        // 8-bit cache only: factor of the stored values
     int Sq;               // query rows per sequence (1; more for the append form of the fp16 kernel)
+    // fp16/bf16 kernel with a single chunk per sequence (n_chunks == 1): the split kernel writes
+    // the result itself and no merge kernel runs (nullptr otherwise)
+    void* o_final;
+    float* lse_final;
 };
 
 
@@ -115,7 +119,19 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     len = max(0, min(len, p.Smax));
     const int k_begin = c * p.chunk;
     const int k_end = min(len, k_begin + p.chunk);
-    if (k_begin >= k_end) return;  // uniform for the CTA
+    auto lse_index = [&](int r) -> long long {   // lse is [B,Hq,Sq]
+        const int R = sub * 16 + r;
+        return ((long long)b * p.Hq + hk * g_all + (kMulti ? R % g_all : R)) * Sq + row_token(r);
+    };
+    if (k_begin >= k_end) {  // uniform for the CTA
+        if (p.o_final != nullptr && tid < 128) {   // a sequence without keys, and nobody else writes its rows
+            for (int r = 0; r < G; ++r) {
+                static_cast<T*>(p.o_final)[row_index(r) * 128 + tid] = T(0.f);
+                if (tid == 0 && p.lse_final) p.lse_final[lse_index(r)] = -INFINITY;
+            }
+        }
+        return;
+    }
     const int n_tiles = (k_end - k_begin + kDecTile - 1) / kDecTile;
 
     if (tid == 0) {
@@ -374,10 +390,17 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     l += sw * ml[(w * 16 + r) * 2 + 1];
                     acc += sw * mo[(w * 16 + r) * 128 + tid];
                 }
-                const long long slot = row_index(r) * p.n_chunks + c;
                 // (l == 0: a query token that sees none of this chunk's keys)
-                p.o_part[slot * 128 + tid] = (l > 0.f) ? acc / l : 0.f;
-                if (tid == 0) p.lse_part[slot] = (l > 0.f) ? (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                const float out = (l > 0.f) ? acc / l : 0.f;
+                const float lse = (l > 0.f) ? (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                if (p.o_final != nullptr) {   // the only chunk: this is the result
+                    static_cast<T*>(p.o_final)[row_index(r) * 128 + tid] = T(out);
+                    if (tid == 0 && p.lse_final) p.lse_final[lse_index(r)] = lse;
+                } else {
+                    const long long slot = row_index(r) * p.n_chunks + c;
+                    p.o_part[slot * 128 + tid] = out;
+                    if (tid == 0) p.lse_part[slot] = lse;
+                }
             }
         }
     }

@@ -508,6 +508,10 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.page_size = block_table ? page_size : 1;
     dp.table_stride = table_stride;
     dp.v_scale = 1.f;
+    // one chunk per sequence: the split kernel writes the result itself, no merge kernel
+    const bool direct = Skv_max > 0 && dp.n_chunks == 1;
+    dp.o_final = direct ? o : nullptr;
+    dp.lse_final = direct ? lse : nullptr;
     const int g = Hq / Hkv;
 
     if (Skv_max > 0) {
@@ -535,6 +539,7 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
     }
+    if (direct) return FA_OK;
     if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
     else fa::fa_decode_combine_kernel<__half><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
@@ -587,6 +592,8 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     dp.table_stride = table_stride;
     dp.v_scale = v_scale;
     dp.Sq = 1;
+    dp.o_final = nullptr;
+    dp.lse_final = nullptr;
     const int g = Hq / Hkv;
     if (Skv_max > 0) {
         CUtensorMap tk, tv;

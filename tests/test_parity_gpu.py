@@ -644,6 +644,37 @@ def test_decode_ex_both_types_all_forms(fa, form, dtype):
     assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=f"decode_ex {form} {dtype}")
 
 
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("sq", [1, 3])
+def test_decode_with_a_single_chunk_per_sequence(fa, sq, dtype):
+    # caches short enough for one chunk: the split kernel writes the result itself and no merge
+    # kernel runs; an empty sequence must still get its zeros and -inf.  Also a large batch of
+    # 4K-key caches, where the chunk is the whole cache
+    for (B, hq, hkv, smax, lens) in [(4, 8, 2, 200, [200, 0, 1, 129]), (130, 4, 1, 4096, None)]:
+        cfg = synth.DecodeConfig("t", B, hq, hkv, smax, 1, smax, dtype=dtype, seed=1300 + B + sq)
+        _, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+        if lens is not None:
+            sl[:] = torch.tensor(lens, dtype=torch.int32)
+        sl[0] = smax
+        for b in range(B):
+            k[b, int(sl[b]):] = float("nan")
+            v[b, int(sl[b]):] = float("nan")
+        assert fa.fa_decode_workspace_bytes(B, hq, hkv, smax, 128) == B * hq * 129 * 4     # one chunk
+        gen = torch.Generator().manual_seed(cfg.seed + 1)
+        q = torch.randn(B, sq, hq, 128, generator=gen).to(k.dtype)
+        o_ref, l_ref = oracle.decode_append(q, k.nan_to_num(0.0), v.nan_to_num(0.0), sl, cfg.scale)
+        absv = oracle.decode_append(q, k.nan_to_num(0.0), v.nan_to_num(0.0).abs(), sl, cfg.scale)[0] if dtype == "bf16" else None
+        o, chk_o = guard_alloc((B, sq, hq, 128), k.dtype, DEV)
+        lse, chk_l = guard_alloc((B, hq, sq), torch.float32, DEV)
+        ws, chk_w = guard_alloc((fa.fa_decode_append_workspace_bytes(B, sq, hq, hkv, smax, 128) // 4,), torch.float32, DEV)
+        fa.fa_decode_ex(q.to(DEV), k.to(DEV), v.to(DEV), o, lse, sl.to(DEV), cfg.scale, ws)
+        torch.cuda.synchronize()
+        check_status(fa)
+        chk_o(); chk_l(); chk_w()
+        assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv,
+                               what=f"single-chunk decode B{B} sq{sq} {dtype}")
+
+
 # ------------------------------------------------------------------ decode over an FP8 cache
 def run_decode_fp8(fa, q, k8, v8, seqlens_dev, scale, k_scale, v_scale):
     B, _, Hq, d = q.shape
