@@ -156,13 +156,23 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     const int nq = min(2, p.n_qtiles - qt0);              // its query tiles
     const int off = p.Skv - p.Sq;
 
-    if (tid == 0) {
-        for (int i = 0; i < 6; ++i) mbar_init(smem_u32(&bars[i]), 1);
+    if (tid == 32) {
+        // barriers and all loads of the CTA at once, while warp 0 allocates tensor memory
+        for (int i = 0; i < 6; ++i) mbar_init(smem_u32(&bars[i]), i == 5 ? 2 : 1);   // two threads issue P V
         abort_flag = 0;
         fence_mbar_init();
-        tma_prefetch_desc(&tm_q);
-        tma_prefetch_desc(&tm_k);
-        tma_prefetch_desc(&tm_v);
+        mbar_expect_tx(bar_q0, kD64TileBytes);
+        tma_load_4d(sQ, &tm_q, bar_q0, 0, h, qt0 * kTile, b);
+        mbar_expect_tx(bar_k, 2 * kD64TileBytes);   // rows past the keys arrive as zeros
+        tma_load_4d(sK, &tm_k, bar_k, 0, hk, 0, b);
+        tma_load_4d(sK + kD64TileBytes, &tm_k, bar_k, 0, hk, kTile, b);
+        if (nq > 1) {
+            mbar_expect_tx(bar_q0 + 8, kD64TileBytes);
+            tma_load_4d(sQ + kD64TileBytes, &tm_q, bar_q0 + 8, 0, h, (qt0 + 1) * kTile, b);
+        }
+        mbar_expect_tx(bar_v, 2 * kD64TileBytes);
+        tma_load_4d(sV, &tm_v, bar_v, 0, hk, 0, b);
+        tma_load_4d(sV + kD64TileBytes, &tm_v, bar_v, 0, hk, kTile, b);
     }
     if (warp == 0) {
         __syncwarp();
@@ -181,21 +191,6 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     constexpr uint32_t idesc_qk = instr_desc_f16(kBf16, 128, 256, false, false);
     constexpr uint32_t idesc_pv = instr_desc_f16(kBf16, 128, 64, false, true);
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_q0, kD64TileBytes);
-        tma_load_4d(sQ, &tm_q, bar_q0, 0, h, qt0 * kTile, b);
-        mbar_expect_tx(bar_k, 2 * kD64TileBytes);   // rows past the keys arrive as zeros
-        tma_load_4d(sK, &tm_k, bar_k, 0, hk, 0, b);
-        tma_load_4d(sK + kD64TileBytes, &tm_k, bar_k, 0, hk, kTile, b);
-        if (nq > 1) {
-            mbar_expect_tx(bar_q0 + 8, kD64TileBytes);
-            tma_load_4d(sQ + kD64TileBytes, &tm_q, bar_q0 + 8, 0, h, (qt0 + 1) * kTile, b);
-        }
-        mbar_expect_tx(bar_v, 2 * kD64TileBytes);
-        tma_load_4d(sV, &tm_v, bar_v, 0, hk, 0, b);
-        tma_load_4d(sV + kD64TileBytes, &tm_v, bar_v, 0, hk, kTile, b);
-    }
-    __syncwarp();
 
     const int n_chunks = (p.Skv + 31) / 32;   // chunks of 32 columns that hold keys (5..8)
     bool ok = true;
@@ -230,14 +225,18 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         tc_fence_before();
         __syncthreads();
         // ---- O = P V
-        if (tid == 0) {
+        // Two threads issue one half of the keys each (an N = 64 MMA takes as long to issue as a
+        // wide one, so one thread would spend a thousand clocks on sixteen of them): keys 0..127
+        // into columns [128,192), keys 128..255 into [192,256); the epilogue adds the two.
+        if (tid == 0 || tid == 32) {
+            const int half = tid >> 5;
             if (t == 0) ok = mbar_wait(bar_v, 0, &abort_flag, 54);
             if (ok) {
                 tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 16; ++ks)  // 16 keys per step: 2048 bytes down the two V boxes
-                    mma_ts(tmem_base + 128, tmem_base + ks * 8, smem_desc_sw128(sV + ks * 2048, 16, 1024), idesc_pv,
-                           ks > 0);
+                for (int ks = 0; ks < 8; ++ks)  // 16 keys per step: 2048 bytes down the V boxes
+                    mma_ts(tmem_base + 128 + 64 * half, tmem_base + (half * 8 + ks) * 8,
+                           smem_desc_sw128(sV + (half * 8 + ks) * 2048, 16, 1024), idesc_pv, ks > 0);
                 mma_commit(bar_o);
             }
         }
@@ -250,9 +249,12 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         const long long obase = (long long)b * p.o_sb + (long long)row * p.o_ss + (long long)h * p.o_sh;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-            uint32_t r[32];
+            uint32_t r[32], r2[32];
             tmem_ld_x32(tO + c * 32, r);
+            tmem_ld_x32(tO + 64 + c * 32, r2);
             tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
             if (live_row) {
                 if (p.o_fp32) {
                     float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
