@@ -231,7 +231,7 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64ShortSmem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid((fp.n_qtiles + 1) / 2, fp.Hq, fp.B);
-        kern<<<grid, 128, fa::kD64ShortSmem, st>>>(tq, tk, tv, fp);
+        kern<<<grid, fa::kD64ShortThreads, fa::kD64ShortSmem, st>>>(tq, tk, tv, fp);
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? FA_OK : cuda_fail(e);
     }

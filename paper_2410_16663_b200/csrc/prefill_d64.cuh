@@ -15,20 +15,25 @@ constexpr int kD64TileBytes = 16384;   // 128 rows x 64 16-bit elements: one TMA
 
 // ---------------------------------------------------------------------------------------
 // Short sequences (128 < Skv <= 256, d = 64): the whole key range is one 256-wide tile, so the
-// softmax needs no running state.  One CTA per (batch, head, pair of query tiles): K and V are
-// loaded once for both query tiles; per query tile one N = 256 score MMA into tensor-memory
-// columns [0,256), a first pass over the row for its max, a second pass that writes
-// P = exp(S - max) packed over columns [0,128) (a chunk's P lands in columns the thread has
-// already read), then O = P V into columns [128,192), which the scores no longer need.
-// Chunks of 32 columns that lie entirely past the keys are skipped (their P is written as 0).
-// Two CTAs per SM (97 KiB of shared memory, 256 tensor-memory columns each).
+// softmax needs no running state.  One CTA of two warpgroups per (batch, head, pair of query
+// tiles): K and V are loaded once for both query tiles; per query tile one N = 256 score MMA
+// into tensor-memory columns [0,256).  Warpgroup w then owns keys [128 w, 128 w + 128) of every
+// row: a first pass over its 128 columns for the row max of that half, a second pass that writes
+// P = exp(S - max) packed over the half's first 64 columns (a chunk's P lands in columns the
+// thread has already read), then the half's product P V into the half's last 64 columns, which
+// the scores no longer need.  The epilogue brings the two products to a common reference max
+// (their row max and row sum cross through shared memory) and each thread writes 32 of its
+// row's 64 output columns.  Chunks of 32 columns that lie entirely past the keys are skipped
+// (their P is written as 0).  Two CTAs per SM (97 KiB of shared memory, 256 tensor-memory
+// columns each).
 constexpr int kD64ShortSmem = 1024 + 6 * kD64TileBytes;
 
-// One query row against up to 256 keys whose raw scores sit in tensor-memory columns [0,256) at
-// tS (this thread's lane): row max m (raw units), row sum l of P = exp2((S - m) * scale_log2),
-// and P written packed over columns [0,128).  Columns >= lim are hidden; n_chunks = chunks of 32
-// columns that hold keys.  Warp-collective (tensor-memory loads and stores).
-template <typename T>
+// One query row against up to 32 * kChunks keys whose raw scores sit in tensor-memory columns
+// [0, 32 kChunks) at tS (this thread's lane): row max m (raw units), row sum l of
+// P = exp2((S - m) * scale_log2), and P written packed over columns [0, 16 kChunks).  Columns
+// >= lim are hidden (lim may be negative); n_chunks = chunks of 32 columns that hold keys.
+// Warp-collective (tensor-memory loads and stores).
+template <typename T, int kChunks>
 __device__ __forceinline__ void d64_row_softmax(uint32_t tS, int lim, int n_chunks, float scale_log2, float& m,
                                                 float& l) {
     // ---- pass 1: row max
@@ -61,7 +66,7 @@ __device__ __forceinline__ void d64_row_softmax(uint32_t tS, int lim, int n_chun
     l = 0.f;
     const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
     uint64_t l2 = f2_pack(0.f, 0.f);
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < kChunks; ++c) {
         uint32_t pk[16];
         if (c < my_chunks) {
             uint32_t r[32];
@@ -128,8 +133,10 @@ __device__ __forceinline__ void d64_store_row(const FwdParams& p, long long obas
 }
 
 
+constexpr int kD64ShortThreads = 256;
+
 template <typename T>
-__global__ void __launch_bounds__(128, 2)
+__global__ void __launch_bounds__(kD64ShortThreads, 2)
 fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                         const __grid_constant__ CUtensorMap tm_v, const FwdParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -140,6 +147,7 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     __shared__ __align__(8) uint64_t bars[8];
     __shared__ uint32_t tmem_holder;
     __shared__ volatile uint32_t abort_flag;
+    __shared__ float ex_m[2][kTile], ex_l[2][kTile];   // row max and row sum of each half of the keys
 
     const uint32_t bar_q0 = smem_u32(&bars[0]);  // +8 for the second query tile
     const uint32_t bar_k = smem_u32(&bars[2]);
@@ -149,6 +157,8 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
+    const int wg = tid >> 7;          // 0: keys 0..127, 1: keys 128..255
+    const int r_in = tid & 127;       // row of the query tile (both warpgroups cover all rows)
     const int h = blockIdx.y;
     const int b = blockIdx.z;
     const int hk = h / (p.Hq / p.Hkv);
@@ -183,20 +193,24 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_holder;
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
-    const uint32_t tS = tmem_base + lane_sel;        // columns [0,256): S; P packed in [0,128)
-    const uint32_t tO = tmem_base + lane_sel + 128;  // columns [128,192): O, once P is written
+    // warps w and w + 4 reach the same 32 lanes (rows) of tensor memory
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    // Columns: [0,128) scores of keys 0..127, P of those keys packed over [0,64), their product
+    // P V in [64,128); the same for keys 128..255 in [128,256).  Each half belongs to one
+    // warpgroup until the epilogue, so the two never wait for each other before it.
+    const uint32_t tS = tmem_base + lane_sel + 128 * wg;
+    const uint32_t tOa = tmem_base + lane_sel + 64 + 32 * wg;    // this thread's 32 output columns, keys 0..127
+    const uint32_t tOb = tmem_base + lane_sel + 192 + 32 * wg;   // the same of keys 128..255
 
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
     constexpr uint32_t idesc_qk = instr_desc_f16(kBf16, 128, 256, false, false);
     constexpr uint32_t idesc_pv = instr_desc_f16(kBf16, 128, 64, false, true);
 
-
-    const int n_chunks = (p.Skv + 31) / 32;   // chunks of 32 columns that hold keys (5..8)
+    const int n_chunks = min(4, (p.Skv + 31) / 32 - 4 * wg);   // chunks of 32 columns of this half that hold keys
     bool ok = true;
     for (int t = 0; t < nq && ok; ++t) {
         const int q0 = (qt0 + t) * kTile;
-        const int row = q0 + tid;
+        const int row = q0 + r_in;
         // ---- S = Q K^T over all keys
         if (tid == 0) {
             ok = mbar_wait(bar_q0 + 8 * t, 0, &abort_flag, 51);
@@ -219,65 +233,74 @@ fa_fwd_d64_short_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         int lim = p.Skv;
         if (p.causal) lim = min(lim, row + off + 1);
         if (row >= p.Sq) lim = 0;
+        // softmax of this half of the keys relative to the half's own row max; the epilogue
+        // brings the two halves to a common reference
         float m, l;
-        d64_row_softmax<T>(tS, lim, n_chunks, p.scale_log2, m, l);
+        d64_row_softmax<T, 4>(tS, lim - 128 * wg, n_chunks, p.scale_log2, m, l);
+        ex_m[wg][r_in] = m;
+        ex_l[wg][r_in] = l;
         tmem_wait_st();
         tc_fence_before();
-        __syncthreads();
-        // ---- O = P V
-        // Two threads issue one half of the keys each (an N = 64 MMA takes as long to issue as a
-        // wide one, so one thread would spend a thousand clocks on sixteen of them): keys 0..127
-        // into columns [128,192), keys 128..255 into [192,256); the epilogue adds the two.
-        if (tid == 0 || tid == 32) {
-            const int half = tid >> 5;
+        if (wg == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+        else asm volatile("bar.sync 2, 128;" ::: "memory");
+        // ---- O = P V, one half of the keys per warpgroup (each issued by the warpgroup's first thread)
+        if (r_in == 0) {
             if (t == 0) ok = mbar_wait(bar_v, 0, &abort_flag, 54);
             if (ok) {
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // 16 keys per step: 2048 bytes down the V boxes
-                    mma_ts(tmem_base + 128 + 64 * half, tmem_base + (half * 8 + ks) * 8,
-                           smem_desc_sw128(sV + (half * 8 + ks) * 2048, 16, 1024), idesc_pv, ks > 0);
+                    mma_ts(tmem_base + 64 + 128 * wg, tmem_base + 128 * wg + ks * 8,
+                           smem_desc_sw128(sV + (wg * 8 + ks) * 2048, 16, 1024), idesc_pv, ks > 0);
                 mma_commit(bar_o);
             }
         }
         __syncwarp();
         if (!mbar_wait(bar_o, t & 1, &abort_flag, 55)) { ok = false; break; }
         tc_fence_after();
-        // ---- epilogue: O / l, LSE = max * scale + ln l
-        const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+        __syncthreads();   // the other half's row max and row sum are in shared memory
+        // ---- epilogue: both halves on a common reference, O / l, LSE = max * scale + ln l;
+        // a thread writes 32 of its row's 64 columns
+        const float m_o = ex_m[wg ^ 1][r_in], l_o = ex_l[wg ^ 1][r_in];
+        const float mm = fmaxf(m, m_o);
+        const float w_me = (m == -INFINITY) ? 0.f : fast_exp2((m - mm) * p.scale_log2);
+        const float w_ot = (m_o == -INFINITY) ? 0.f : fast_exp2((m_o - mm) * p.scale_log2);
+        const float lt = l * w_me + l_o * w_ot;
+        const float inv_l = (lt > 0.f) ? 1.f / lt : 0.f;
+        const float fa_ = (wg == 0 ? w_me : w_ot) * inv_l;   // weight of the product over keys 0..127
+        const float fb_ = (wg == 0 ? w_ot : w_me) * inv_l;
         const bool live_row = row < p.Sq;
-        const long long obase = (long long)b * p.o_sb + (long long)row * p.o_ss + (long long)h * p.o_sh;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        const long long obase =
+            (long long)b * p.o_sb + (long long)row * p.o_ss + (long long)h * p.o_sh + 32 * wg;
+        {
             uint32_t r[32], r2[32];
-            tmem_ld_x32(tO + c * 32, r);
-            tmem_ld_x32(tO + 64 + c * 32, r2);
+            tmem_ld_x32(tOa, r);
+            tmem_ld_x32(tOb, r2);
             tmem_wait_ld();
+            float o[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(r[i]) * fa_ + __uint_as_float(r2[i]) * fb_;
             if (live_row) {
                 if (p.o_fp32) {
-                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase + c * 32);
+                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[i] = make_float4(__uint_as_float(r[4 * i]) * inv_l, __uint_as_float(r[4 * i + 1]) * inv_l,
-                                             __uint_as_float(r[4 * i + 2]) * inv_l, __uint_as_float(r[4 * i + 3]) * inv_l);
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 } else {
-                    uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.o) + obase + c * 32);
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<T*>(p.o) + obase);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint4 w;
-                        w.x = pack2<T>(__uint_as_float(r[8 * i]) * inv_l, __uint_as_float(r[8 * i + 1]) * inv_l);
-                        w.y = pack2<T>(__uint_as_float(r[8 * i + 2]) * inv_l, __uint_as_float(r[8 * i + 3]) * inv_l);
-                        w.z = pack2<T>(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
-                        w.w = pack2<T>(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
+                        w.x = pack2<T>(o[8 * i], o[8 * i + 1]);
+                        w.y = pack2<T>(o[8 * i + 2], o[8 * i + 3]);
+                        w.z = pack2<T>(o[8 * i + 4], o[8 * i + 5]);
+                        w.w = pack2<T>(o[8 * i + 6], o[8 * i + 7]);
                         dst[i] = w;
                     }
                 }
             }
         }
-        if (live_row && p.lse != nullptr) {
-            const float lse = (l > 0.f) ? (m * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        if (wg == 0 && live_row && p.lse != nullptr) {
+            const float lse = (lt > 0.f) ? (mm * p.scale_log2 + log2f(lt)) * 0.6931471805599453f : -INFINITY;
             p.lse[((long long)b * p.Hq + h) * p.Sq + row] = lse;
         }
         // the next query tile's scores overwrite the columns O was read from
