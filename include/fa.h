@@ -59,8 +59,9 @@ extern "C" {
 /*
  * Prefill / general forward, fp16 inputs and output (Section 5.1 operator; Section 4.1 method).
  *   q [B,Sq,Hq,d], k,v [B,Skv,Hkv,d], o [B,Sq,Hq,d] fp16, contiguous; lse [B,Hq,Sq] float or NULL.
- *   d must be 128, or 64 (the short vision workload of the evaluation section; fa_forward,
- *   fa_forward_bf16 and fa_forward_ex with variant 0 only; every other entry point wants 128).
+ *   d must be 128, 64 (the short vision workload of the evaluation section) or 256; 64 and 256
+ *   have kernels of their own and are taken by fa_forward, fa_forward_bf16 and fa_forward_ex
+ *   with variant 0 only; every other entry point wants 128.
  *   B == 0 or Sq == 0 is a successful no-op.  Skv == 0 gives O = 0, LSE = -inf.
  *   o and lse must not alias the inputs.
  */

@@ -14,6 +14,7 @@
 #include "decode.cuh"
 #include "prefill_pingpong.cuh"
 #include "prefill_d64.cuh"
+#include "prefill_d256.cuh"
 #include "decode_fp8.cuh"
 #include "prefill_pipelined.cuh"
 #include "prefill_simple.cuh"
@@ -153,8 +154,8 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     // ---- validation (no CUDA call before it passes)
     if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
     if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
-    if (p.d != 128 && p.d != 64) return FA_ERR_UNSUPPORTED;
-    if (p.d == 64 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // the shape picks the d = 64 kernel
+    if (p.d != 128 && p.d != 64 && p.d != 256) return FA_ERR_UNSUPPORTED;
+    if (p.d != 128 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // d = 64 and d = 256 have kernels of their own
     if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
     if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
@@ -242,6 +243,17 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
             return cuda_fail(static_cast<cudaError_t>(ce));
         dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
         kern<<<grid, 128, fa::kD64SlimSmem, st>>>(tq, tk, tv, fp);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
+
+    if (p.d == 256) {  // one CTA per (batch, head, query tile), one CTA per SM
+        auto kern = bf16 ? fa::fa_fwd_d256_kernel<__nv_bfloat16> : fa::fa_fwd_d256_kernel<__half>;
+        int sm_count = 0;
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD256Smem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
+        dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
+        kern<<<grid, 128, fa::kD256Smem, st>>>(tq, tk, tv, fp);
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? FA_OK : cuda_fail(e);
     }

@@ -24,7 +24,7 @@ def main():
     ap.add_argument("--S", type=int, default=8192)
     ap.add_argument("--Skv", type=int, default=0)
     ap.add_argument("--Smax", type=int, default=16384)
-    ap.add_argument("--d", type=int, default=128, choices=[64, 128], help="head dimension (prefill only)")
+    ap.add_argument("--d", type=int, default=128, choices=[64, 128, 256], help="head dimension (prefill only)")
     ap.add_argument("--dtype", default="fp16", choices=["fp16", "bf16"])
     ap.add_argument("--noncausal", action="store_true")
     ap.add_argument("--fp8", action="store_true", help="decode: the cache as FP8 e4m3 (factors 1/4 and 1/8)")

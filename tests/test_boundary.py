@@ -57,7 +57,7 @@ def test_forward_validation_happens_before_any_cuda_call(fa):
     assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 0, 4, 4, 128, 1, 0.1, None) == fa.FA_ERR_SHAPE
     # unsupported
     assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 96, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
-    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 256, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 512, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
     assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 5, 4, 128, 1, 0.1, None) == fa.FA_ERR_UNSUPPORTED
     assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, -1.0, None) == fa.FA_ERR_UNSUPPORTED
     assert L.fa_forward(P(q), P(k), P(k), P(o), None, 1, 4, 2, 4, 4, 128, 1, float("nan"), None) == fa.FA_ERR_UNSUPPORTED

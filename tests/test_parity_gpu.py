@@ -376,6 +376,40 @@ def test_d64_is_refused_where_it_is_not_built(fa):
     assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=3, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
 
 
+# ------------------------------------------------------------------ head dimension 256
+def full_case_d256(fa, B, Hq, Hkv, Sq, Skv, causal, dtype, seed):
+    cfg = synth.PrefillConfig("t", B, Hq, Hkv, Sq, Skv, d=256, dtype=dtype, causal=causal, seed=seed)
+    q, k, v = synth.prefill_inputs(cfg, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, causal, cfg.scale)
+    absv = oracle.attention_full(q, k, v.abs(), causal, cfg.scale)[0] if dtype == "bf16" else None
+    what = f"d256 B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {dtype}"
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=what)
+    if dtype == "bf16":
+        o32, lse32 = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), causal, cfg.scale, o_dtype=torch.float32)
+        assert_close_to_oracle(o32, lse32, o_ref, l_ref, p_absv=absv, what=what + " fp32-out")
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", [(1, 1), (127, 127), (128, 128), (129, 129), (300, 300), (1, 129), (17, 1000),
+                                    (100, 257), (300, 700)])
+def test_d256_shape_grid(fa, sq, skv, causal):
+    full_case_d256(fa, 2, 3, 3, sq, skv, causal, "fp16", seed=sq * 1000 + skv + 13)
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_d256_gqa_both_types_and_more_ctas_than_sms(fa, dtype):
+    full_case_d256(fa, 2, 8, 2, 333, 333, True, dtype, seed=91)
+    full_case_d256(fa, 1, 4, 1, 130, 1500, False, dtype, seed=92)     # many kv tiles through the single slots
+    full_case_d256(fa, 6, 16, 4, 500, 500, True, dtype, seed=93)      # 384 CTAs on 148 SMs
+
+
+def test_d256_is_refused_where_it_is_not_built(fa):
+    q = torch.zeros(1, 4, 2, 256, dtype=torch.float16, device=DEV)
+    o = torch.empty_like(q); lse = torch.empty(1, 2, 4, device=DEV)
+    assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=1, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------------ packed variable-length batches
 def varlen_case(fa, cfg, what):
     q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
