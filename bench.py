@@ -278,6 +278,7 @@ def run_product(args, rank, world, local_rank):
         out["decode_append"] = run_decode_append(fa, dec[-1], dev, peaks)
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
+        out["prefill_d256"] = run_d256(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
         out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
         print(json.dumps(out), flush=True)
@@ -342,6 +343,36 @@ def run_d64(fa, dev, peaks, small=False, iters=10):
             "ms": round(ms, 4), "tflops": round(tf, 1), "gbs": round(gbs, 1), "algorithmic_bytes": nbytes,
             "bound": "hbm", "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
             "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
+
+
+def run_d256(fa, dev, peaks, small=False, iters=5):
+    """Head dimension 256 (the first, sequential kernel), outside the timed steps: causal fp16
+    self-attention, B = 2, 16 heads, 8192 tokens (512 MiB of q, k, v, o: larger than L2); one head
+    of 1024 tokens for the small debugging run."""
+    cfg = (synth.PrefillConfig("d256-8K", 2, 16, 16, 8192, 8192, d=256, dtype="fp16", causal=True, seed=1040)
+           if not small else
+           synth.PrefillConfig("d256-small", 1, 4, 4, 1024, 1024, d=256, dtype="fp16", causal=True, seed=1041))
+    q, k, v = synth.prefill_inputs(cfg, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+    for _ in range(5):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    tf = cfg.flops() / (ms * 1e-3) / 1e12
+    return {"workload": f"{cfg.name}: causal B={cfg.B} H={cfg.Hq} S={cfg.Sq} d=256 fp16", "kernel": "fa_fwd_d256_kernel",
+            "ms": round(ms, 4), "tflops": round(tf, 1), "bound": "tensor",
+            "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4),
+            "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4)}
 
 
 def run_varlen(fa, dev, peaks, small=False, iters=10):
