@@ -252,8 +252,11 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         int sm_count = 0;
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD256Smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
+        CUtensorMap tvh;   // V in boxes of 64 keys: the kernel's V slots hold half a tile
+        rc = encode_map(&tvh, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 64, bf16, p.d);
+        if (rc) return rc;
         dim3 grid(fp.n_qtiles, fp.Hq, fp.B);
-        kern<<<grid, 128, fa::kD256Smem, st>>>(tq, tk, tv, fp);
+        kern<<<grid, fa::kD256Threads, fa::kD256Smem, st>>>(tq, tk, tvh, fp);
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? FA_OK : cuda_fail(e);
     }
