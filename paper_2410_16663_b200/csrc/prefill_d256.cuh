@@ -12,8 +12,9 @@
 // per half of V.  A half-slot of V is refilled as soon as the group that read it has completed,
 // so the first half of the next V tile is always a step ahead and the second is in flight for a
 // whole step; K of tile j + 2 is loaded as soon as the score MMA of tile j + 1 has finished
-// with the slot.  Online softmax as in Appendix A (rowmax / rowsum), with O rescaled only on
-// steps where some row of the warp moved its max.
+// with the slot.  Online softmax as in Appendix A (rowmax / rowsum), with a reference max that
+// moves only when the row max outgrew it by 2^8, and O rescaled only on steps where some row of
+// the warp moved it.
 #pragma once
 
 #include "prefill_simple.cuh"
@@ -179,8 +180,8 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
         const uint32_t tO = tmem_base + lane_sel + 128;
         const int row = q0 + tid;
-        float m_run = -INFINITY;           // running row max, in raw score units
-        float l_run = 0.f;                 // running row sum
+        float m_run = -INFINITY;           // reference max of the row, in raw score units
+        float l_run = 0.f;                 // running row sum, relative to it
         bool ok = true;
 
         for (int j = 0; j < n_tiles; ++j) {
@@ -188,16 +189,16 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint32_t tS = tmem_base + lane_sel + (buf ? 384u : 0u);
             if (!mbar_wait(bar_s + 8 * buf, (j >> 1) & 1, &abort_flag, 68)) { ok = false; break; }
             tc_fence_after();
-            // ---- this row of S
+            // ---- this row of S (four loads in flight, one wait)
+            uint32_t sr[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_x32(tS + c * 32, sr[c]);
+            tmem_wait_ld();
             float s[128];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld_x32(tS + c * 32, r);
-                tmem_wait_ld();
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
-            }
+                for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(sr[c][i]);
             // ---- mask: only tiles the diagonal or the end of the keys cross
             const int kv0 = j * kTile;
             const bool need_mask = (p.causal && kv0 + kTile - 1 > q0 + off) || (kv0 + kTile > p.Skv);
@@ -209,7 +210,10 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 for (int i = 0; i < 128; ++i)
                     if (i >= lim) s[i] = -INFINITY;
             }
-            // ---- online softmax update (Appendix A: rowmax / rowsum)
+            // ---- online softmax update (Appendix A: rowmax / rowsum).  m_run is the reference the
+            // exponentials are taken against; it follows the row max only when that outgrew it by
+            // more than 2^8 (P then stays <= 256, O and l carry the same reference, so O / l and
+            // LSE are unchanged) -- the 256 columns of O are rarely rescaled after the first tiles.
             float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];
 #pragma unroll
             for (int i = 4; i < 128; i += 4) {
@@ -219,9 +223,11 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 m3 = fmaxf(m3, s[i + 3]);
             }
             const float m_tile = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-            const float m_new = fmaxf(m_run, m_tile);
+            const bool moved = (m_tile > m_run) && (m_run == -INFINITY || (m_tile - m_run) * p.scale_log2 > 8.f);
+            const float m_new = moved ? m_tile : m_run;
             const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // a row that sees nothing stays finite
-            const float alpha = (m_run == -INFINITY) ? 0.f : fast_exp2((m_run - m_use) * p.scale_log2);
+            const float alpha =
+                moved ? ((m_run == -INFINITY) ? 0.f : fast_exp2((m_run - m_use) * p.scale_log2)) : 1.f;
             const float neg_ms = -m_use * p.scale_log2;
             float l0 = 0.f, l1 = 0.f;
             if (need_mask) {
@@ -243,14 +249,13 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
             }
             l_run = l_run * alpha + (l0 + l1);
-            const bool moved = (m_new != m_run);
             m_run = m_new;
 
             // ---- O <- alpha * O once the previous P V has landed
             if (j > 0) {
                 if (!mbar_wait(bar_o, (j - 1) & 1, &abort_flag, 69)) { ok = false; break; }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, moved)) {   // alpha is exactly 1 for a row whose max stayed
+                if (__any_sync(0xffffffffu, moved)) {   // alpha is exactly 1 for a row whose reference stayed
 #pragma unroll 2
                     for (int c = 0; c < 8; ++c) {
                         uint32_t r[32];
