@@ -346,7 +346,7 @@ def run_d64(fa, dev, peaks, small=False, iters=10):
 
 
 def run_d256(fa, dev, peaks, small=False, iters=5):
-    """Head dimension 256 (the first, sequential kernel), outside the timed steps: causal fp16
+    """Head dimension 256 (its own kernel), outside the timed steps: causal fp16
     self-attention, B = 2, 16 heads, 8192 tokens (512 MiB of q, k, v, o: larger than L2); one head
     of 1024 tokens for the small debugging run."""
     cfg = (synth.PrefillConfig("d256-8K", 2, 16, 16, 8192, 8192, d=256, dtype="fp16", causal=True, seed=1040)
