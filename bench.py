@@ -323,7 +323,7 @@ def run_d64(fa, dev, peaks, small=False, iters=10):
     q, k, v = synth.prefill_inputs(cfg, device=dev)
     o = torch.empty_like(q)
     lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
-    for _ in range(20):   # the legs before this one are memory-bound: let the clocks settle
+    for _ in range(100):   # the legs before this one are memory-bound: let the clocks settle
         fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -355,7 +355,7 @@ def run_d256(fa, dev, peaks, small=False, iters=5):
     q, k, v = synth.prefill_inputs(cfg, device=dev)
     o = torch.empty_like(q)
     lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
-    for _ in range(5):
+    for _ in range(30):   # let the clocks settle after the memory-bound legs
         fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
