@@ -25,12 +25,20 @@ constexpr int kD256TileBytes = 4 * kHalfBytes;              // 128 rows x 256 16
 constexpr int kD256VHalfBytes = kD256TileBytes / 2;         // 64 keys x 256: four boxes of 64 x 64
 constexpr int kD256VBoxBytes = kD256VHalfBytes / 4;         // one of them (the MMA's LBO)
 constexpr int kD256Smem = 1024 + 2 * kD256TileBytes + 3 * kD256VHalfBytes;
-constexpr int kD256Threads = 160;
+constexpr int kD256Threads = 192;   // four softmax warps, the score-MMA warp, the P V warp
 
 __device__ __forceinline__ void d256_load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int h, int s0,
                                                int b) {
 #pragma unroll
     for (int c = 0; c < 4; ++c) tma_load_4d(dst + c * kHalfBytes, tm, bar, 64 * c, h, s0, b);
+}
+
+// Half of a K tile along d (two of its four boxes): half 0 = head dimensions 0..127
+__device__ __forceinline__ void d256_load_k_half(uint32_t sK, const CUtensorMap* tm, uint32_t bar, int half, int h,
+                                                 int s0, int b) {
+    mbar_expect_tx(bar, 2 * kHalfBytes);
+#pragma unroll
+    for (int c = 2 * half; c < 2 * half + 2; ++c) tma_load_4d(sK + c * kHalfBytes, tm, bar, 64 * c, h, s0, b);
 }
 
 // tm_vh: the map over V with boxes of 64 keys
@@ -50,12 +58,14 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kD256TileBytes;
     const uint32_t sV = sK + kD256TileBytes;   // three half-tile slots
-    __shared__ __align__(8) uint64_t bars[12];
+    __shared__ __align__(8) uint64_t bars[14];
     __shared__ uint32_t tmem_holder;
     __shared__ volatile uint32_t abort_flag;
 
     const uint32_t bar_q = smem_u32(&bars[0]);
-    const uint32_t bar_k = smem_u32(&bars[1]);
+    const uint32_t bar_ka = smem_u32(&bars[1]);    // K, head dimensions 0..127 (two boxes) landed
+    const uint32_t bar_kb = smem_u32(&bars[11]);   // K, head dimensions 128..255 landed
+    const uint32_t bar_sa = smem_u32(&bars[12]);   // the score MMAs over the first half of d completed
     const uint32_t bar_vh = smem_u32(&bars[2]);    // +8 per half-slot (3)
     const uint32_t bar_s = smem_u32(&bars[5]);     // +8 per score buffer (2): S landed
     const uint32_t bar_p = smem_u32(&bars[7]);     // +8 per score buffer (2): P written, O rescaled (128 arrivals)
@@ -73,14 +83,14 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int n_tiles = kv_tiles_for(q0, kTile, p.Sq, p.Skv, p.causal);
 
     if (tid == 128) {
-        for (int i = 0; i < 11; ++i) mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8) ? 128 : 1);
+        for (int i = 0; i < 13; ++i) mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8) ? 128 : 1);
         abort_flag = 0;
         fence_mbar_init();
         if (n_tiles > 0) {
             mbar_expect_tx(bar_q, kD256TileBytes);
             d256_load_tile(sQ, &tm_q, bar_q, h, q0, b);
-            mbar_expect_tx(bar_k, kD256TileBytes);
-            d256_load_tile(sK, &tm_k, bar_k, hk, 0, b);
+            d256_load_k_half(sK, &tm_k, bar_ka, 0, hk, 0, b);
+            d256_load_k_half(sK, &tm_k, bar_kb, 1, hk, 0, b);
             for (int hh = 0; hh < 3 && hh < 2 * n_tiles; ++hh)
                 d256_load_v_half(sV + hh * kD256VHalfBytes, &tm_vh, bar_vh + 8 * hh, hk, hh * 64, b);
         }
@@ -100,44 +110,52 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     constexpr uint32_t idesc_pv = instr_desc_f16(kBf16, 128, 256, false, true);
 
     if (warp == 4) {
-        // =========================== loads and MMAs: one thread
+        // =========================== K loads and score MMAs: one thread
         if (tid == 128 && n_tiles > 0) {
-            bool ok = true;
-            auto issue_s = [&](int j) {   // S(j) = Q K_j^T into score buffer j & 1
-                const uint32_t d_tmem = tmem_base + ((j & 1) ? 384u : 0u);
-                tc_fence_after();
+            bool ok = mbar_wait(bar_q, 0, &abort_flag, 61);
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int buf = t & 1;
+                // S(t) overwrites the buffer P(t - 2) sat in: P V of that tile must have completed
+                if (t >= 2) {
+                    ok = mbar_wait(bar_o, t & 1, &abort_flag, 67);
+                    if (!ok) break;
+                }
+                // S(t) = Q K_t^T in two runs of eight k-steps: the first reads the lower half of d (K's
+                // first two boxes), which is refilled as soon as that run has completed
+                const uint32_t d_tmem = tmem_base + (buf ? 384u : 0u);
 #pragma unroll
-                for (int ks = 0; ks < 16; ++ks) {
-                    const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    mma_ss(d_tmem, smem_desc_sw128(sQ + koff, 16, 1024), smem_desc_sw128(sK + koff, 16, 1024), idesc_qk,
-                           ks > 0);
+                for (int run = 0; run < 2; ++run) {
+                    ok = mbar_wait(run ? bar_kb : bar_ka, t & 1, &abort_flag, 62);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 8 * run; ks < 8 * run + 8; ++ks) {
+                        const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                        mma_ss(d_tmem, smem_desc_sw128(sQ + koff, 16, 1024), smem_desc_sw128(sK + koff, 16, 1024),
+                               idesc_qk, ks > 0);
+                    }
+                    mma_commit(run ? bar_s + 8 * buf : bar_sa);
                 }
-                mma_commit(bar_s + 8 * (j & 1));
-            };
-            ok = mbar_wait(bar_q, 0, &abort_flag, 61) && mbar_wait(bar_k, 0, &abort_flag, 62);
-            if (ok) issue_s(0);
-            if (ok && n_tiles > 1) {
-                // S(0) has finished with the K slot: K(1), then S(1) into the second buffer
-                ok = mbar_wait(bar_s, 0, &abort_flag, 63);
-                if (ok) {
-                    mbar_expect_tx(bar_k, kD256TileBytes);
-                    d256_load_tile(sK, &tm_k, bar_k, hk, kTile, b);
-                    ok = mbar_wait(bar_k, 1, &abort_flag, 62);
+                if (!ok) break;
+                if (t + 1 < n_tiles) {
+                    ok = mbar_wait(bar_sa, t & 1, &abort_flag, 63);
+                    if (!ok) break;
+                    d256_load_k_half(sK, &tm_k, bar_ka, 0, hk, (t + 1) * kTile, b);
+                    ok = mbar_wait(bar_s + 8 * buf, (t >> 1) & 1, &abort_flag, 63);
+                    if (!ok) break;
+                    d256_load_k_half(sK, &tm_k, bar_kb, 1, hk, (t + 1) * kTile, b);
                 }
-                if (ok) issue_s(1);
             }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // =========================== V loads and P V MMAs: one thread
+        if (tid == 160 && n_tiles > 0) {
+            bool ok = true;
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int buf = j & 1;
-                const uint32_t use_par = (j >> 1) & 1;   // parity of the buffer's barriers for tile j
-                // K(j + 2) as soon as S(j + 1) has finished with the slot
-                if (j + 2 < n_tiles) {
-                    ok = mbar_wait(bar_s + 8 * (buf ^ 1), ((j + 1) >> 1) & 1, &abort_flag, 63);
-                    if (!ok) break;
-                    mbar_expect_tx(bar_k, kD256TileBytes);
-                    d256_load_tile(sK, &tm_k, bar_k, hk, (j + 2) * kTile, b);
-                }
                 // ---- O += P(j) V_j, one group of four k-steps per half of V
-                ok = mbar_wait(bar_p + 8 * buf, use_par, &abort_flag, 64);
+                ok = mbar_wait(bar_p + 8 * buf, (j >> 1) & 1, &abort_flag, 64);
                 if (!ok) break;
                 const uint32_t p_tmem = tmem_base + (buf ? 384u : 0u);
 #pragma unroll
@@ -166,12 +184,6 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 if (2 * j + 4 < 2 * n_tiles)
                     d256_load_v_half(sV + ((2 * j + 1) % 3) * kD256VHalfBytes, &tm_vh, bar_vh + 8 * ((2 * j + 1) % 3), hk,
                                      (2 * j + 4) * 64, b);
-                // ---- S(j + 2) into the buffer P(j) has just left
-                if (j + 2 < n_tiles) {
-                    ok = mbar_wait(bar_k, j & 1, &abort_flag, 62);   // K(j + 2): the (j + 2)-th completion
-                    if (!ok) break;
-                    issue_s(j + 2);
-                }
             }
         }
         __syncwarp();
