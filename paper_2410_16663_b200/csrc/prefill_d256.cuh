@@ -1,20 +1,20 @@
-// Attention forward for head dimension 256.  One CTA per (batch, head, 128-row query tile):
-// four softmax warps (one thread per query row) and a fifth warp whose first lane issues every
-// TMA load and every MMA.  Tiles are 128 rows x 256 elements = four 64-column swizzled boxes
-// (64 KiB).  Shared memory: Q, one slot for K, and three slots of HALF a V tile each (64 keys x
-// 256, 32 KiB), 224 KiB in all, one CTA per SM.  Tensor memory: two score buffers, columns [0,128)
-// and [384,512), and O in [128,384).
+// Attention forward for head dimension 256.  One CTA of six warps per (batch, head, 128-row query
+// tile): four softmax warps (one thread per query row), a warp whose first lane loads K and
+// issues the score MMAs, and a warp whose first lane loads V and issues the P V MMAs.  Tiles are
+// 128 rows x 256 elements = four 64-column swizzled boxes (64 KiB).  Shared memory: Q, three
+// slots of half a K tile along d (128 keys x 128, two boxes, 32 KiB) and two slots of half a V
+// tile along the keys (64 keys x 256, 32 KiB): 224 KiB in all, one CTA per SM.  Tensor memory:
+// two score buffers, columns [0,128) and [384,512), and O in [128,384).
 //
-// S = Q K^T of kv tile j + 1 is issued before the softmax of tile j begins (into the other score
-// buffer), so the tensor core works under the softmax; P goes back packed over the first 64
-// columns of its score buffer; O += P V is an N = 256 MMA per 16 keys with V as the N-major
-// operand (its four boxes one leading-dimension stride apart), issued in two groups of four, one
-// per half of V.  A half-slot of V is refilled as soon as the group that read it has completed,
-// so the first half of the next V tile is always a step ahead and the second is in flight for a
-// whole step; K of tile j + 2 is loaded as soon as the score MMA of tile j + 1 has finished
-// with the slot.  Online softmax as in Appendix A (rowmax / rowsum), with a reference max that
-// moves only when the row max outgrew it by 2^8, and O rescaled only on steps where some row of
-// the warp moved it.
+// S = Q K^T of kv tile t goes into score buffer t & 1 as soon as P V of tile t - 2 has left it,
+// i.e. while the softmax of tile t - 1 is at work, in two runs of eight k-steps, one per half of
+// d; the K half-slot a run has read is refilled (with the half three further on) as soon as the
+// run has completed, so every K load has about a step to arrive.  P goes back packed over the
+// first 64 columns of its score buffer; O += P V is an N = 256 MMA per 16 keys with V as the
+// N-major operand (its four boxes one leading-dimension stride apart), issued in two groups of
+// four, one per half of V, and a V half-slot is refilled as soon as its group has completed.
+// Online softmax as in Appendix A (rowmax / rowsum), with a reference max that moves only when
+// the row max outgrew it by 2^8, and O rescaled only on steps where some row of the warp moved it.
 #pragma once
 
 #include "prefill_simple.cuh"
@@ -24,7 +24,8 @@ namespace fa {
 constexpr int kD256TileBytes = 4 * kHalfBytes;              // 128 rows x 256 16-bit elements
 constexpr int kD256VHalfBytes = kD256TileBytes / 2;         // 64 keys x 256: four boxes of 64 x 64
 constexpr int kD256VBoxBytes = kD256VHalfBytes / 4;         // one of them (the MMA's LBO)
-constexpr int kD256Smem = 1024 + 2 * kD256TileBytes + 3 * kD256VHalfBytes;
+constexpr int kD256KHalfBytes = kD256TileBytes / 2;         // 128 keys x 128 of d: two boxes of 128 x 64
+constexpr int kD256Smem = 1024 + kD256TileBytes + 3 * kD256KHalfBytes + 2 * kD256VHalfBytes;
 constexpr int kD256Threads = 192;   // four softmax warps, the score-MMA warp, the P V warp
 
 __device__ __forceinline__ void d256_load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int h, int s0,
@@ -33,12 +34,12 @@ __device__ __forceinline__ void d256_load_tile(uint32_t dst, const CUtensorMap* 
     for (int c = 0; c < 4; ++c) tma_load_4d(dst + c * kHalfBytes, tm, bar, 64 * c, h, s0, b);
 }
 
-// Half of a K tile along d (two of its four boxes): half 0 = head dimensions 0..127
-__device__ __forceinline__ void d256_load_k_half(uint32_t sK, const CUtensorMap* tm, uint32_t bar, int half, int h,
+// Half of a K tile along d (two of its four boxes) into a half-slot: half 0 = head dimensions 0..127
+__device__ __forceinline__ void d256_load_k_half(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int half, int h,
                                                  int s0, int b) {
-    mbar_expect_tx(bar, 2 * kHalfBytes);
+    mbar_expect_tx(bar, kD256KHalfBytes);
 #pragma unroll
-    for (int c = 2 * half; c < 2 * half + 2; ++c) tma_load_4d(sK + c * kHalfBytes, tm, bar, 64 * c, h, s0, b);
+    for (int c = 0; c < 2; ++c) tma_load_4d(dst + c * kHalfBytes, tm, bar, 64 * (2 * half + c), h, s0, b);
 }
 
 // tm_vh: the map over V with boxes of 64 keys
@@ -56,21 +57,20 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base;
-    const uint32_t sK = sQ + kD256TileBytes;
-    const uint32_t sV = sK + kD256TileBytes;   // three half-tile slots
+    const uint32_t sK = sQ + kD256TileBytes;       // three half-tile slots (128 keys x 128 of d each)
+    const uint32_t sV = sK + 3 * kD256KHalfBytes;   // two half-tile slots (64 keys x 256 each)
     __shared__ __align__(8) uint64_t bars[14];
     __shared__ uint32_t tmem_holder;
     __shared__ volatile uint32_t abort_flag;
 
     const uint32_t bar_q = smem_u32(&bars[0]);
-    const uint32_t bar_ka = smem_u32(&bars[1]);    // K, head dimensions 0..127 (two boxes) landed
-    const uint32_t bar_kb = smem_u32(&bars[11]);   // K, head dimensions 128..255 landed
+    const uint32_t bar_kh = smem_u32(&bars[1]);    // +8 per K half-slot (3): half a K tile along d landed
+    const uint32_t bar_vh = smem_u32(&bars[4]);    // +8 per V half-slot (2): half a V tile along the keys landed
+    const uint32_t bar_s = smem_u32(&bars[6]);     // +8 per score buffer (2): S landed
+    const uint32_t bar_p = smem_u32(&bars[8]);     // +8 per score buffer (2): P written, O rescaled (128 arrivals)
+    const uint32_t bar_g = smem_u32(&bars[10]);    // first group of a tile's P V completed
+    const uint32_t bar_o = smem_u32(&bars[11]);    // a tile's P V completed
     const uint32_t bar_sa = smem_u32(&bars[12]);   // the score MMAs over the first half of d completed
-    const uint32_t bar_vh = smem_u32(&bars[2]);    // +8 per half-slot (3)
-    const uint32_t bar_s = smem_u32(&bars[5]);     // +8 per score buffer (2): S landed
-    const uint32_t bar_p = smem_u32(&bars[7]);     // +8 per score buffer (2): P written, O rescaled (128 arrivals)
-    const uint32_t bar_g = smem_u32(&bars[9]);     // first group of a tile's P V completed
-    const uint32_t bar_o = smem_u32(&bars[10]);    // a tile's P V completed
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -83,15 +83,15 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int n_tiles = kv_tiles_for(q0, kTile, p.Sq, p.Skv, p.causal);
 
     if (tid == 128) {
-        for (int i = 0; i < 13; ++i) mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8) ? 128 : 1);
+        for (int i = 0; i < 13; ++i) mbar_init(smem_u32(&bars[i]), (i == 8 || i == 9) ? 128 : 1);
         abort_flag = 0;
         fence_mbar_init();
         if (n_tiles > 0) {
             mbar_expect_tx(bar_q, kD256TileBytes);
             d256_load_tile(sQ, &tm_q, bar_q, h, q0, b);
-            d256_load_k_half(sK, &tm_k, bar_ka, 0, hk, 0, b);
-            d256_load_k_half(sK, &tm_k, bar_kb, 1, hk, 0, b);
-            for (int hh = 0; hh < 3 && hh < 2 * n_tiles; ++hh)
+            for (int kh = 0; kh < 3 && kh < 2 * n_tiles; ++kh)
+                d256_load_k_half(sK + kh * kD256KHalfBytes, &tm_k, bar_kh + 8 * kh, kh & 1, hk, (kh >> 1) * kTile, b);
+            for (int hh = 0; hh < 2; ++hh)
                 d256_load_v_half(sV + hh * kD256VHalfBytes, &tm_vh, bar_vh + 8 * hh, hk, hh * 64, b);
         }
     }
@@ -120,30 +120,39 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     ok = mbar_wait(bar_o, t & 1, &abort_flag, 67);
                     if (!ok) break;
                 }
-                // S(t) = Q K_t^T in two runs of eight k-steps: the first reads the lower half of d (K's
-                // first two boxes), which is refilled as soon as that run has completed
+                // S(t) = Q K_t^T in two runs of eight k-steps, one per half of d; K's halves go round
+                // three half-slots, and the slot a run has read is refilled (with the half three
+                // further on) as soon as that run has completed
                 const uint32_t d_tmem = tmem_base + (buf ? 384u : 0u);
 #pragma unroll
                 for (int run = 0; run < 2; ++run) {
-                    ok = mbar_wait(run ? bar_kb : bar_ka, t & 1, &abort_flag, 62);
+                    const int kh = 2 * t + run;
+                    const uint32_t sKh = sK + (kh % 3) * kD256KHalfBytes;
+                    ok = mbar_wait(bar_kh + 8 * (kh % 3), (kh / 3) & 1, &abort_flag, 62);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
-                    for (int ks = 8 * run; ks < 8 * run + 8; ++ks) {
+                    for (int ks = 0; ks < 8; ++ks) {
                         const uint32_t koff = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_ss(d_tmem, smem_desc_sw128(sQ + koff, 16, 1024), smem_desc_sw128(sK + koff, 16, 1024),
-                               idesc_qk, ks > 0);
+                        mma_ss(d_tmem, smem_desc_sw128(sQ + run * 2 * kHalfBytes + koff, 16, 1024),
+                               smem_desc_sw128(sKh + koff, 16, 1024), idesc_qk, run > 0 || ks > 0);
                     }
                     mma_commit(run ? bar_s + 8 * buf : bar_sa);
                 }
                 if (!ok) break;
-                if (t + 1 < n_tiles) {
+                if (2 * t + 3 < 2 * n_tiles) {
                     ok = mbar_wait(bar_sa, t & 1, &abort_flag, 63);
                     if (!ok) break;
-                    d256_load_k_half(sK, &tm_k, bar_ka, 0, hk, (t + 1) * kTile, b);
+                    const int kh = 2 * t + 3;
+                    d256_load_k_half(sK + (kh % 3) * kD256KHalfBytes, &tm_k, bar_kh + 8 * (kh % 3), kh & 1, hk,
+                                     (kh >> 1) * kTile, b);
+                }
+                if (2 * t + 4 < 2 * n_tiles) {
                     ok = mbar_wait(bar_s + 8 * buf, (t >> 1) & 1, &abort_flag, 63);
                     if (!ok) break;
-                    d256_load_k_half(sK, &tm_k, bar_kb, 1, hk, (t + 1) * kTile, b);
+                    const int kh = 2 * t + 4;
+                    d256_load_k_half(sK + (kh % 3) * kD256KHalfBytes, &tm_k, bar_kh + 8 * (kh % 3), kh & 1, hk,
+                                     (kh >> 1) * kTile, b);
                 }
             }
         }
@@ -160,9 +169,8 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const uint32_t p_tmem = tmem_base + (buf ? 384u : 0u);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const int hh = 2 * j + half;
-                    const int slot = hh % 3;
-                    ok = mbar_wait(bar_vh + 8 * slot, (hh / 3) & 1, &abort_flag, 65);
+                    const int slot = half;   // half 2 j + half of V sits in slot `half`, its j-th use
+                    ok = mbar_wait(bar_vh + 8 * slot, j & 1, &abort_flag, 65);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -176,14 +184,11 @@ fa_fwd_d256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 // ---- refill the half-slots as their groups complete
                 ok = mbar_wait(bar_g, j & 1, &abort_flag, 66);
                 if (!ok) break;
-                if (2 * j + 3 < 2 * n_tiles)
-                    d256_load_v_half(sV + ((2 * j) % 3) * kD256VHalfBytes, &tm_vh, bar_vh + 8 * ((2 * j) % 3), hk,
-                                     (2 * j + 3) * 64, b);
+                if (j + 1 < n_tiles) d256_load_v_half(sV, &tm_vh, bar_vh, hk, (2 * j + 2) * 64, b);
                 ok = mbar_wait(bar_o, j & 1, &abort_flag, 67);
                 if (!ok) break;
-                if (2 * j + 4 < 2 * n_tiles)
-                    d256_load_v_half(sV + ((2 * j + 1) % 3) * kD256VHalfBytes, &tm_vh, bar_vh + 8 * ((2 * j + 1) % 3), hk,
-                                     (2 * j + 4) * 64, b);
+                if (j + 1 < n_tiles)
+                    d256_load_v_half(sV + kD256VHalfBytes, &tm_vh, bar_vh + 8, hk, (2 * j + 3) * 64, b);
             }
         }
         __syncwarp();
