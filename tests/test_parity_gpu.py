@@ -404,6 +404,21 @@ def test_d256_gqa_both_types_and_more_ctas_than_sms(fa, dtype):
     full_case_d256(fa, 6, 16, 4, 500, 500, True, dtype, seed=93)      # 384 CTAs on 148 SMs
 
 
+def test_d256_bench_size_sampled(fa):
+    # the benchmark's d = 256 case (2 x 16 heads x 8192, causal): sampled rows against the oracle, everything finite
+    cfg = synth.PrefillConfig("d256-8K", 2, 16, 16, 8192, 8192, d=256, dtype="fp16", causal=True, seed=1040)
+    q, k, v = synth.prefill_inputs(cfg, DEV)
+    o, lse = run_forward(fa, q, k, v, cfg.causal, cfg.scale)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    rows = synth.sample_rows(cfg, 5, seed=6, pairs=[(0, 0), (0, 15), (1, 7), (1, 15)])
+    rows += [(0, 3, 0), (1, 3, 8191), (0, 9, 127), (1, 9, 128), (0, 12, 4095)]   # first, last, tile edges
+    o_ref, l_ref = oracle_rows_for(q, k, v, rows, cfg.causal, cfg.scale)
+    idx = torch.tensor(rows)
+    o_s = o[idx[:, 0], idx[:, 2], idx[:, 1]].view(1, len(rows), 1, cfg.d)
+    l_s = lse[idx[:, 0], idx[:, 1], idx[:, 2]].view(1, 1, len(rows))
+    assert_close_to_oracle(o_s, l_s, o_ref.view(1, len(rows), 1, cfg.d), l_ref.view(1, 1, len(rows)), what="d256 8K")
+
+
 def test_d256_is_refused_where_it_is_not_built(fa):
     q = torch.zeros(1, 4, 2, 256, dtype=torch.float16, device=DEV)
     o = torch.empty_like(q); lse = torch.empty(1, 2, 4, device=DEV)
