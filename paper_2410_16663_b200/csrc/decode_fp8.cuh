@@ -54,7 +54,15 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     len = max(0, min(len, p.Smax));
     const int k_begin = c * p.chunk;
     const int k_end = min(len, k_begin + p.chunk);
-    if (k_begin >= k_end) return;  // uniform for the CTA
+    if (k_begin >= k_end) {  // uniform for the CTA
+        if (p.o_final != nullptr && tid < 128) {   // a sequence without keys, and nobody else writes its rows
+            for (int r = 0; r < G; ++r) {
+                static_cast<__half*>(p.o_final)[((long long)b * p.Hq + h0 + r) * 128 + tid] = __half(0.f);
+                if (tid == 0 && p.lse_final) p.lse_final[(long long)b * p.Hq + h0 + r] = -INFINITY;
+            }
+        }
+        return;
+    }
     const int n_tiles = (k_end - k_begin + kDecTile - 1) / kDecTile;
 
     if (tid == 0) {
@@ -342,9 +350,17 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     l += sw * ml[(w * 16 + r) * 2 + 1];
                     acc += sw * mo[(w * 16 + r) * 128 + col];
                 }
-                const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;
-                p.o_part[slot * 128 + col] = acc / l * p.v_scale;
-                if (col == 0) p.lse_part[slot] = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
+                const float out = acc / l * p.v_scale;
+                const float lse = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
+                if (p.o_final != nullptr) {   // the only chunk: this is the result
+                    const long long row = (long long)b * p.Hq + h0 + r;
+                    static_cast<__half*>(p.o_final)[row * 128 + col] = __half(out);
+                    if (col == 0 && p.lse_final) p.lse_final[row] = lse;
+                } else {
+                    const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;
+                    p.o_part[slot * 128 + col] = out;
+                    if (col == 0) p.lse_part[slot] = lse;
+                }
             }
         }
     }

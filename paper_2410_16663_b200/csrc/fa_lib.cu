@@ -607,8 +607,10 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     dp.table_stride = table_stride;
     dp.v_scale = v_scale;
     dp.Sq = 1;
-    dp.o_final = nullptr;
-    dp.lse_final = nullptr;
+    // one chunk per sequence: the split kernel writes O and LSE itself and no merge is launched
+    const bool direct = Skv_max > 0 && dp.n_chunks == 1;
+    dp.o_final = direct ? o : nullptr;
+    dp.lse_final = direct ? lse : nullptr;
     const int g = Hq / Hkv;
     if (Skv_max > 0) {
         CUtensorMap tk, tv;
@@ -631,6 +633,7 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
         if (rc) return rc;
     }
+    if (direct) return FA_OK;
     fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);

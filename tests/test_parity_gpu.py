@@ -753,6 +753,26 @@ def test_decode_fp8_small_full(fa, hq, hkv):
     assert float(o[1].abs().max()) == 0.0 and torch.isneginf(lse[1]).all()
 
 
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (4, 1), (12, 1)])
+def test_decode_fp8_with_a_single_chunk_per_sequence(fa, hq, hkv):
+    # caches short enough for one chunk: the split kernel writes the result itself and no merge
+    # kernel runs; an empty sequence must still get its zeros and -inf.  Also a large batch of
+    # 4K-key caches, where the chunk is the whole cache
+    for (B, smax, lens) in [(4, 200, [200, 0, 1, 129]), (130, 4096, None)]:
+        cfg = synth.DecodeConfig("t", B, hq, hkv, smax, 1, smax, seed=1700 + B + hq)
+        q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+        if lens is not None:
+            sl[:] = torch.tensor(lens, dtype=torch.int32)
+        sl[0] = smax
+        assert fa.fa_decode_workspace_bytes(B, hq, hkv, smax, 128) == B * hq * 129 * 4     # one chunk
+        k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+        o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, 0.25, 0.125)
+        o, lse = run_decode_fp8(fa, q.to(DEV), k8.to(DEV), v8.to(DEV), sl.to(DEV), cfg.scale, 0.25, 0.125)
+        assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, what=f"fp8 single-chunk decode B{B} {hq}/{hkv}")
+        if lens is not None:
+            assert float(o[1].abs().max()) == 0.0 and torch.isneginf(lse[1]).all()
+
+
 def test_decode_fp8_every_bit_pattern_in_every_position(fa):
     # every finite e4m3 pattern in K and V (drawn uniformly over the bit patterns, so that
     # subnormals, both signs and the largest values occur), lengths around tile and chunk
