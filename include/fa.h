@@ -114,8 +114,8 @@ int fa_forward_ex(const fa_params* p, void* stream);
  *   (they size the launch: a longer sequence would be cut off at the bound).
  *   A sequence without keys, and under the causal mask every row that sees no key (a sequence
  *   with more queries than keys), gives O = 0 and LSE = -inf.  The prefix sums are read by the
- *   kernel only and are not validated.  K and V rows of the NEXT sequence may be loaded and
- *   multiplied by exact zeros; like everything in k and v they must be finite.
+ *   kernel only and are not validated.  K and V rows of the NEXT sequence may be loaded, but they
+ *   never reach a result (their scores are masked and their V rows are cleared on chip).
  * Errors: as fa_forward; FA_ERR_SHAPE also for max_seqlen_q > total_q or max_seqlen_k > total_k.
  */
 int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, float* lse,
@@ -150,8 +150,8 @@ size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
  * v_pages [num_pages, page_size, Hkv, d]; page_size a positive multiple of 128; max_seqlen_k an
  * upper bound of seqlens_k, at most max_pages * page_size.  The causal mask is aligned
  * bottom-right per sequence (the queries are the sequence's LAST rows).  Only the table entries
- * that cover keys [0, seqlens_k[b]) are read.  Rows of a page past the end of its sequence are
- * multiplied by exact zeros: they must hold finite values (zeros, or stale keys and values).
+ * that cover keys [0, seqlens_k[b]) are read (none for a sequence without keys).  Rows of a page
+ * past the end of its sequence, and unused pages, may hold anything (NaN too).
  * Errors: as fa_forward_varlen; FA_ERR_SHAPE also for a page_size that is not a multiple of 128,
  * table_stride < max_pages or max_seqlen_k > max_pages * page_size.
  */
@@ -270,7 +270,8 @@ int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, con
  *     the same call first.  All calls share the one array, so two calls whose kernels may
  *     overlap on the GPU (different streams, no ordering between them) race on it; order them.
  *   - The function itself allocates nothing: no cudaMalloc, cudaFree or allocating library call.
- * Results are identical to fa_decode's for the same arguments.
+ * Results are bit-identical to fa_decode's for the same arguments, and so are the argument checks
+ * and their error codes (they run before the size limit is looked at and before any CUDA call).
  */
 #define FA_DECODE_NOALLOC_BYTES (4u << 20)
 int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
@@ -288,7 +289,8 @@ int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, v
  * the copies on two streams the library creates once per device (with a handful of events) and
  * keeps; nothing else is created and no device memory is allocated.  Make the first call on a
  * device outside stream capture.  Calls that share a staging buffer must be issued on the same
- * stream.
+ * stream.  Host threads may call concurrently on one device with staging buffers and streams of
+ * their own: the enqueue sequence of a call is serialised inside the library.
  */
 int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, void* o_host,
                     float* lse_host, int B, int Hq, int Hkv, int Sq, int Skv, int d, int causal,
@@ -302,6 +304,16 @@ size_t fa_forward_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Skv, in
  * (detail[0] = where, detail[1] = block index, if detail != NULL), or FA_ERR_CUDA.
  */
 int fa_device_status(unsigned int detail[2]);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper): launches one small CTA whose 64
+ * threads wait, for at most limit_us microseconds (1 .. 100000), on a barrier that nothing will
+ * ever complete.  The wait gives up by construction -- no trap, no fault, no endless loop -- and
+ * every thread returns normally.  Afterwards *gave_up (a DEVICE counter the caller zeroed) has
+ * been raised by 64 and fa_device_status() reports FA_ERR_TIMEOUT once, with detail[0] == 990,
+ * then FA_OK again: the same path a kernel of the library takes if one of its waits ever expired.
+ */
+int fa_selftest_wait(unsigned int limit_us, unsigned int* gave_up, void* stream);
 
 const char* fa_strerror(int code);
 int fa_version(void);         /* major * 10000 + minor * 100 + patch */

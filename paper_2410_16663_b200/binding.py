@@ -77,6 +77,8 @@ lib.fa_forward_host_staging_bytes.restype = _sz
 lib.fa_forward_host_staging_bytes.argtypes = [_i, _i, _i, _i, _i, _i]
 lib.fa_device_status.restype = _i
 lib.fa_device_status.argtypes = [ctypes.POINTER(ctypes.c_uint * 2)]
+lib.fa_selftest_wait.restype = _i
+lib.fa_selftest_wait.argtypes = [ctypes.c_uint, _p, _p]
 lib.fa_strerror.restype = ctypes.c_char_p
 lib.fa_strerror.argtypes = [_i]
 lib.fa_version.restype = _i
@@ -86,7 +88,7 @@ FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
            "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
-           "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_strerror",
+           "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_selftest_wait", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
 
@@ -306,6 +308,13 @@ def fa_forward_host(q_host, k_host, v_host, o_host, lse_host, causal: bool, scal
                              Hkv, Sq, Skv, d, int(bool(causal)), float(scale), dt, _ptr(staging),
                              staging.numel() * staging.element_size(), _stream())
     return _check(rc, "fa_forward_host", raise_on_error)
+
+
+def fa_selftest_wait(limit_us: int, gave_up, raise_on_error: bool = True) -> int:
+    """``fa_selftest_wait``: one CTA runs a bounded wait that cannot be satisfied; ``gave_up`` is a zeroed
+    uint32/int32 device tensor of one element that ends up holding the number of threads that gave up."""
+    rc = lib.fa_selftest_wait(int(limit_us), _ptr(gave_up), _stream())
+    return _check(rc, "fa_selftest_wait", raise_on_error)
 
 
 def fa_device_status():

@@ -297,6 +297,9 @@ struct HostPipe {
     cudaStream_t in = nullptr, out = nullptr;
     cudaEvent_t start = nullptr, finish = nullptr, in_done[kHostParts] = {}, fwd_done[kHostParts] = {};
     bool ready = false;
+    // held by fa_forward_host from its first event record to its last wait: the events are shared
+    // by every call on the device, so two host threads must not interleave their enqueue sequences
+    std::mutex enqueue;
 };
 HostPipe* host_pipe() {
     constexpr int kMaxDev = 64;
@@ -486,12 +489,10 @@ size_t fa_decode_append_workspace_bytes(int B, int Sq, int Hq, int Hkv, int Skv_
 }  // extern "C"
 
 namespace {
-// Decode over a contiguous cache (block_table == nullptr; k_cache, v_cache [B,Skv_max,Hkv,128])
-// or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
-int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
-                int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
-                void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1,
-                bool bf16 = false) {
+// The argument checks every 16-bit decode entry point shares, in the order the header documents
+// (shape, unsupported, NULL, alignment); no CUDA call.  B == 0 passes: the caller returns FA_OK.
+int decode_check_args(const void* q, const void* k_cache, const void* v_cache, const void* o, const int* seqlens_k,
+                      int B, int Hq, int Hkv, int Skv_max, int d, float scale, int Sq) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0 || Sq < 1) return FA_ERR_SHAPE;
     if (Sq > 64 || Sq > Skv_max) return FA_ERR_UNSUPPORTED;   // several query rows are the LAST rows of the cache
     if (Hq % Hkv) return FA_ERR_SHAPE;
@@ -501,11 +502,23 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     if (B == 0) return FA_OK;
     if (!q || !o || !seqlens_k) return FA_ERR_NULL;
     if (Skv_max > 0 && (!k_cache || !v_cache)) return FA_ERR_NULL;
-    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(workspace))
-        return FA_ERR_ALIGN;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o)) return FA_ERR_ALIGN;
+    return FA_OK;
+}
+
+// Decode over a contiguous cache (block_table == nullptr; k_cache, v_cache [B,Skv_max,Hkv,128])
+// or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
+int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
+                int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
+                void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1,
+                bool bf16 = false) {
+    int rc = decode_check_args(q, k_cache, v_cache, o, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, Sq);
+    if (rc) return rc;
+    if (B == 0) return FA_OK;
+    if (!aligned16(workspace)) return FA_ERR_ALIGN;
     const size_t need = fa_decode_append_workspace_bytes(B, Sq, Hq, Hkv, Skv_max, d);
     if (need > 0 && (!workspace || workspace_bytes < need)) return FA_ERR_WORKSPACE;
-    int rc = check_device();
+    rc = check_device();
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
@@ -708,13 +721,15 @@ static __device__ __align__(256) unsigned char g_decode_scratch[FA_DECODE_NOALLO
 int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
                       const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
                       void* stream) {
-    // sizes first: nothing CUDA-related happens for a problem the fixed scratch cannot hold
-    if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
-    if (Hq % Hkv) return FA_ERR_SHAPE;
-    if (d != 128) return FA_ERR_UNSUPPORTED;
+    // every argument check of fa_decode first, with the same codes in the same order, then the size
+    // limit of the fixed scratch: nothing CUDA-related happens for a call that is going to be refused
+    int rc = decode_check_args(q, k_cache, v_cache, o, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, 1);
+    if (rc) return rc;
+    if (B == 0) return FA_OK;
     if (fa_decode_workspace_bytes(B, Hq, Hkv, Skv_max, d) > (size_t)FA_DECODE_NOALLOC_BYTES)
         return FA_ERR_WORKSPACE;
-    if (B == 0) return FA_OK;
+    rc = check_device();   // a GPU this library has no code for is FA_ERR_DEVICE, not a failed symbol lookup
+    if (rc) return rc;
     constexpr int kMaxDevices = 64;
     static void* scratch_of_device[kMaxDevices] = {nullptr};
     int dev = 0;
@@ -772,6 +787,7 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
     // `stream`, and `stream` waits for the last copy out.
     HostPipe* hp = host_pipe();
     if (!hp) return FA_ERR_CUDA;
+    std::lock_guard<std::mutex> enqueue_lock(hp->enqueue);
     const int parts = B < kHostParts ? B : kHostParts;
     if ((e = cudaEventRecord(hp->start, st)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return cuda_fail(e);
@@ -822,6 +838,17 @@ int fa_device_status(unsigned int detail[2]) {
     e = cudaMemcpyToSymbol(fa::g_status, z, sizeof z);
     if (e != cudaSuccess) return cuda_fail(e);
     return FA_ERR_TIMEOUT;
+}
+
+int fa_selftest_wait(unsigned int limit_us, unsigned int* gave_up, void* stream) {
+    if (!gave_up) return FA_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(gave_up) & 3u) return FA_ERR_ALIGN;
+    if (limit_us == 0 || limit_us > 100000u) return FA_ERR_UNSUPPORTED;   // at most a tenth of a second
+    int rc = check_device();
+    if (rc) return rc;
+    fa::fa_selftest_wait_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(1000ull * limit_us, gave_up);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
 const char* fa_strerror(int code) {

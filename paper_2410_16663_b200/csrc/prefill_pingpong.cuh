@@ -277,7 +277,10 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
 // become (row inside the page, page).  The page of tile j + 1 is looked up before the loader
 // waits for tile j's ring slot, so that the table read is off the path that refills a slot.
 template <bool kVarlen>
-__device__ __forceinline__ int pp_page_of(const FwdParams& p, int b, int j, int n) {
+__device__ __forceinline__ int pp_page_of(const FwdParams& p, int b, int j, int n, int Skv) {
+    // a sequence without keys still runs one (fully masked) step; it has no table entry to read:
+    // page -1 is outside the tensor map, so the loads of that step deliver zeros
+    if (kVarlen && p.block_table != nullptr && Skv == 0) return -1;
     if (kVarlen && p.block_table != nullptr && j < n) {
         // (volatile: issued here, ahead of the wait that follows, not where the value is used)
         int page;
@@ -316,9 +319,9 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
         load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
                        kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
-        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n);
+        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n, it.Skv);
         for (int j = 0; j < it.n; ++j, ring.next()) {
-            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n);
+            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
@@ -340,9 +343,9 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
     while (items.next(p, total_items)) {
         const int ord = items.ord;
         const PpItem& it = items.it;
-        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n);
+        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n, it.Skv);
         for (int j = 0; j < it.n; ++j, ring.next()) {
-            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n);
+            const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
             mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
@@ -362,7 +365,7 @@ __device__ __forceinline__ bool pp_warp_wait(uint32_t bar, uint32_t parity, vola
 }
 
 // One thread of a softmax warpgroup: its state across the steps of an item, and the step.
-template <typename T>
+template <typename T, bool kVarlen>
 struct PpSoftmax {
     // fixed for the kernel
     uint32_t bar0;
@@ -373,6 +376,8 @@ struct PpSoftmax {
     uint32_t tO, tS, tP;    // this warp's lane quarter of O, S_w, P_w in tensor memory
     float scale_log2;
     int causal, Skv, off;
+    uint32_t sV;            // V ring in shared memory (packed batches: see the end of step())
+    int r;                  // this thread's row of the tile
     // per item
     int row;                // query row of this thread
     float l_part;           // row sum over this warpgroup's steps, relative to m_loc
@@ -473,6 +478,23 @@ struct PpSoftmax {
             f2_unpack(lb, b0, b1);
             l_part += (a0 + a1) + (b0 + b1);
         }
+        if (kVarlen && (kMasked == 1 || (kMasked == 2 && masked)) && Skv - j * kTile < kTile) {
+            // Packed batches, the tile that holds a sequence's last key: the rows of V after it
+            // belong to the next sequence, or to the unused rest of a page, and may hold anything.
+            // Their probabilities are exact zeros, but 0 * NaN would still poison O, so those
+            // rows are cleared in shared memory before P V of this step may start (a contiguous
+            // tensor gets the same from the zero fill of its TMA loads).  Thread r owns key row r:
+            // its 256 bytes are one 128-byte line in each half of the tile, whatever the swizzle.
+            static_assert(kPpNV == 2, "the V slot of step g is taken to be g & 1");
+            if (!pp_warp_wait(pp_bar(bar0, ppb::v_full + w), (g >> 1) & 1, abort_flag, 124 + w)) return false;
+            if (r >= Skv - j * kTile) {
+                const uint32_t line = sV + (uint32_t)w * kTileBytes + (uint32_t)r * 128u;
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(line + (uint32_t)(c >> 3) * kHalfBytes + (uint32_t)(c & 7) * 16u), "r"(0u) : "memory");
+            }
+            fence_proxy_async_smem();
+        }
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(pp_bar(bar0, ppb::p_full + w));
@@ -543,7 +565,9 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t tS = tmem_base + lane_sel + 128 + 128 * w;
         const uint32_t tP = tmem_base + lane_sel + 384 + 64 * w;
         const float scale_log2 = p.scale_log2;
-        PpSoftmax<T> sm;
+        PpSoftmax<T, kVarlen> sm;
+        sm.sV = sV;
+        sm.r = r;
         sm.bar0 = bar0;
         sm.abort_flag = abort_flag;
         sm.m_mine = &ss.m_xch[w][r];

@@ -75,8 +75,8 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 // Waits until the barrier's phase with the given parity has completed.  Gives up after
 // kWaitLimitNs or as soon as another thread of the CTA has given up (abort flag), records
 // the location, and returns false; the caller then leaves its loop and goes to teardown.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
-                                          volatile uint32_t* abort_flag, unsigned int where) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                              unsigned int where, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     uint32_t spins = 0;
@@ -84,13 +84,37 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0xffu) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1u;
                 record_timeout(where);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
+                                          volatile uint32_t* abort_flag, unsigned int where) {
+    return mbar_wait_for(bar, parity, abort_flag, where, kWaitLimitNs);
+}
+
+// Self-test of the give-up path above (fa_selftest_wait): one CTA waits, with a short limit, on a
+// barrier that is one arrival short of completing its phase and that nothing will ever complete.
+// The wait must run out, one thread records the location, the others see the abort flag, and
+// every thread returns normally.  gave_up counts the threads whose wait returned false.
+constexpr unsigned int kSelftestWhere = 990;
+__global__ void fa_selftest_wait_kernel(unsigned long long limit_ns, unsigned int* gave_up) {
+    __shared__ __align__(8) uint64_t bar_storage;
+    __shared__ uint32_t abort_flag;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 2);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_arrive(bar);   // the second arrival never comes
+    const bool ok = mbar_wait_for(bar, 0, &abort_flag, kSelftestWhere, limit_ns);
+    if (!ok) atomicAdd(gave_up, 1u);
 }
 
 // ------------------------------------------------------------------ proxies / fences

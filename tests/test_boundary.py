@@ -267,3 +267,11 @@ def test_product_never_imports_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in text and "oracle/" not in text, f
+
+
+def test_selftest_wait_validates_before_any_cuda_call(fa):
+    c = torch.zeros(4, dtype=torch.int32)
+    assert fa.lib.fa_selftest_wait(1000, None, None) == fa.FA_ERR_NULL
+    assert fa.lib.fa_selftest_wait(1000, c.data_ptr() + 2, None) == fa.FA_ERR_ALIGN
+    assert fa.lib.fa_selftest_wait(0, c.data_ptr(), None) == fa.FA_ERR_UNSUPPORTED
+    assert fa.lib.fa_selftest_wait(100001, c.data_ptr(), None) == fa.FA_ERR_UNSUPPORTED

@@ -270,13 +270,17 @@ def test_closed_form_identical_keys_on_gpu(fa):
 
 
 # ------------------------------------------------------------------ benchmark-size configs, sampled rows
-def sampled_case(fa, cfg, n_random, pairs=None):
+def sampled_case(fa, cfg, n_random, pairs=None, cross_check=False):
     q, k, v = synth.prefill_inputs(cfg, DEV)
-    o = torch.empty_like(q)
-    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=DEV)
+    # outputs start as NaN inside NaN guard bands: an element no work item wrote stays NaN
+    o, chk_o = guard_alloc(tuple(q.shape), q.dtype, DEV)
+    lse, chk_l = guard_alloc((cfg.B, cfg.Hq, cfg.Sq), torch.float32, DEV)
     fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)    # the launch configuration bench.py times
     torch.cuda.synchronize()
     check_status(fa)
+    chk_o()
+    chk_l()
+    assert not torch.isnan(o).any() and not torch.isnan(lse).any(), f"{cfg.name}: an output element was never written"
     assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
     rows = synth.sample_rows(cfg, n_random, seed=cfg.seed + 99, pairs=pairs)
     bf16 = cfg.dtype == "bf16"
@@ -288,22 +292,51 @@ def sampled_case(fa, cfg, n_random, pairs=None):
     assert_close_to_oracle(o_s, l_s, o_ref, l_ref, stored_bf16=bf16, p_absv=absv, what=cfg.name)
     if bf16:
         # gate on the accumulator through the fp32-output mode
-        o32 = torch.empty(cfg.B, cfg.Sq, cfg.Hq, cfg.d, dtype=torch.float32, device=DEV)
-        fa.fa_forward_ex(q, k, v, o32, lse, cfg.causal, cfg.scale)
+        o32 = torch.full((cfg.B, cfg.Sq, cfg.Hq, cfg.d), float("nan"), dtype=torch.float32, device=DEV)
+        lse32 = torch.full_like(lse, float("nan"))
+        fa.fa_forward_ex(q, k, v, o32, lse32, cfg.causal, cfg.scale)
         torch.cuda.synchronize()
         check_status(fa)
-        assert_close_to_oracle(o32[idx[:, 0], idx[:, 2], idx[:, 1]], lse[idx[:, 0], idx[:, 1], idx[:, 2]],
+        assert not torch.isnan(o32).any() and not torch.isnan(lse32).any()
+        assert_close_to_oracle(o32[idx[:, 0], idx[:, 2], idx[:, 1]], lse32[idx[:, 0], idx[:, 1], idx[:, 2]],
                                o_ref, l_ref, p_absv=absv, what=cfg.name + " fp32-out")
+    if cross_check:
+        whole_tensor_cross_check(fa, cfg, q, k, v, o, lse)
     return len(rows)
 
 
+def whole_tensor_cross_check(fa, cfg, q, k, v, o, lse):
+    """Every element of the default kernel's O and LSE against a second, much simpler kernel.
+
+    The oracle can only afford sampled rows at these sizes; the simple kernel (one CTA per query
+    tile, every stage sequential, P through shared memory) is itself compared with the oracle at
+    every element on the small shapes above, so agreement with it over the whole tensor covers the
+    rows the sample missed.  Both kernels accumulate in fp32 and differ only in summation order and
+    in the reference the exponentials are taken against, so the fp32 outputs are compared at the
+    oracle tolerances and the stored 16-bit outputs with one rounding step of the format on top."""
+    o2 = torch.full((cfg.B, cfg.Sq, cfg.Hq, cfg.d), float("nan"), dtype=torch.float32, device=DEV)
+    l2 = torch.full_like(lse, float("nan"))
+    fa.fa_forward_ex(q, k, v, o2, l2, cfg.causal, cfg.scale, variant=2)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert not torch.isnan(o2).any() and not torch.isnan(l2).any()
+    ulp = 2.0 ** -8 if cfg.dtype == "bf16" else 2.0 ** -11
+    worst_o, worst_l = 0.0, 0.0
+    for b in range(cfg.B):                     # batch by batch: bounds the temporaries
+        diff = (o[b].float() - o2[b]).abs() - ulp * o2[b].abs()
+        worst_o = max(worst_o, float(diff.max()))
+        worst_l = max(worst_l, float((lse[b] - l2[b]).abs().max()))
+    assert worst_o <= TOL_O, f"{cfg.name}: whole-tensor max(|dO| - one rounding step) = {worst_o:.3e}"
+    assert worst_l <= TOL_LSE, f"{cfg.name}: whole-tensor max|dLSE| = {worst_l:.3e}"
+
+
 def test_c2_llama7b_prefill_sampled(fa):
-    assert sampled_case(fa, synth.C2, 80) >= 256
+    assert sampled_case(fa, synth.C2, 80, cross_check=True) >= 256
 
 
 @pytest.mark.parametrize("s", [8192, 32768])
 def test_c3_long_context_sampled(fa, s):
-    assert sampled_case(fa, synth.C3[s], 80) >= 256
+    assert sampled_case(fa, synth.C3[s], 80, cross_check=(s == 8192)) >= 256
 
 
 @pytest.mark.parametrize("s", [131072, 262144])
@@ -313,8 +346,8 @@ def test_c3_very_long_context_sampled(fa, s):
 
 
 def test_c4_gqa_sampled(fa):
-    assert sampled_case(fa, synth.C4, 64) >= 256
-    assert sampled_case(fa, synth.C4_NC, 64) >= 256
+    assert sampled_case(fa, synth.C4, 64, cross_check=True) >= 256
+    assert sampled_case(fa, synth.C4_NC, 64, cross_check=True) >= 256
 
 
 # ------------------------------------------------------------------ head dimension 64
@@ -486,11 +519,13 @@ def test_varlen_equal_lengths_match_the_batched_call_bit_for_bit(fa):
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
 def test_varlen_over_a_paged_cache(fa, causal, dtype):
     # chunked prefill against a page pool: each sequence's queries are its last rows, its keys sit
-    # in 128- or 256-key pages handed out in random order; unused pages hold NaN (a wrong page
-    # would show), the unused rows of a last page zeros (the contract: finite).  Lengths: a key
-    # count that ends exactly on a page, one key, more pages than queries, queries = keys
-    lq = (70, 1, 130, 300, 128, 5)
-    lk = (700, 1, 130, 1000, 256, 1500)
+    # in 128- or 256-key pages handed out in random order; unused pages and the rows of a last page
+    # past the end of its sequence hold NaN (serving systems do not clear fresh pages: a wrong page
+    # would show, and so would a product with a row that is not the sequence's).  Lengths: a key
+    # count that ends exactly on a page, one key, more pages than queries, queries = keys, and a
+    # sequence with queries but no keys, whose table row is never to be read and holds garbage
+    lq = (70, 1, 130, 300, 128, 5, 40)
+    lk = (700, 1, 130, 1000, 256, 1500, 0)
     for page in (128, 256):
         cfg = synth.VarlenConfig("t", 4, 2, lq, lk, dtype=dtype, causal=causal, seed=700 + page)
         q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
@@ -501,10 +536,8 @@ def test_varlen_over_a_paged_cache(fa, causal, dtype):
             vc[b, :lk[b]] = v[int(cu_k[b]):int(cu_k[b + 1])]
         sk = torch.tensor(lk, dtype=torch.int32)
         kp, vp, table = synth.paged_cache(kc, vc, sk, page, seed=cfg.seed, spare_pages=3, poison=True)
-        for b in range(B):      # the rows of a sequence's last page past its end: finite
-            last = (lk[b] - 1) // page
-            kp[int(table[b, last]), lk[b] - last * page:] = 0
-            vp[int(table[b, last]), lk[b] - last * page:] = 0
+        assert torch.isnan(vp[int(table[0, (lk[0] - 1) // page]), -1]).all()     # page tails stay poisoned
+        table[6, :] = torch.tensor([0x7ffffff0, -12345] * table.shape[1])[:table.shape[1]]
         o_ref, l_ref = oracle.attention_varlen_paged(q, kp, vp, table, cu_q, sk, causal, cfg.scale)
         o_chk, l_chk = oracle.attention_varlen(q, k, v, cu_q, cu_k, causal, cfg.scale)
         assert torch.equal(o_ref, o_chk) and torch.equal(l_ref, l_chk)
@@ -985,3 +1018,29 @@ def test_forward_host_entry_batch_parts(fa, B):
         assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=True, p_absv=absv, what=f"host entry B={B}")
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
+
+
+# ------------------------------------------------------------------ the give-up path of the bounded waits
+def test_a_wait_that_cannot_be_satisfied_gives_up_and_is_reported(fa):
+    # every device-side wait of the library is bounded; this runs the give-up path on purpose, in
+    # a kernel made for it: 64 threads wait at most 2 ms on a barrier that stays one arrival short.
+    # The wait expires by itself (nothing traps, faults or spins for ever), every thread returns,
+    # the status word names the place once, and the device is as usable as before.
+    check_status(fa)
+    gave_up = torch.zeros(1, dtype=torch.int32, device=DEV)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    fa.fa_selftest_wait(2000, gave_up)
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(gave_up.item()) == 64
+    assert 1.5 <= t0.elapsed_time(t1) <= 500.0           # it waited about the limit, not for ever
+    rc, where, blk = fa.fa_device_status()
+    assert rc == fa.FA_ERR_TIMEOUT and where == 990 and blk == 0
+    assert fa.fa_device_status()[0] == fa.FA_OK          # reported once, then cleared
+    # and an ordinary forward right after it is still correct
+    c = synth.C1
+    q, k, v = synth.prefill_inputs(c, "cpu")
+    o_ref, l_ref = oracle.attention_full(q, k, v, c.causal, c.scale)
+    o, lse = run_forward(fa, q.to(DEV), k.to(DEV), v.to(DEV), c.causal, c.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what="C1 after the self-test")
