@@ -196,6 +196,8 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.cls_log2 = 0;  // set by the ping-pong launcher
     fp.by_class.set(1);
     fp.by_lastcls.set(1);
+    fp.rounds_per_head = 0;
+    fp.by_rph.set(1);
     fp.cu_q = nullptr;
     fp.cu_k = nullptr;
     fp.total_q = 0;
@@ -415,6 +417,8 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     fp.cls_log2 = 0;
     fp.by_class.set(1);
     fp.by_lastcls.set(1);
+    fp.rounds_per_head = 0;
+    fp.by_rph.set(1);
     fp.cu_q = cu_seqlens_q;
     fp.cu_k = cu_seqlens_k;
     fp.total_q = total_q;

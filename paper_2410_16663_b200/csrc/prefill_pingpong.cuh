@@ -95,19 +95,24 @@ struct PpItem {
 // of its sequence (every role skips it), and a live item visits at least one kv tile (so that
 // rows without any visible key are still written, as zeros).
 template <bool kVarlen>
-__device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
-    PpItem it;
+__device__ __forceinline__ void pp_class_order(const FwdParams& p, int idx, int& bh, int& qt) {
     int c, rem;  // class, index inside the class
     p.by_class.divmod(idx, c, rem);
     const int first = c << p.cls_log2;  // tiles in the classes before this one
-    int bh, j;
+    int j;
     if (p.n_qtiles - first >= (1 << p.cls_log2)) {
         bh = rem >> p.cls_log2;
         j = rem & ((1 << p.cls_log2) - 1);
     } else {
         p.by_lastcls.divmod(rem, bh, j);
     }
-    const int qt = p.n_qtiles - 1 - first - j;
+    qt = p.n_qtiles - 1 - first - j;
+}
+
+// The work item that is query tile qt of (batch, head) pair bh.
+template <bool kVarlen>
+__device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int bh, int qt) {
+    PpItem it;
     p.by_hq.divmod(bh, it.b, it.h);
     it.hk = p.by_group.div(it.h);
     it.q0 = qt * kTile;
@@ -131,6 +136,16 @@ __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int idx) {
 // The items of this CTA in order.  `ord` counts the items the CTA works on (it selects the
 // double buffers); with variable-length batches the items past the end of their sequence are
 // passed over, identically in every role.
+// Very long sequences (rounds_per_head > 0; one head's K and V no longer fit in L2) go head by
+// head, and every head takes a whole number of rounds of the grid: in round r of a head CTA b
+// takes the head's (r * gridDim.x + b)-th longest tile -- b counted from the other end in every
+// second round, and the other way around for every second head -- and nothing if the head has no
+// such tile (only in a head's last round, whose items are its shortest).  The CTAs of a round
+// then all walk the same head's keys from the first on, a few dozen tiles apart at most, and
+// stay together from head to head, so a K or V tile is fetched from HBM once per round and
+// found in L2 by everyone else.  (Without the padding a round straddles two heads, the CTAs
+// that get the next head's longest tiles fall a thousand tiles behind the others, and the
+// groups, each walking the head on its own, fetch everything several times.)
 template <bool kVarlen>
 struct PpItems {
     int round = -1, ord = -1;
@@ -138,9 +153,22 @@ struct PpItems {
     __device__ __forceinline__ bool next(const FwdParams& p, int total_items) {
         for (;;) {
             ++round;
+            if (!kVarlen && p.rounds_per_head > 0) {
+                int bh, r;
+                p.by_rph.divmod(round, bh, r);
+                if (bh >= p.B * p.Hq) return false;
+                const int g = gridDim.x, b = blockIdx.x;
+                const int j = r * g + (((r + bh) & 1) ? (g - 1 - b) : b);
+                if (j >= p.n_qtiles) continue;
+                it = pp_decode_item<kVarlen>(p, bh, p.n_qtiles - 1 - j);
+                ++ord;
+                return true;
+            }
             const int idx = item_of_round(round, total_items);
             if (idx >= total_items) return false;
-            it = pp_decode_item<kVarlen>(p, idx);
+            int bh, qt;
+            pp_class_order<kVarlen>(p, idx, bh, qt);
+            it = pp_decode_item<kVarlen>(p, bh, qt);
             if (!kVarlen || it.n > 0) {
                 ++ord;
                 return true;
@@ -812,6 +840,14 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
         while ((grid >> cls_log2) * head_bytes > budget && (2 << cls_log2) <= cap) ++cls_log2;
 #endif
         while (cls_log2 > 0 && (1 << cls_log2) > fp.n_qtiles) --cls_log2;
+    }
+    // From three rounds per head on (56K keys on 148 SMs) and once a head's K and V are past what
+    // L2 keeps, the head-by-head order with whole rounds per head (see PpItems); the empty slots of
+    // a head's last round cost little there because its items are the head's shortest.
+    const double kv_bytes_per_head = 2.0 * fp.Skv * 128 * 2;
+    if (!varlen && fp.n_qtiles >= 3 * grid && kv_bytes_per_head > 24.0 * 1024 * 1024) {
+        fpc.rounds_per_head = (fp.n_qtiles + grid - 1) / grid;
+        fpc.by_rph.set(fpc.rounds_per_head);
     }
     fpc.cls_log2 = cls_log2;
     const long long class_items = ((long long)fp.B * fp.Hq) << cls_log2;  // > total only for a single class

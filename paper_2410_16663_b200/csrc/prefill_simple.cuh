@@ -52,6 +52,10 @@ struct FwdParams {
     // the size of the last (possibly smaller) class
     int cls_log2;
     FastDiv by_class, by_lastcls;
+    // head-by-head order of the ping-pong kernel for very long sequences (see PpItems::next):
+    // every head takes rounds_per_head whole rounds of the grid; 0 = the class order above
+    int rounds_per_head;
+    FastDiv by_rph;
     // packed variable-length batch (ping-pong kernel only; nullptr otherwise): sequence b owns
     // rows [cu_q[b], cu_q[b+1]) of q and o and rows [cu_k[b], cu_k[b+1]) of k and v; Sq and Skv
     // above are then the longest sequence's, and lse is [Hq, total_q]

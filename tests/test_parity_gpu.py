@@ -345,6 +345,18 @@ def test_c3_very_long_context_sampled(fa, s):
     assert sampled_case(fa, cfg, 20, pairs=[(0, 0), (0, 13), (0, 31)]) >= 64
 
 
+@pytest.mark.parametrize("causal", [True, False])
+def test_long_context_item_order_with_whole_rounds_per_head(fa, causal):
+    # from about 56K keys on (148 SMs) the ping-pong kernel goes head by head and gives every head
+    # a whole number of rounds of the grid, the last one partly empty: 469 query tiles are three
+    # full rounds and one of 25 items, walked in opposite directions for odd and even heads.  A
+    # ragged last tile, GQA, every output element written exactly once (NaN pre-fill), sampled
+    # rows of every head against the oracle.
+    cfg = synth.PrefillConfig("order-60K", 1, 4, 2, 60000, 60000, dtype="bf16", causal=causal,
+                              seed=1050 + int(causal))
+    assert sampled_case(fa, cfg, 12, pairs=[(0, 0), (0, 1), (0, 2), (0, 3)]) >= 64
+
+
 def test_c4_gqa_sampled(fa):
     assert sampled_case(fa, synth.C4, 64, cross_check=True) >= 256
     assert sampled_case(fa, synth.C4_NC, 64, cross_check=True) >= 256
