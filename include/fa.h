@@ -102,6 +102,29 @@ typedef struct fa_params {
 int fa_forward_ex(const fa_params* p, void* stream);
 
 /*
+ * Forward with 8-bit operands (Appendix D.2 evaluates the operator with 8-bit operands; the paper
+ * names no format, scales or granularity, so this is the reading taken here): the computation of
+ * fa_forward with Q = q_scale * q, K = k_scale * k, V = v_scale * v, where q [B,Sq,Hq,d] and
+ * k, v [B,Skv,Hkv,d] hold FP8 e4m3 bit patterns (1 sign, 4 exponent, 3 mantissa bits, bias 7, no
+ * infinities; one byte per element, contiguous, 16-byte aligned) and the three factors are
+ * positive and finite, one per tensor.  Both products run on the tensor cores with 8-bit
+ * operands and fp32 accumulation; for the second one the probabilities are rounded to e4m3 as
+ * well (after a fixed power-of-two factor that is divided out again), which is the one place
+ * where this entry point is less accurate than the 16-bit ones: a probability carries a relative
+ * rounding of up to 2^-4, so O_i moves by up to 2^-4 * sum_j P_ij |V_j| (plus a much smaller
+ * absolute term from probabilities below the format's normal range).  LSE is computed from the
+ * unrounded probabilities and is as accurate as fa_forward's.
+ *   o [B,Sq,Hq,d] of o_dtype (FA_DTYPE_FP16 or FA_DTYPE_BF16), lse [B,Hq,Sq] float or NULL;
+ *   d must be 128.  Everything else (mask, head mapping, no-ops, aliasing) as for fa_forward.
+ *   No NaN pattern (0x7f, 0xff) may occur in q, k, v.
+ * Errors: as fa_forward; FA_ERR_UNSUPPORTED also for a factor that is not positive and finite
+ * and for an o_dtype other than the two 16-bit types.
+ */
+int fa_forward_fp8(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq,
+                   int Hkv, int Sq, int Skv, int d, int causal, float scale, float q_scale,
+                   float k_scale, float v_scale, int o_dtype, void* stream);
+
+/*
  * Forward over a packed batch of sequences of different lengths (the batched serving runs of the
  * evaluation section process requests of unequal length together): the same computation as
  * fa_forward, sequence by sequence.  Sequence b owns rows [cu_seqlens_q[b], cu_seqlens_q[b+1])

@@ -255,6 +255,25 @@ def e4m3_to_float64(bits):
     return torch.where(nan, torch.full_like(val, float("nan")), val)
 
 
+def attention_fp8(q_bits, k_bits, v_bits, causal: bool, scale: float, q_scale: float, k_scale: float,
+                  v_scale: float, rows=None, abs_v: bool = False, nthreads: int = 0):
+    """Standard attention on FP8 e4m3 operands (Appendix D.2 runs the operator on 8-bit
+    operands): ``attention_full`` -- or ``attention_rows`` when ``rows`` is given -- on
+    Q = q_scale * value(q_bits), K = k_scale * value(k_bits), V = v_scale * value(v_bits), all
+    widened exactly and evaluated in float64.  Nothing here is rounded to 8 bits: the
+    probabilities stay float64, so a kernel that rounds them differs by what that rounding costs.
+    ``abs_v`` evaluates with |V| in place of V (the weight sum_j P_ij |V_j| that bounds it).
+    ``*_bits``: uint8 ``[B,S,H,d]``."""
+    q = (e4m3_to_float64(q_bits) * float(q_scale)).contiguous()
+    k = (e4m3_to_float64(k_bits) * float(k_scale)).contiguous()
+    v = (e4m3_to_float64(v_bits) * float(v_scale)).contiguous()
+    if abs_v:
+        v = v.abs()
+    if rows is None:
+        return attention_full(q, k, v, causal, scale, nthreads)
+    return attention_rows(q, k, v, causal, scale, rows, nthreads)
+
+
 def decode_fp8(q, k_bits, v_bits, seqlens, scale: float, k_scale: float, v_scale: float, nthreads: int = 0):
     """Decode-stage attention over an FP8 e4m3 cache: ``decode`` on K = k_scale * value(k_bits),
     V = v_scale * value(v_bits), evaluated in float64 (Appendix D.2 runs the operator on 8-bit

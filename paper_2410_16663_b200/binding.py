@@ -41,6 +41,8 @@ lib.fa_forward_bf16.restype = _i
 lib.fa_forward_bf16.argtypes = _FWD_ARGS
 lib.fa_forward_ex.restype = _i
 lib.fa_forward_ex.argtypes = [ctypes.POINTER(fa_params), _p]
+lib.fa_forward_fp8.restype = _i
+lib.fa_forward_fp8.argtypes = [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _f, _f, _f, _i, _p]
 lib.fa_decode.restype = _i
 lib.fa_decode.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_workspace_bytes.restype = _sz
@@ -86,7 +88,7 @@ lib.fa_last_cuda_error.restype = _i
 
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
-EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_decode", "fa_decode_workspace_bytes",
+EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_forward_fp8", "fa_decode", "fa_decode_workspace_bytes",
            "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_selftest_wait", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
@@ -152,6 +154,18 @@ def fa_forward_ex(q, k, v, o, lse, causal: bool, scale: float, variant: int = 0,
     p.variant = int(variant)
     rc = lib.fa_forward_ex(ctypes.byref(p), _stream())
     return _check(rc, "fa_forward_ex", raise_on_error)
+
+
+def fa_forward_fp8(q, k, v, o, lse, causal: bool, scale: float, q_scale: float, k_scale: float, v_scale: float,
+                   raise_on_error: bool = True) -> int:
+    """``fa_forward_fp8``: q [B,Sq,Hq,d], k, v [B,Skv,Hkv,d] contiguous device tensors of FP8 e4m3
+    (``torch.float8_e4m3fn`` or uint8 bit patterns) with one factor each; o fp16 or bf16."""
+    B, Sq, Hq, d = q.shape
+    _, Skv, Hkv, _ = k.shape
+    dt = FA_DTYPE_BF16 if o.dtype == torch.bfloat16 else FA_DTYPE_FP16
+    rc = lib.fa_forward_fp8(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Hq, Hkv, Sq, Skv, d, int(bool(causal)),
+                            float(scale), float(q_scale), float(k_scale), float(v_scale), dt, _stream())
+    return _check(rc, "fa_forward_fp8", raise_on_error)
 
 
 def fa_forward_varlen(q, k, v, o, lse, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int,

@@ -198,6 +198,7 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.by_lastcls.set(1);
     fp.rounds_per_head = 0;
     fp.by_rph.set(1);
+    fp.out_scale = 1.f;
     fp.cu_q = nullptr;
     fp.cu_k = nullptr;
     fp.total_q = 0;
@@ -368,6 +369,79 @@ int fa_forward_bf16(const void* q, const void* k, const void* v, void* o, float*
     return forward_plain(q, k, v, o, lse, B, Hq, Hkv, Sq, Skv, d, causal, scale, FA_DTYPE_BF16, stream);
 }
 
+int fa_forward_fp8(const void* q, const void* k, const void* v, void* o, float* lse, int B, int Hq, int Hkv, int Sq,
+                   int Skv, int d, int causal, float scale, float q_scale, float k_scale, float v_scale, int o_dtype,
+                   void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Sq < 0 || Skv < 0 || d <= 0) return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (o_dtype != FA_DTYPE_FP16 && o_dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
+    if (!(q_scale > 0.f) || isinf(q_scale) || !(k_scale > 0.f) || isinf(k_scale) || !(v_scale > 0.f) || isinf(v_scale))
+        return FA_ERR_UNSUPPORTED;
+    if (causal && Sq > Skv) return FA_ERR_UNSUPPORTED;
+    if (Hq > 65535 || B > 65535) return FA_ERR_UNSUPPORTED;
+    if (B == 0 || Sq == 0) return FA_OK;
+    if (!q || !o) return FA_ERR_NULL;
+    if (Skv > 0 && (!k || !v)) return FA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return FA_ERR_ALIGN;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return FA_ERR_ALIGN;
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf16 = o_dtype == FA_DTYPE_BF16;
+
+    fa::FwdParams fp;
+    fp.o = o;
+    fp.lse = lse;
+    fp.B = B; fp.Hq = Hq; fp.Hkv = Hkv; fp.Sq = Sq; fp.Skv = Skv;
+    fp.causal = causal ? 1 : 0;
+    // the scores are products of the stored 8-bit values: both factors go into the softmax scale
+    fp.scale_log2 = fmaxf(scale * q_scale * k_scale * 1.4426950408889634f, 1e-30f);
+    fp.o_sb = (long long)Sq * Hq * 128; fp.o_ss = (long long)Hq * 128; fp.o_sh = 128;
+    fp.o_fp32 = 0;
+    fp.o_align32 = 0;
+    fp.n_qtiles = (Sq + fa::kTile - 1) / fa::kTile;
+    fp.by_bh.set(B * Hq);
+    fp.by_hq.set(Hq);
+    fp.by_group.set(Hq / Hkv);
+    fp.by_qtiles.set(fp.n_qtiles);
+    fp.by_qpairs.set((fp.n_qtiles + 1) / 2);
+    fp.cls_log2 = 0;
+    fp.by_class.set(1);
+    fp.by_lastcls.set(1);
+    fp.rounds_per_head = 0;
+    fp.by_rph.set(1);
+    fp.out_scale = v_scale;
+    fp.cu_q = nullptr;
+    fp.cu_k = nullptr;
+    fp.total_q = 0;
+    fp.block_table = nullptr;
+    fp.seqlens_k = nullptr;
+    fp.table_stride = 0;
+    fp.page_size = 1;
+    fp.d = 128;
+    if (Skv == 0) {
+        const long long rows = (long long)B * Sq * Hq;
+        const int blocks = (int)((rows + 127) / 128 < 4096 ? (rows + 127) / 128 : 4096);
+        if (bf16) fa::fa_fill_empty_kernel<__nv_bfloat16><<<blocks, 128, 0, st>>>(fp);
+        else fa::fa_fill_empty_kernel<__half><<<blocks, 128, 0, st>>>(fp);
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    }
+    CUtensorMap tq, tk, tv, to;
+    rc = encode_map_u8(&tq, q, B, Sq, Hq, 128);
+    if (rc) return rc;
+    rc = encode_map_u8(&tk, k, B, Skv, Hkv, 128);
+    if (rc) return rc;
+    rc = encode_map_u8(&tv, v, B, Skv, Hkv, 128);
+    if (rc) return rc;
+    rc = encode_map(&to, o, B, Sq, Hq, (int64_t)Sq * Hq * 128, (int64_t)Hq * 128, 128, 32, bf16);
+    if (rc) return rc;
+    return bf16 ? fa::launch_pingpong<__nv_bfloat16, true>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
+                : fa::launch_pingpong<__half, true>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
+}
+
 int fa_forward_ex(const fa_params* p, void* stream) {
     if (!p) return FA_ERR_NULL;
     return forward_impl(*p, static_cast<cudaStream_t>(stream));
@@ -419,6 +493,7 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     fp.by_lastcls.set(1);
     fp.rounds_per_head = 0;
     fp.by_rph.set(1);
+    fp.out_scale = 1.f;
     fp.cu_q = cu_seqlens_q;
     fp.cu_k = cu_seqlens_k;
     fp.total_q = total_q;

@@ -46,6 +46,22 @@ constexpr int kPpQBufs = 2;
 constexpr bool kPpTurns = FA_PP_TURNS != 0;
 static_assert((kPpQBufs + kPpNK + kPpNV) * kTileBytes + 3072 <= 232448, "shared memory budget");
 
+// What changes with FP8 e4m3 operands (kF8; Appendix D.2 evaluates the operator with 8-bit
+// operands): a tile of 128 rows x 128 bytes is one swizzled TMA box of 16 KiB (a Q slot keeps its
+// 32 KiB, because the 16-bit output tile is staged there); one MMA covers 32 elements of the
+// contraction, so a product takes four instead of eight; the probabilities are rounded to e4m3
+// four to a 32-bit column of tensor memory, times kP8Scale so that they use the format's range:
+// with the reference max at most 2^kP8Threshold behind the row max they stay below 2^8 < 448.
+template <bool kF8>
+struct PpOperands {
+    static constexpr int kKvSlotBytes = kF8 ? 16384 : kTileBytes;   // one K or V ring slot
+    static constexpr int kQBytes = kF8 ? 16384 : kTileBytes;        // bytes a Q load delivers
+    static constexpr int kSteps = kF8 ? 4 : 8;                      // MMAs per 128 x 128 x 128 product
+    static constexpr int kPCols = kF8 ? 8 : 16;                     // tensor-memory columns of 32 probabilities
+};
+constexpr float kP8Threshold = 4.0f;   // log2 units: how far the row max may outgrow the reference (FP8)
+constexpr float kP8ScaleLog2 = 4.0f;   // log2 of the factor on the FP8 probabilities
+
 // ---- barriers: indices into one array
 namespace ppb {
 constexpr int q_full = 0;                       // [2]  TMA -> S thread
@@ -191,9 +207,9 @@ __device__ __forceinline__ float pp_row_max(const uint32_t (&s)[128]) {
 }
 
 // exp2(s * scale_log2 + neg_ms) of 32 scores -> 16 packed 16-bit pairs; adds them to (la, lb).
-template <typename T>
+template <typename T, bool kF8>
 __device__ __forceinline__ void pp_exp_chunk(const uint32_t (&s)[128], int c, uint64_t sc2, uint64_t nm2,
-                                             uint64_t& la, uint64_t& lb, uint32_t (&pk)[16]) {
+                                             uint64_t& la, uint64_t& lb, uint32_t (&pk)[PpOperands<kF8>::kPCols]) {
 #pragma unroll
     for (int i = 0; i < 32; i += 8) {
         const int e = c * 32 + i;
@@ -215,10 +231,21 @@ __device__ __forceinline__ void pp_exp_chunk(const uint32_t (&s)[128], int c, ui
         lb = f2_add(lb, f2_pack(pv[2], pv[3]));
         la = f2_add(la, f2_pack(pv[4], pv[5]));
         lb = f2_add(lb, f2_pack(pv[6], pv[7]));
+        if (kF8) {
+            pk[i / 4] = pack4_e4m3(pv[0], pv[1], pv[2], pv[3]);
+            pk[i / 4 + 1] = pack4_e4m3(pv[4], pv[5], pv[6], pv[7]);
+        } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) pk[i / 2 + q] = pack2<T>(pv[2 * q], pv[2 * q + 1]);
+            for (int q = 0; q < 4; ++q) pk[i / 2 + q] = pack2<T>(pv[2 * q], pv[2 * q + 1]);
+        }
     }
 }
+template <bool kF8>
+__device__ __forceinline__ void pp_store_p(uint32_t taddr, const uint32_t (&pk)[PpOperands<kF8>::kPCols]);
+template <>
+__device__ __forceinline__ void pp_store_p<false>(uint32_t taddr, const uint32_t (&pk)[16]) { tmem_st_x16(taddr, pk); }
+template <>
+__device__ __forceinline__ void pp_store_p<true>(uint32_t taddr, const uint32_t (&pk)[8]) { tmem_st_x8(taddr, pk); }
 
 __device__ __forceinline__ uint32_t pp_bar(uint32_t bar0, int i) { return bar0 + 8 * i; }
 
@@ -235,11 +262,12 @@ struct PpRing {
 };
 
 // The thread that issues S = Q K^T of every step.
-template <typename T, bool kTmaOut, bool kVarlen>
+template <typename T, bool kTmaOut, bool kVarlen, bool kF8>
 __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK, uint32_t tmem, const FwdParams& p,
                                          int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
-    constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, false);
+    constexpr uint32_t idesc = kF8 ? instr_desc_e4m3(128, 128, false, false) : instr_desc_f16(kBf16, 128, 128, false, false);
+    using Op = PpOperands<kF8>;
     uint32_t g = 0;
     PpRing<kPpNK> ring;
     PpItems<kVarlen> items;
@@ -256,11 +284,14 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
             // with its reference max)
             if (g >= 2 && !mbar_wait(pp_bar(bar0, ppb::m_ready + buf), ((g >> 1) - 1) & 1, abort_flag, 132)) return;
             tc_fence_after();
-            const uint32_t b_lo = desc_lo(sK + ring.slot * kTileBytes, 16);
+            const uint32_t b_lo = desc_lo(sK + ring.slot * Op::kKvSlotBytes, 16);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                const uint32_t koff = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
-                mma_ss_lo(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
+            for (int ks = 0; ks < Op::kSteps; ++ks) {
+                // one MMA takes 32 bytes of every row: 16 16-bit elements (a row of d = 128 is two
+                // 128-byte boxes) or 32 8-bit ones (one box)
+                const uint32_t koff = kF8 ? (uint32_t)(ks * 32) >> 4 : ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                if (kF8) mma_ss_lo_f8(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
+                else mma_ss_lo(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
             }
             mma_commit(pp_bar(bar0, ppb::s_full + buf));
             mma_commit(pp_bar(bar0, ppb::k_empty + ring.slot));
@@ -271,11 +302,12 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
 }
 
 // The thread that issues O += P V of every step.
-template <typename T, bool kVarlen>
+template <typename T, bool kVarlen, bool kF8>
 __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t tmem, const FwdParams& p,
                                           int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
-    constexpr uint32_t idesc = instr_desc_f16(kBf16, 128, 128, false, true);
+    constexpr uint32_t idesc = kF8 ? instr_desc_e4m3(128, 128, false, true) : instr_desc_f16(kBf16, 128, 128, false, true);
+    using Op = PpOperands<kF8>;
     uint32_t g = 0;
     PpRing<kPpNV> ring;
     PpItems<kVarlen> items;
@@ -289,11 +321,17 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
             if (j == 0 && ord > 0 && !mbar_wait(pp_bar(bar0, ppb::o_free), (ord - 1) & 1, abort_flag, 141)) return;
             if (!mbar_wait(pp_bar(bar0, ppb::p_full + buf), (g >> 1) & 1, abort_flag, 142)) return;
             tc_fence_after();
-            const uint32_t b_lo = desc_lo(sV + ring.slot * kTileBytes, kHalfBytes);  // V: N-major, 16 kv rows per step
+            // V is the N-major operand: a key is a row of 128 elements of d.  16-bit: two 128-byte
+            // column blocks kHalfBytes apart, 16 keys (2048 bytes) per MMA; 8-bit: one block, 32 keys
+            // (4096 bytes) per MMA.  Either way an MMA reads 8 columns of P.
+            const uint32_t b_lo = desc_lo(sV + ring.slot * Op::kKvSlotBytes, kHalfBytes);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ts_lo(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (2048 >> 4), idesc,
-                          (ks > 0) ? 1u : (j > 0 ? 1u : 0u));
+            for (int ks = 0; ks < Op::kSteps; ++ks) {
+                if (kF8) mma_ts_lo_f8(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (4096 >> 4), idesc,
+                                      (ks > 0) ? 1u : (j > 0 ? 1u : 0u));
+                else mma_ts_lo(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (2048 >> 4), idesc,
+                               (ks > 0) ? 1u : (j > 0 ? 1u : 0u));
+            }
             mma_commit(pp_bar(bar0, ppb::pv_done + buf));
             mma_commit(pp_bar(bar0, ppb::v_empty + ring.slot));
             if (j == it.n - 1) mma_commit(pp_bar(bar0, ppb::o_final + (ord & 1)));
@@ -329,7 +367,15 @@ __device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int page, int 
 
 // The thread that loads Q of every item and K of every step.  (Packed batches: the tensor maps
 // have one batch entry that holds every sequence back to back.)
-template <bool kVarlen>
+// One tile: two 64-element boxes of a 16-bit tensor, or one 128-byte box of an 8-bit one.
+template <bool kF8>
+__device__ __forceinline__ void pp_load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int h, int s0, int b,
+                                             uint64_t policy) {
+    if (kF8) tma_load_4d_hint(dst, tm, bar, 0, h, s0, b, policy);
+    else load_tile_hint(dst, tm, bar, h, s0, b, policy);
+}
+
+template <bool kVarlen, bool kF8>
 __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint32_t sK, const CUtensorMap* tm_q,
                                                const CUtensorMap* tm_k, const FwdParams& p, int total_items,
                                                volatile uint32_t* abort_flag) {
@@ -344,24 +390,24 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         const uint32_t qb = ord & 1;
         // passes at once the first time each buffer is used
         if (!mbar_wait(pp_bar(bar0, ppb::q_empty + qb), ((ord >> 1) & 1) ^ 1, abort_flag, 150)) return;
-        mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), kTileBytes);
-        load_tile_hint(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
+        mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), PpOperands<kF8>::kQBytes);
+        pp_load_tile<kF8>(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
                        kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
         int page = pp_page_of<kVarlen>(p, it.b, 0, it.n, it.Skv);
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
-            mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), kTileBytes);
+            mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), PpOperands<kF8>::kKvSlotBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
             pp_paged_tile<kVarlen>(p, page, j, row, slab);
             page = page_next;
-            load_tile_hint(sK + ring.slot * kTileBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
+            pp_load_tile<kF8>(sK + ring.slot * PpOperands<kF8>::kKvSlotBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }
 
 // The thread that loads V of every step.
-template <bool kVarlen>
+template <bool kVarlen, bool kF8>
 __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const CUtensorMap* tm_v, const FwdParams& p,
                                               int total_items, volatile uint32_t* abort_flag) {
     tma_prefetch_desc(tm_v);
@@ -375,11 +421,11 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
-            mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), kTileBytes);
+            mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), PpOperands<kF8>::kKvSlotBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
             pp_paged_tile<kVarlen>(p, page, j, row, slab);
             page = page_next;
-            load_tile_hint(sV + ring.slot * kTileBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
+            pp_load_tile<kF8>(sV + ring.slot * PpOperands<kF8>::kKvSlotBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }
@@ -393,8 +439,10 @@ __device__ __forceinline__ bool pp_warp_wait(uint32_t bar, uint32_t parity, vola
 }
 
 // One thread of a softmax warpgroup: its state across the steps of an item, and the step.
-template <typename T, bool kVarlen>
+template <typename T, bool kVarlen, bool kF8>
 struct PpSoftmax {
+    static_assert(!(kF8 && kVarlen), "packed batches take 16-bit operands");
+    using Op = PpOperands<kF8>;
     // fixed for the kernel
     uint32_t bar0;
     volatile uint32_t* abort_flag;
@@ -447,7 +495,7 @@ struct PpSoftmax {
         m_before = m_prev;
         // lazy reference update: the reference moves only when the row max outgrew it by more than
         // the threshold (always on the first visible score; never on -inf)
-        const bool grow = (mx - m_prev) * scale_log2 > kRescaleThreshold;
+        const bool grow = (mx - m_prev) * scale_log2 > (kF8 ? kP8Threshold : kRescaleThreshold);
         const float m_new = grow ? mx : m_prev;
         *m_mine = m_new;
         // one arrival per thread: publishes its reference max and, the scores being in registers,
@@ -457,7 +505,7 @@ struct PpSoftmax {
             if (l_part > 0.f) l_part *= fast_exp2((m_loc - m_new) * scale_log2);
             m_loc = m_new;
         }
-        const float neg_ms = -((m_new == -INFINITY) ? 0.f : m_new) * scale_log2;
+        const float neg_ms = -((m_new == -INFINITY) ? 0.f : m_new) * scale_log2 + (kF8 ? kP8ScaleLog2 : 0.f);
         const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
         uint64_t la = f2_pack(0.f, 0.f), lb = la;
         if (kPpTurns && g >= 1) {
@@ -465,9 +513,9 @@ struct PpSoftmax {
             if (!pp_warp_wait(pp_bar(bar0, ppb::p_full + (1 - w)), ((g - 1) >> 1) & 1, abort_flag, 122 + w)) return false;
         }
         {
-            uint32_t pk[16];
+            uint32_t pk[Op::kPCols];
             const bool p_free = g < 2 || mbar_test(pp_bar(bar0, ppb::pv_done + w), ((g >> 1) - 1) & 1);
-            pp_exp_chunk<T>(s, 0, sc2, nm2, la, lb, pk);
+            pp_exp_chunk<T, kF8>(s, 0, sc2, nm2, la, lb, pk);
             if (g >= 2) {
                 // O += P V of step g-2 has read this P buffer
                 if (!__all_sync(0xffffffffu, p_free) &&
@@ -492,13 +540,13 @@ struct PpSoftmax {
                     tmem_st_x16(tO + c * 16, o);
                 }
             }
-            tmem_st_x16(tP, pk);
+            pp_store_p<kF8>(tP, pk);
         }
 #pragma unroll
         for (int c = 1; c < 4; ++c) {
-            uint32_t pk[16];
-            pp_exp_chunk<T>(s, c, sc2, nm2, la, lb, pk);
-            tmem_st_x16(tP + c * 16, pk);
+            uint32_t pk[Op::kPCols];
+            pp_exp_chunk<T, kF8>(s, c, sc2, nm2, la, lb, pk);
+            pp_store_p<kF8>(tP + c * Op::kPCols, pk);
         }
         {
             float a0, a1, b0, b1;
@@ -541,7 +589,8 @@ struct PpSoftmax {
 // to its epilogue stays within the 32 KB the instruction cache serves at full rate, which is
 // what counts when an item has few steps.
 // kVarlen (needs kTmaOut): a packed batch of sequences of different lengths (see FwdParams).
-template <typename T, bool kTmaOut, bool kSingle, bool kVarlen>
+// kF8: q, k, v hold FP8 e4m3 bytes (see PpOperands); T is then the type of the output only.
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8 = false>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -554,7 +603,7 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t smem_base = smem_u32(smem_raw);
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kPpQBufs * kTileBytes;
-    const uint32_t sV = sK + kPpNK * kTileBytes;
+    const uint32_t sV = sK + kPpNK * PpOperands<kF8>::kKvSlotBytes;
     const uint32_t bar0 = smem_u32(&ss.bars[0]);
     volatile uint32_t* abort_flag = &ss.abort_flag;
 
@@ -593,7 +642,7 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t tS = tmem_base + lane_sel + 128 + 128 * w;
         const uint32_t tP = tmem_base + lane_sel + 384 + 64 * w;
         const float scale_log2 = p.scale_log2;
-        PpSoftmax<T, kVarlen> sm;
+        PpSoftmax<T, kVarlen, kF8> sm;
         sm.sV = sV;
         sm.r = r;
         sm.bar0 = bar0;
@@ -706,11 +755,12 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 // O is in registers: the next item's first P V may overwrite it
                 tc_fence_before();
                 mbar_arrive(pp_bar(bar0, ppb::o_free));
-                const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+                // (FP8: O and the row sum carry the same factor on the probabilities; V's own factor goes on O)
+                const float inv_l = (l_run > 0.f) ? (kF8 ? p.out_scale / l_run : 1.f / l_run) : 0.f;
                 const long long obase = kVarlen ? (long long)(it.q_base + row) * p.o_ss + (long long)it.h * p.o_sh
                                                 : (long long)it.b * p.o_sb + (long long)row * p.o_ss + (long long)it.h * p.o_sh;
                 if (row < Sq_i && p.lse != nullptr) {
-                    const float lse = (l_run > 0.f) ? (m_loc * scale_log2 + log2f(l_run)) * 0.6931471805599453f
+                    const float lse = (l_run > 0.f) ? (m_loc * scale_log2 + log2f(l_run) - (kF8 ? kP8ScaleLog2 : 0.f)) * 0.6931471805599453f
                                                     : -INFINITY;
                     if (kVarlen) p.lse[(long long)it.h * p.total_q + it.q_base + row] = lse;
                     else p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = lse;
@@ -781,10 +831,10 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else {
         setmaxnreg_dec<kPipeOtherRegs>();
         if (lane == 0) {
-            if (warp == 8) pp_run_s<T, kTmaOut, kVarlen>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
-            else if (warp == 10) pp_run_pv<T, kVarlen>(bar0, sV, tmem_base, p, total_items, abort_flag);
-            else if (warp == 9) pp_run_load_qk<kVarlen>(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
-            else pp_run_load_v<kVarlen>(bar0, sV, &tm_v, p, total_items, abort_flag);
+            if (warp == 8) pp_run_s<T, kTmaOut, kVarlen, kF8>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
+            else if (warp == 10) pp_run_pv<T, kVarlen, kF8>(bar0, sV, tmem_base, p, total_items, abort_flag);
+            else if (warp == 9) pp_run_load_qk<kVarlen, kF8>(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
+            else pp_run_load_v<kVarlen, kF8>(bar0, sV, &tm_v, p, total_items, abort_flag);
         }
         __syncwarp();
     }
@@ -799,19 +849,22 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 // to: map over the output with boxes of 32 rows x 64 columns; read only when the output has the
 // operands' type (any valid map otherwise).
-template <typename T>
+// kF8: tq, tk, tv are maps over FP8 e4m3 bytes (boxes of 128 rows x 128 bytes) and T is the output type.
+template <typename T, bool kF8 = false>
 int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                     const FwdParams& fp, cudaStream_t st, int* cuda_err) {
-    constexpr int smem = (kPpQBufs + kPpNK + kPpNV) * kTileBytes;
+    constexpr int smem = kPpQBufs * kTileBytes + (kPpNK + kPpNV) * PpOperands<kF8>::kKvSlotBytes;
     // the single-copy step up to 32 kv tiles per item (timed: ahead by 3 % at 2048 keys, level at
     // 4096, behind by 1 % at 8192)
     const bool single = fp.o_fp32 || fp.Skv <= 32 * kTile;
     const bool varlen = fp.cu_q != nullptr;
     if (varlen && fp.o_fp32) return -3;
-    auto kern = varlen ? fa_fwd_pingpong_kernel<T, true, true, true>
-                       : (fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true, false>
-                                    : (single ? fa_fwd_pingpong_kernel<T, true, true, false>
-                                              : fa_fwd_pingpong_kernel<T, true, false, false>));
+    if (kF8 && (varlen || fp.o_fp32)) return -3;
+    auto kern = kF8 ? fa_fwd_pingpong_kernel<T, true, true, false, kF8>
+                    : (varlen ? fa_fwd_pingpong_kernel<T, true, true, kF8 ? false : true>
+                              : (fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true, false>
+                                           : (single ? fa_fwd_pingpong_kernel<T, true, true, false>
+                                                     : fa_fwd_pingpong_kernel<T, true, false, false>)));
     int sm_count = 0;
     cudaError_t e;
     if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }
@@ -833,7 +886,7 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
 #ifdef FA_PP_CLASS_LOG2
         cls_log2 = FA_PP_CLASS_LOG2;
 #else
-        const double head_bytes = 512.0 * fp.Skv / (fp.Hq / fp.Hkv);
+        const double head_bytes = (kF8 ? 256.0 : 512.0) * fp.Skv / (fp.Hq / fp.Hkv);
         const double budget = 32.0 * 1024 * 1024;
         const int half = fp.n_qtiles / 2 < 16 ? fp.n_qtiles / 2 : 16;
         const int cap = (fp.causal && fp.n_qtiles < 16) ? 1 : half;
@@ -844,7 +897,7 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
     // From three rounds per head on (56K keys on 148 SMs) and once a head's K and V are past what
     // L2 keeps, the head-by-head order with whole rounds per head (see PpItems); the empty slots of
     // a head's last round cost little there because its items are the head's shortest.
-    const double kv_bytes_per_head = 2.0 * fp.Skv * 128 * 2;
+    const double kv_bytes_per_head = 2.0 * fp.Skv * 128 * (kF8 ? 1 : 2);
     if (!varlen && fp.n_qtiles >= 3 * grid && kv_bytes_per_head > 24.0 * 1024 * 1024) {
         fpc.rounds_per_head = (fp.n_qtiles + grid - 1) / grid;
         fpc.by_rph.set(fpc.rounds_per_head);

@@ -69,6 +69,7 @@ struct FwdParams {
     const int* seqlens_k;
     int table_stride, page_size;
     int d;  // head dimension: 128, or 64 (its own kernel)
+    float out_scale;  // factor on O (FP8 operands: the factor of V; 1 otherwise)
 };
 
 constexpr int kTile = 128;          // query rows per tile == kv rows per tile == head dim

@@ -209,6 +209,13 @@ def fp8_cache(k, v, seqlens, k_scale: float, v_scale: float, poison: bool = True
     return k8, v8
 
 
+def fp8_operands(q, k, v, q_scale: float, k_scale: float, v_scale: float):
+    """The tensors of ``prefill_inputs`` as FP8 e4m3 bit patterns (uint8) for given factors: each
+    value divided by its tensor's factor and rounded to e4m3 by torch's conversion (an input
+    generator: 8-bit operands are what ``fa_forward_fp8`` is handed)."""
+    return tuple((t.float() / s).to(torch.float8_e4m3fn).view(torch.uint8) for t, s in ((q, q_scale), (k, k_scale), (v, v_scale)))
+
+
 def paged_cache(k, v, seqlens, page_size: int, seed: int, spare_pages: int = 3, poison: bool = True):
     """The caches of ``decode_inputs`` laid out in pages: returns ``(k_pages, v_pages, block_table)``.
 

@@ -275,3 +275,25 @@ def test_selftest_wait_validates_before_any_cuda_call(fa):
     assert fa.lib.fa_selftest_wait(1000, c.data_ptr() + 2, None) == fa.FA_ERR_ALIGN
     assert fa.lib.fa_selftest_wait(0, c.data_ptr(), None) == fa.FA_ERR_UNSUPPORTED
     assert fa.lib.fa_selftest_wait(100001, c.data_ptr(), None) == fa.FA_ERR_UNSUPPORTED
+
+
+def test_forward_fp8_validation(fa):
+    q = torch.zeros(1, 4, 4, 128, dtype=torch.uint8)
+    o = torch.zeros(1, 4, 4, 128, dtype=torch.float16)
+    P = lambda t: t.data_ptr()
+    L = fa.lib.fa_forward_fp8
+    ok = dict(B=1, Hq=4, Hkv=2, Sq=4, Skv=4, d=128, causal=1, scale=0.1, qs=0.5, ks=0.5, vs=0.5, od=fa.FA_DTYPE_FP16)
+    def call(qp=P(q), kp=P(q), vp=P(q), op=P(o), **kw):
+        a = dict(ok); a.update(kw)
+        return L(qp, kp, vp, op, None, a["B"], a["Hq"], a["Hkv"], a["Sq"], a["Skv"], a["d"], a["causal"], a["scale"],
+                 a["qs"], a["ks"], a["vs"], a["od"], None)
+    assert call(B=0) == fa.FA_OK and call(Sq=0) == fa.FA_OK
+    assert call(Hq=3) == fa.FA_ERR_SHAPE and call(B=-1) == fa.FA_ERR_SHAPE
+    assert call(d=64) == fa.FA_ERR_UNSUPPORTED and call(od=fa.FA_DTYPE_FP32) == fa.FA_ERR_UNSUPPORTED
+    assert call(Sq=5) == fa.FA_ERR_UNSUPPORTED                       # causal with more queries than keys
+    for bad in (0.0, -1.0, float("inf"), float("nan")):
+        assert call(qs=bad) == fa.FA_ERR_UNSUPPORTED and call(ks=bad) == fa.FA_ERR_UNSUPPORTED
+        assert call(vs=bad) == fa.FA_ERR_UNSUPPORTED
+    assert call(scale=-0.1) == fa.FA_ERR_UNSUPPORTED
+    assert call(qp=None) == fa.FA_ERR_NULL and call(op=None) == fa.FA_ERR_NULL and call(kp=None) == fa.FA_ERR_NULL
+    assert call(qp=P(q) + 4) == fa.FA_ERR_ALIGN and call(op=P(o) + 2) == fa.FA_ERR_ALIGN

@@ -378,6 +378,41 @@ def test_e4m3_values_and_fp8_decode():
     assert torch.allclose(O3, O, rtol=1e-12, atol=1e-14) and torch.allclose(L3, LSE, rtol=1e-12, atol=1e-14)
 
 
+def test_fp8_attention_is_attention_on_the_widened_operands():
+    # 8-bit operands: the definition on Q = q_scale * value(bits) etc.  Pins: torch's own widening and
+    # softmax.matmul in float64 (library routines the oracle does not use); the factors of q and k
+    # are interchangeable with the softmax scale; v's factor scales O and leaves LSE; a value
+    # tensor whose bit patterns all read 1.0 (0x38) gives O = v_scale exactly; rows mode = full mode
+    B, Sq, Skv, Hq, Hkv, d = 2, 5, 7, 4, 2, 8
+    gen = torch.Generator().manual_seed(91)
+    def bits(shape):
+        return torch.randint(0, 0x78, shape, generator=gen, dtype=torch.uint8) | (torch.randint(0, 2, shape, generator=gen, dtype=torch.uint8) << 7)
+    q8, k8, v8 = bits((B, Sq, Hq, d)), bits((B, Skv, Hkv, d)), bits((B, Skv, Hkv, d))
+    for causal in (False, True):
+        O, LSE = oracle.attention_fp8(q8, k8, v8, causal, 0.02, 0.5, 0.25, 0.125)
+        qf = q8.view(torch.float8_e4m3fn).to(torch.float64) * 0.5
+        kf = (k8.view(torch.float8_e4m3fn).to(torch.float64) * 0.25).repeat_interleave(Hq // Hkv, dim=2)
+        vf = (v8.view(torch.float8_e4m3fn).to(torch.float64) * 0.125).repeat_interleave(Hq // Hkv, dim=2)
+        s = torch.einsum("bihd,bjhd->bhij", qf, kf) * 0.02
+        if causal:
+            vis = torch.ones(Sq, Skv, dtype=torch.bool).tril(Skv - Sq)
+            s = s.masked_fill(~vis, float("-inf"))
+        want = torch.einsum("bhij,bjhd->bihd", torch.softmax(s, -1), vf)
+        assert torch.allclose(O, want, rtol=1e-12, atol=1e-13)
+        assert torch.allclose(LSE, torch.logsumexp(s, -1), rtol=1e-12, atol=1e-13)
+        O2, L2 = oracle.attention_fp8(q8, k8, v8, causal, 0.02 * 0.5 * 0.25, 1.0, 1.0, 0.25)
+        assert torch.allclose(O2, 2 * O, rtol=1e-12, atol=1e-13) and torch.allclose(L2, LSE, rtol=1e-12, atol=1e-13)
+        ones = torch.full_like(v8, 0x38)
+        O3, _ = oracle.attention_fp8(q8, k8, ones, causal, 0.02, 0.5, 0.25, 0.125)
+        assert torch.allclose(O3, torch.full_like(O3, 0.125), rtol=1e-14, atol=0)
+        rows = [(0, 0, 0), (1, 3, 4), (0, 2, 2)]
+        Or, Lr = oracle.attention_fp8(q8, k8, v8, causal, 0.02, 0.5, 0.25, 0.125, rows=rows)
+        for n, (b, h, i) in enumerate(rows):
+            assert torch.equal(Or[n], O[b, i, h]) and Lr[n] == LSE[b, h, i]
+        Oa, _ = oracle.attention_fp8(q8, k8, v8, causal, 0.02, 0.5, 0.25, 0.125, abs_v=True)
+        assert torch.allclose(Oa, torch.einsum("bhij,bjhd->bihd", torch.softmax(s, -1), vf.abs()), rtol=1e-12, atol=1e-13)
+
+
 def test_paged_packed_batch_equals_the_packed_batch_on_the_same_keys():
     # pools filled by hand, page by page in a scrambled order; NaN wherever no key lives
     Hq, Hkv, d, ps = 4, 2, 4, 4

@@ -470,6 +470,87 @@ def test_d256_is_refused_where_it_is_not_built(fa):
     assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=1, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
 
 
+# ------------------------------------------------------------------ 8-bit operands in prefill
+FP8_SCALES = (0.125, 0.25, 0.0625)      # factors of q, k, v
+
+
+def fp8_allowance(q8, k8, v8, rows, causal, scale, stored_bf16):
+    """What rounding the probabilities to FP8 e4m3 may cost, per output element of the given rows
+    (b, h, i), from oracle-side quantities only.  The kernel rounds F * 2^(x_ij - m_ref), with F = 2^4
+    and the reference m_ref at most 2^4 behind the running row max, to e4m3: a relative rounding of
+    at most 2^-4 for values in the normal range and an absolute one of at most 2^-10 below it.
+    Carried through O_i = sum_j P_ij V_j / l_i that is at most
+        2^-4 * sum_j P_ij |V_j|  +  2^-14 * sum_j |V_j| / L_i ,   L_i = sum_j exp(s_ij - max_j s_ij)
+    (visible j only).  The first term comes from the oracle run on |V|; the row max for the second
+    is taken from the scores of the row, computed here in float64."""
+    qs, ks, vs = FP8_SCALES
+    o_abs, _ = oracle.attention_fp8(q8, k8, v8, causal, scale, qs, ks, vs, rows=rows, abs_v=True)
+    g = q8.shape[2] // k8.shape[2]
+    Sq, Skv = q8.shape[1], k8.shape[1]
+    out = torch.zeros_like(o_abs)
+    for n, (b, h, i) in enumerate(rows):
+        qf = oracle.e4m3_to_float64(q8[b, i, h]) * qs
+        kf = oracle.e4m3_to_float64(k8[b, :, h // g]) * ks
+        vf = (oracle.e4m3_to_float64(v8[b, :, h // g]) * vs).abs()
+        nvis = min(Skv, i + (Skv - Sq) + 1) if causal else Skv
+        sc = (kf[:nvis] @ qf) * scale
+        L = torch.exp(sc - sc.max()).sum()
+        out[n] = 2.0 ** -4 * o_abs[n] + 2.0 ** -14 * vf[:nvis].sum(0) / L
+    return out
+
+
+def fp8_case(fa, B, Hq, Hkv, Sq, Skv, causal, o_dtype, seed, rows=None):
+    cfg = synth.PrefillConfig("fp8", B, Hq, Hkv, Sq, Skv, dtype="fp16", causal=causal, seed=seed)
+    dev = DEV if rows is not None else "cpu"
+    q, k, v = synth.prefill_inputs(cfg, dev)
+    qs, ks, vs = FP8_SCALES
+    q8, k8, v8 = synth.fp8_operands(q, k, v, qs, ks, vs)
+    qd, kd, vd = q8.to(DEV), k8.to(DEV), v8.to(DEV)
+    o, chk_o = guard_alloc((B, Sq, Hq, 128), o_dtype, DEV)
+    lse, chk_l = guard_alloc((B, Hq, Sq), torch.float32, DEV)
+    fa.fa_forward_fp8(qd, kd, vd, o, lse, causal, cfg.scale, qs, ks, vs)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l()
+    assert not torch.isnan(o).any() and not torch.isnan(lse).any()
+    q8c, k8c, v8c = q8.cpu(), k8.cpu(), v8.cpu()
+    if rows is None:
+        rows = [(b, h, i) for b in range(B) for h in range(Hq) for i in range(Sq)]
+    o_ref, l_ref = oracle.attention_fp8(q8c, k8c, v8c, causal, cfg.scale, qs, ks, vs, rows=rows)
+    allow = fp8_allowance(q8c, k8c, v8c, rows, causal, cfg.scale, o_dtype == torch.bfloat16)
+    idx = torch.tensor(rows, device=DEV)
+    o_s = o[idx[:, 0], idx[:, 2], idx[:, 1]].double().cpu()
+    l_s = lse[idx[:, 0], idx[:, 1], idx[:, 2]].double().cpu()
+    if o_dtype == torch.bfloat16:
+        allow = allow + 2.0 ** -8 * o_ref.abs()
+    diff = (o_s - o_ref).abs()
+    what = f"fp8 B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} causal{int(causal)} {o_dtype}"
+    assert float((diff - allow).max()) <= TOL_O, f"{what}: max(|dO| - allowance) = {float((diff - allow).max()):.3e}"
+    assert float((l_s - l_ref).abs().max()) <= TOL_LSE, f"{what}: max|dLSE| = {float((l_s - l_ref).abs().max()):.3e}"
+    return float(diff.max()), float(allow.max())
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("sq,skv", [(1, 1), (127, 127), (128, 128), (129, 129), (300, 300), (1, 129), (17, 1000), (100, 257),
+                                    (257, 1000), (130, 2200)])
+def test_fp8_prefill_shape_grid(fa, sq, skv, causal):
+    fp8_case(fa, 2, 2, 1, sq, skv, causal, torch.float16, seed=sq * 1000 + skv + 21)
+
+
+def test_fp8_prefill_gqa_many_items_and_bf16_output(fa):
+    fp8_case(fa, 2, 8, 2, 333, 333, True, torch.bfloat16, seed=95)
+    fp8_case(fa, 3, 64, 64, 300, 300, True, torch.float16, seed=96)        # several items per CTA
+    fp8_case(fa, 1, 4, 4, 700, 1300, False, torch.bfloat16, seed=97)
+
+
+def test_fp8_prefill_bench_sizes_sampled(fa):
+    # C2's shape and the 8K long-context shape with 8-bit operands, sampled rows against the oracle
+    for cfg in (synth.C2, synth.C3[8192]):
+        rows = synth.sample_rows(cfg, 30, seed=cfg.seed + 7)
+        worst, allow = fp8_case(fa, cfg.B, cfg.Hq, cfg.Hkv, cfg.Sq, cfg.Skv, True, torch.float16, seed=cfg.seed + 50, rows=rows)
+        print(f"fp8 {cfg.name}: max|dO| {worst:.2e} (largest allowance {allow:.2e})")
+
+
 # ------------------------------------------------------------------ packed variable-length batches
 def varlen_case(fa, cfg, what):
     q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
