@@ -125,6 +125,34 @@ int fa_forward_fp8(const void* q, const void* k, const void* v, void* o, float* 
                    float k_scale, float v_scale, int o_dtype, void* stream);
 
 /*
+ * Attention followed by the output projection (Section 4.2 fuses the attention kernel with the
+ * Linear that follows it; Appendix C writes the projection as the decoder layer's last step of
+ * attention).  On one GPU there is no collective behind the Linear, so this is that fused kernel
+ * without its AllReduce:
+ *     O   = fa_forward(q, k, v)                       [B, Sq, Hq, d], also returned
+ *     out = O viewed as [B, Sq, Hq * d]  times  w_o   [B, Sq, d_model]
+ * with w_o [Hq * d, d_model] row-major (d_model contiguous), all in the 16-bit type `dtype`, fp32
+ * accumulation in both products, O rounded to 16 bits between them.
+ *   fused != 0: ONE launch.  The attention phase is the ping-pong kernel of fa_forward; a CTA that
+ *   has finished its attention items goes on to 128 x 256 blocks of the projection, each as soon as
+ *   the attention output of every head for its 128 query rows has reached global memory (a counter
+ *   per row block in `workspace`, which the call zeroes; the wait on it is bounded like every
+ *   other).  The launch is cooperative: it fails with FA_ERR_CUDA rather than start if the GPU
+ *   cannot hold the whole grid at once.
+ *   fused == 0: the same two kernels as two launches on `stream` (no workspace needed).
+ *   d must be 128, d_model a multiple of 256; out 32-byte aligned; workspace of at least
+ *   fa_forward_proj_workspace_bytes(B, Sq) bytes, 4-byte aligned.  lse may be NULL.
+ * Errors: as fa_forward; FA_ERR_UNSUPPORTED also for other d_model, FA_ERR_WORKSPACE for a missing
+ * or short workspace with fused != 0.
+ */
+int fa_forward_proj(const void* q, const void* k, const void* v, const void* w_o, void* o, float* lse,
+                    void* out, int B, int Hq, int Hkv, int Sq, int Skv, int d, int d_model, int causal,
+                    float scale, int dtype, int fused, void* workspace, size_t workspace_bytes,
+                    void* stream);
+
+size_t fa_forward_proj_workspace_bytes(int B, int Sq);
+
+/*
  * Forward over a packed batch of sequences of different lengths (the batched serving runs of the
  * evaluation section process requests of unequal length together): the same computation as
  * fa_forward, sequence by sequence.  Sequence b owns rows [cu_seqlens_q[b], cu_seqlens_q[b+1])

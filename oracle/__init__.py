@@ -255,6 +255,23 @@ def e4m3_to_float64(bits):
     return torch.where(nan, torch.full_like(val, float("nan")), val)
 
 
+def attention_proj(q, k, v, w_o, causal: bool, scale: float, nthreads: int = 0):
+    """Attention followed by the output projection (Section 4.2's fused attention + Linear on one
+    device; Appendix C's last step of the attention block): ``O = attention_full(q, k, v)``, then
+    ``out[b, i, :] = O16[b, i, :, :].reshape(Hq * d) @ w_o`` in float64, where ``O16`` is O rounded
+    to the operands' 16-bit type -- the operator returns O in that type and the projection reads
+    what it returns.  ``w_o``: ``[Hq*d, d_model]``.  Returns ``(O, LSE, out)`` float64, O unrounded."""
+    O, LSE = attention_full(q, k, v, causal, scale, nthreads)
+    q = torch.as_tensor(q)
+    w = torch.as_tensor(w_o).to(torch.float64)
+    B, Sq, Hq, d = O.shape
+    if w.shape[0] != Hq * d:
+        raise ValueError("w_o must have Hq * d rows")
+    O16 = O.to(q.dtype).to(torch.float64) if q.dtype in (torch.float16, torch.bfloat16) else O
+    out = torch.matmul(O16.reshape(B, Sq, Hq * d), w)
+    return O, LSE, out
+
+
 def attention_fp8(q_bits, k_bits, v_bits, causal: bool, scale: float, q_scale: float, k_scale: float,
                   v_scale: float, rows=None, abs_v: bool = False, nthreads: int = 0):
     """Standard attention on FP8 e4m3 operands (Appendix D.2 runs the operator on 8-bit

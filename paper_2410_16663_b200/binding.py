@@ -43,6 +43,10 @@ lib.fa_forward_ex.restype = _i
 lib.fa_forward_ex.argtypes = [ctypes.POINTER(fa_params), _p]
 lib.fa_forward_fp8.restype = _i
 lib.fa_forward_fp8.argtypes = [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _f, _f, _f, _i, _p]
+lib.fa_forward_proj.restype = _i
+lib.fa_forward_proj.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _i, _p, _sz, _p]
+lib.fa_forward_proj_workspace_bytes.restype = _sz
+lib.fa_forward_proj_workspace_bytes.argtypes = [_i, _i]
 lib.fa_decode.restype = _i
 lib.fa_decode.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _p, _sz, _p]
 lib.fa_decode_workspace_bytes.restype = _sz
@@ -88,7 +92,7 @@ lib.fa_last_cuda_error.restype = _i
 
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
-EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_forward_fp8", "fa_decode", "fa_decode_workspace_bytes",
+EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_forward_fp8", "fa_forward_proj", "fa_forward_proj_workspace_bytes", "fa_decode", "fa_decode_workspace_bytes",
            "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_selftest_wait", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
@@ -165,7 +169,25 @@ def fa_forward_fp8(q, k, v, o, lse, causal: bool, scale: float, q_scale: float, 
     dt = FA_DTYPE_BF16 if o.dtype == torch.bfloat16 else FA_DTYPE_FP16
     rc = lib.fa_forward_fp8(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Hq, Hkv, Sq, Skv, d, int(bool(causal)),
                             float(scale), float(q_scale), float(k_scale), float(v_scale), dt, _stream())
-    return _check(rc, "fa_forward_fp8", raise_on_error)
+    return _check(rc, "fa_forward_fp8", "fa_forward_proj", "fa_forward_proj_workspace_bytes", raise_on_error)
+
+
+def fa_forward_proj_workspace_bytes(B: int, Sq: int) -> int:
+    return int(lib.fa_forward_proj_workspace_bytes(B, Sq))
+
+
+def fa_forward_proj(q, k, v, w_o, o, lse, out, causal: bool, scale: float, fused: bool, workspace=None,
+                    raise_on_error: bool = True) -> int:
+    """``fa_forward_proj``: attention, then ``out = O.view(B, Sq, Hq*d) @ w_o`` with w_o [Hq*d, d_model];
+    one launch (``fused``, needs a workspace of ``fa_forward_proj_workspace_bytes`` bytes) or two."""
+    B, Sq, Hq, d = q.shape
+    _, Skv, Hkv, _ = k.shape
+    dt = FA_DTYPE_BF16 if q.dtype == torch.bfloat16 else FA_DTYPE_FP16
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_forward_proj(_ptr(q), _ptr(k), _ptr(v), _ptr(w_o), _ptr(o), _ptr(lse), _ptr(out), B, Hq, Hkv, Sq, Skv, d,
+                             w_o.shape[1], int(bool(causal)), float(scale), dt, int(bool(fused)), _ptr(workspace), wbytes,
+                             _stream())
+    return _check(rc, "fa_forward_proj", raise_on_error)
 
 
 def fa_forward_varlen(q, k, v, o, lse, cu_seqlens_q, cu_seqlens_k, max_seqlen_q: int, max_seqlen_k: int,

@@ -13,6 +13,7 @@
 
 #include "decode.cuh"
 #include "prefill_pingpong.cuh"
+#include "proj_gemm.cuh"
 #include "prefill_d64.cuh"
 #include "prefill_d256.cuh"
 #include "decode_fp8.cuh"
@@ -91,6 +92,26 @@ int encode_map_u8(CUtensorMap* tm, const void* base, int B, int S, int H, int bo
     return FA_OK;
 }
 
+// Tensor map over a row-major [rows, cols] 16-bit matrix: a box is 64 rows x 64 columns, 128-byte
+// swizzled (the projection weight, an N-major MMA operand).  Encoded with four dimensions so that
+// the kernels' one load wrapper serves it; the outer two have extent 1.
+int encode_map_matrix(CUtensorMap* tm, const void* base, int rows, int cols, bool bf16) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return FA_ERR_DEVICE;
+    cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)rows, 1, 1};
+    cuuint64_t strides[3] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * rows, (cuuint64_t)cols * 2 * rows};
+    cuuint32_t box[4] = {64, 64, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
+                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        t_last_cuda_error = static_cast<int>(r);
+        return FA_ERR_CUDA;
+    }
+    return FA_OK;
+}
+
 // a page holds a multiple of the 128-key tile, or 16, 32 or 64 keys (several pages per tile)
 bool page_size_ok(int ps) { return ps > 0 && (ps % fa::kDecTile == 0 || ps == 16 || ps == 32 || ps == 64); }
 
@@ -149,34 +170,9 @@ int launch_simple(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMa
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
-int forward_impl(const fa_params& in, cudaStream_t st) {
-    fa_params p = in;
-    // ---- validation (no CUDA call before it passes)
-    if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
-    if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
-    if (p.d != 128 && p.d != 64 && p.d != 256) return FA_ERR_UNSUPPORTED;
-    if (p.d != 128 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // d = 64 and d = 256 have kernels of their own
-    if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
-    if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
-    if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
-    if (p.causal && p.Sq > p.Skv) return FA_ERR_UNSUPPORTED;
-    if (p.Hq > 65535 || p.B > 65535) return FA_ERR_UNSUPPORTED;
-    if (p.B == 0 || p.Sq == 0) return FA_OK;
-    if (!p.q || !p.o) return FA_ERR_NULL;
-    if (p.Skv > 0 && (!p.k || !p.v)) return FA_ERR_NULL;
-    default_strides(p.q_stride, p.Sq, p.Hq, p.d);
-    default_strides(p.k_stride, p.Skv, p.Hkv, p.d);
-    default_strides(p.v_stride, p.Skv, p.Hkv, p.d);
-    default_strides(p.o_stride, p.Sq, p.Hq, p.d);
-    if (!strides_ok(p.q_stride, p.B, p.Sq, p.Hq, p.d) || !strides_ok(p.k_stride, p.B, p.Skv, p.Hkv, p.d) ||
-        !strides_ok(p.v_stride, p.B, p.Skv, p.Hkv, p.d) || !strides_ok(p.o_stride, p.B, p.Sq, p.Hq, p.d))
-        return FA_ERR_SHAPE;
-    if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.o)) return FA_ERR_ALIGN;
-    if (p.lse && (reinterpret_cast<uintptr_t>(p.lse) & 3u)) return FA_ERR_ALIGN;
-
-    int rc = check_device();
-    if (rc) return rc;
-
+// Kernel parameters of a dense (not packed, not paged) forward from validated arguments whose
+// strides have been filled in.
+fa::FwdParams dense_fwd_params(const fa_params& p) {
     fa::FwdParams fp;
     fp.o = p.o;
     fp.lse = p.lse;
@@ -209,6 +205,38 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     fp.d = p.d;
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
+    return fp;
+}
+
+int forward_impl(const fa_params& in, cudaStream_t st) {
+    fa_params p = in;
+    // ---- validation (no CUDA call before it passes)
+    if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
+    if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
+    if (p.d != 128 && p.d != 64 && p.d != 256) return FA_ERR_UNSUPPORTED;
+    if (p.d != 128 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // d = 64 and d = 256 have kernels of their own
+    if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
+    if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
+    if (p.causal && p.Sq > p.Skv) return FA_ERR_UNSUPPORTED;
+    if (p.Hq > 65535 || p.B > 65535) return FA_ERR_UNSUPPORTED;
+    if (p.B == 0 || p.Sq == 0) return FA_OK;
+    if (!p.q || !p.o) return FA_ERR_NULL;
+    if (p.Skv > 0 && (!p.k || !p.v)) return FA_ERR_NULL;
+    default_strides(p.q_stride, p.Sq, p.Hq, p.d);
+    default_strides(p.k_stride, p.Skv, p.Hkv, p.d);
+    default_strides(p.v_stride, p.Skv, p.Hkv, p.d);
+    default_strides(p.o_stride, p.Sq, p.Hq, p.d);
+    if (!strides_ok(p.q_stride, p.B, p.Sq, p.Hq, p.d) || !strides_ok(p.k_stride, p.B, p.Skv, p.Hkv, p.d) ||
+        !strides_ok(p.v_stride, p.B, p.Skv, p.Hkv, p.d) || !strides_ok(p.o_stride, p.B, p.Sq, p.Hq, p.d))
+        return FA_ERR_SHAPE;
+    if (!aligned16(p.q) || !aligned16(p.k) || !aligned16(p.v) || !aligned16(p.o)) return FA_ERR_ALIGN;
+    if (p.lse && (reinterpret_cast<uintptr_t>(p.lse) & 3u)) return FA_ERR_ALIGN;
+
+    int rc = check_device();
+    if (rc) return rc;
+
+    fa::FwdParams fp = dense_fwd_params(p);
     const bool bf16 = p.dtype == FA_DTYPE_BF16;
 
     if (p.Skv == 0) {
@@ -440,6 +468,88 @@ int fa_forward_fp8(const void* q, const void* k, const void* v, void* o, float* 
     if (rc) return rc;
     return bf16 ? fa::launch_pingpong<__nv_bfloat16, true>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
                 : fa::launch_pingpong<__half, true>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
+}
+
+size_t fa_forward_proj_workspace_bytes(int B, int Sq) {
+    if (B <= 0 || Sq <= 0) return 0;
+    return (size_t)B * ((Sq + fa::kTile - 1) / fa::kTile) * sizeof(unsigned int);
+}
+
+int fa_forward_proj(const void* q, const void* k, const void* v, const void* w_o, void* o, float* lse, void* out,
+                    int B, int Hq, int Hkv, int Sq, int Skv, int d, int d_model, int causal, float scale, int dtype,
+                    int fused, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Sq < 0 || Skv < 0 || d <= 0 || d_model <= 0) return FA_ERR_SHAPE;
+    if (Hq % Hkv) return FA_ERR_SHAPE;
+    if (d != 128 || d_model % 256) return FA_ERR_UNSUPPORTED;
+    if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
+    if (causal && Sq > Skv) return FA_ERR_UNSUPPORTED;
+    if (Hq > 16383 || B > 65535) return FA_ERR_UNSUPPORTED;
+    if ((long long)B * ((Sq + fa::kTile - 1) / fa::kTile) * (d_model / 256) > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
+    if (B == 0 || Sq == 0) return FA_OK;
+    if (!q || !o || !out || !w_o) return FA_ERR_NULL;
+    if (Skv > 0 && (!k || !v)) return FA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(w_o)) return FA_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(out) & 31u) return FA_ERR_ALIGN;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return FA_ERR_ALIGN;
+    if (fused) {
+        if (reinterpret_cast<uintptr_t>(workspace) & 3u) return FA_ERR_ALIGN;
+        if (!workspace || workspace_bytes < fa_forward_proj_workspace_bytes(B, Sq)) return FA_ERR_WORKSPACE;
+    }
+    int rc = check_device();
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool bf16 = dtype == FA_DTYPE_BF16;
+    cudaError_t e;
+
+    fa_params ap;
+    memset(&ap, 0, sizeof ap);
+    ap.q = q; ap.k = k; ap.v = v; ap.o = o; ap.lse = lse;
+    ap.B = B; ap.Hq = Hq; ap.Hkv = Hkv; ap.Sq = Sq; ap.Skv = Skv; ap.d = d;
+    ap.causal = causal; ap.scale = scale; ap.dtype = dtype; ap.o_dtype = dtype;
+    ap.variant = 3;   // the ping-pong kernel in both forms, so that they compute the same O
+    default_strides(ap.q_stride, Sq, Hq);
+    default_strides(ap.k_stride, Skv, Hkv);
+    default_strides(ap.v_stride, Skv, Hkv);
+    default_strides(ap.o_stride, Sq, Hq);
+
+    fa::ProjParams pp;
+    pp.out = out;
+    pp.B = B; pp.Sq = Sq; pp.Hq = Hq; pp.N = d_model;
+    pp.n_qtiles = (Sq + fa::kTile - 1) / fa::kTile;
+    pp.n_cblocks = d_model / 256;
+    pp.done = nullptr;
+    pp.done_target = 4u * (unsigned int)Hq;
+
+    CUtensorMap tq, tk, tv, to, ta, tw;
+    // O as the projection's K-major operand: the attention output read back in 128 x 64 boxes
+    rc = encode_map(&ta, o, B, Sq, Hq, (int64_t)Sq * Hq * 128, (int64_t)Hq * 128, 128, 128, bf16);
+    if (rc) return rc;
+    rc = encode_map_matrix(&tw, w_o, Hq * 128, d_model, bf16);
+    if (rc) return rc;
+
+    if (!fused || Skv == 0) {
+        // two launches: the attention kernel (or, without keys, the fill that writes O = 0), then the projection
+        rc = forward_impl(ap, st);
+        if (rc) return rc;
+        rc = bf16 ? fa::launch_proj<__nv_bfloat16>(ta, tw, ta, ta, ta, tw, dense_fwd_params(ap), pp, 0, st, &t_last_cuda_error)
+                  : fa::launch_proj<__half>(ta, tw, ta, ta, ta, tw, dense_fwd_params(ap), pp, 0, st, &t_last_cuda_error);
+        return rc;
+    }
+    e = cudaMemsetAsync(workspace, 0, fa_forward_proj_workspace_bytes(B, Sq), st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    pp.done = static_cast<unsigned int*>(workspace);
+    rc = encode_map(&tq, q, B, Sq, Hq, ap.q_stride[0], ap.q_stride[1], ap.q_stride[2], 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tk, k, B, Skv, Hkv, ap.k_stride[0], ap.k_stride[1], ap.k_stride[2], 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&tv, v, B, Skv, Hkv, ap.v_stride[0], ap.v_stride[1], ap.v_stride[2], 128, bf16);
+    if (rc) return rc;
+    rc = encode_map(&to, o, B, Sq, Hq, ap.o_stride[0], ap.o_stride[1], ap.o_stride[2], 32, bf16);
+    if (rc) return rc;
+    const fa::FwdParams fp = dense_fwd_params(ap);
+    return bf16 ? fa::launch_proj<__nv_bfloat16>(tq, tk, tv, to, ta, tw, fp, pp, 1, st, &t_last_cuda_error)
+                : fa::launch_proj<__half>(tq, tk, tv, to, ta, tw, fp, pp, 1, st, &t_last_cuda_error);
 }
 
 int fa_forward_ex(const fa_params* p, void* stream) {

@@ -249,6 +249,16 @@ __device__ __forceinline__ void pp_store_p<true>(uint32_t taddr, const uint32_t 
 
 __device__ __forceinline__ uint32_t pp_bar(uint32_t bar0, int i) { return bar0 + 8 * i; }
 
+// Counter in global memory that one SM raises after its writes and another reads before its loads.
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(unsigned int* p, unsigned int v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 // Ring cursor: slot and phase parity of the g-th entry of a ring of N slots.
 template <int N>
 struct PpRing {
@@ -590,17 +600,16 @@ struct PpSoftmax {
 // what counts when an item has few steps.
 // kVarlen (needs kTmaOut): a packed batch of sequences of different lengths (see FwdParams).
 // kF8: q, k, v hold FP8 e4m3 bytes (see PpOperands); T is then the type of the output only.
-template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8 = false>
-__global__ void __launch_bounds__(kPipeThreads, 1)
-fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
-                       const FwdParams p, const int total_items) {
-    // Shared memory is used to the last byte: 3 KiB of static state (sized so that the dynamic
-    // part that follows it starts on a 1024-byte boundary, which the 128-byte swizzle needs)
-    // plus seven 32 KiB tiles.  The alignment is checked rather than assumed.
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(1024) PpStatic ss;
-    const uint32_t smem_base = smem_u32(smem_raw);
+// kProj (needs kTmaOut): a projection phase follows in the same launch (proj_gemm.cuh): a warp
+// that has stored its rows of an item's output waits until the stores have reached global memory
+// and counts them in done[batch * n_qtiles + query tile]; four warps and Hq heads make a row
+// block of O complete.
+// The whole kernel but for the release of tensor memory; returns false if nothing was set up.
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8, bool kProj>
+__device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                             const CUtensorMap& tm_o, const FwdParams& p, const int total_items,
+                                             PpStatic& ss, const uint32_t smem_base, unsigned int* done) {
+    static_assert(!kProj || (kTmaOut && !kVarlen), "the projection phase reads a contiguous 16-bit O");
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kPpQBufs * kTileBytes;
     const uint32_t sV = sK + kPpNK * PpOperands<kF8>::kKvSlotBytes;
@@ -612,7 +621,7 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int lane = tid & 31;
     if (smem_base & 1023u) {  // uniform for the CTA: nothing has been set up yet
         if (tid == 0) record_timeout(900);
-        return;
+        return false;
     }
     if (tid == 0) {
         for (int i = 0; i < ppb::count; ++i) {
@@ -665,10 +674,16 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         // this warp's next step: early enough for the load of the item after the next, and off
         // the path from one item's last step to the next item's first.
         int q_back = -1;
+        int done_slot = 0;     // kProj: the row block the pending stores belong to
         auto hand_back_q = [&]() {
             if (kTmaOut && q_back >= 0) {
                 if (lane == 0) {
-                    tma_store_wait_read();
+                    if (kProj) {
+                        tma_store_wait_all();          // written, not only read out of shared memory
+                        red_release_gpu_add(done + done_slot, 1u);
+                    } else {
+                        tma_store_wait_read();
+                    }
                     mbar_arrive(pp_bar(bar0, ppb::q_empty + q_back));
                 }
                 q_back = -1;
@@ -791,6 +806,7 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         tma_store_commit();
                     }
                     q_back = ord & 1;  // handed back to the loader after this warp's next step
+                    if (kProj) done_slot = it.b * p.n_qtiles + it.q0 / kTile;
                     __syncwarp();
                     if (kVarlen && !box && row < Sq_i) {
                         // the ragged end of a sequence: each thread writes its own row
@@ -827,7 +843,8 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (n >= 2) ++items2;
         }
         // the stores read shared memory, which has to outlive them
-        if (kTmaOut && lane == 0) tma_store_wait_all();
+        if (kProj) hand_back_q();
+        else if (kTmaOut && lane == 0) tma_store_wait_all();
     } else {
         setmaxnreg_dec<kPipeOtherRegs>();
         if (lane == 0) {
@@ -838,17 +855,71 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
         __syncwarp();
     }
+    return true;
+}
 
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8 = false>
+__global__ void __launch_bounds__(kPipeThreads, 1)
+fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                       const FwdParams p, const int total_items) {
+    // Shared memory is used to the last byte: 3 KiB of static state (sized so that the dynamic
+    // part that follows it starts on a 1024-byte boundary, which the 128-byte swizzle needs)
+    // plus seven 32 KiB tiles.  The alignment is checked rather than assumed.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    __shared__ __align__(1024) PpStatic ss;
+    if (!pp_attention<T, kTmaOut, kSingle, kVarlen, kF8, false>(tm_q, tm_k, tm_v, tm_o, p, total_items, ss,
+                                                                smem_u32(smem_raw), nullptr))
+        return;
     tc_fence_before();
     __syncthreads();
-    if (warp == 8) {
+    if ((threadIdx.x >> 5) == 8) {
         __syncwarp();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc(ss.tmem_holder, 512);
     }
 }
 
 // to: map over the output with boxes of 32 rows x 64 columns; read only when the output has the
 // operands' type (any valid map otherwise).
+// The item order of a launch on `grid` CTAs (see pp_class_order and PpItems): returns the
+// parameters with the order's fields filled in.  bytes_per_key: K plus V bytes of one key and head.
+inline FwdParams pp_plan_items(const FwdParams& fp, int grid, double bytes_per_key) {
+    const bool varlen = fp.cu_q != nullptr;
+    // Class size of the item order: large enough that the K and V of the kv heads one round of
+    // CTAs works on (about grid / (C * group) of them, Skv * 512 bytes each) fit in a fraction of
+    // L2, but at most half of a head's tiles and 16 (a class that is the whole head makes all
+    // its tiles read the same K/V lines at the same moment, which measured slower).  Under the
+    // causal mask the items of a class differ in length, which costs balance when a head has few
+    // tiles: heads with fewer than 16 keep the plain longest-first order.  When one head alone
+    // fills every CTA, a single class: the plain head-by-head order.
+    FwdParams fpc = fp;
+    int cls_log2 = 0;
+    if (fp.n_qtiles >= grid) {
+        while ((1 << cls_log2) < fp.n_qtiles) ++cls_log2;
+    } else {
+        const double head_bytes = bytes_per_key * fp.Skv / (fp.Hq / fp.Hkv);
+        const double budget = 32.0 * 1024 * 1024;
+        const int half = fp.n_qtiles / 2 < 16 ? fp.n_qtiles / 2 : 16;
+        const int cap = (fp.causal && fp.n_qtiles < 16) ? 1 : half;
+        while ((grid >> cls_log2) * head_bytes > budget && (2 << cls_log2) <= cap) ++cls_log2;
+        while (cls_log2 > 0 && (1 << cls_log2) > fp.n_qtiles) --cls_log2;
+    }
+    // From three rounds per head on (56K keys on 148 SMs) and once a head's K and V are past what
+    // L2 keeps, the head-by-head order with whole rounds per head (see PpItems); the empty slots of
+    // a head's last round cost little there because its items are the head's shortest.
+    const double kv_bytes_per_head = bytes_per_key * fp.Skv;
+    if (!varlen && fp.n_qtiles >= 3 * grid && kv_bytes_per_head > 24.0 * 1024 * 1024) {
+        fpc.rounds_per_head = (fp.n_qtiles + grid - 1) / grid;
+        fpc.by_rph.set(fpc.rounds_per_head);
+    }
+    fpc.cls_log2 = cls_log2;
+    const long long class_items = ((long long)fp.B * fp.Hq) << cls_log2;  // > total only for a single class
+    fpc.by_class.set(class_items > 0x7fffffffll ? 0x7fffffff : (int)class_items);
+    const int last = fp.n_qtiles & ((1 << cls_log2) - 1);
+    fpc.by_lastcls.set(last ? last : 1);
+    return fpc;
+}
+
 // kF8: tq, tk, tv are maps over FP8 e4m3 bytes (boxes of 128 rows x 128 bytes) and T is the output type.
 template <typename T, bool kF8 = false>
 int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
@@ -871,42 +942,7 @@ int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
     const long long total = (long long)fp.n_qtiles * fp.B * fp.Hq;
     if (total > 0x7fffffffll) return -3;
     const int grid = (int)(total < sm_count ? total : sm_count);
-    // Class size of the item order: large enough that the K and V of the kv heads one round of
-    // CTAs works on (about grid / (C * group) of them, Skv * 512 bytes each) fit in a fraction of
-    // L2, but at most half of a head's tiles and 16 (a class that is the whole head makes all
-    // its tiles read the same K/V lines at the same moment, which measured slower).  Under the
-    // causal mask the items of a class differ in length, which costs balance when a head has few
-    // tiles: heads with fewer than 16 keep the plain longest-first order.  When one head alone
-    // fills every CTA, a single class: the plain head-by-head order.
-    FwdParams fpc = fp;
-    int cls_log2 = 0;
-    if (fp.n_qtiles >= grid) {
-        while ((1 << cls_log2) < fp.n_qtiles) ++cls_log2;
-    } else {
-#ifdef FA_PP_CLASS_LOG2
-        cls_log2 = FA_PP_CLASS_LOG2;
-#else
-        const double head_bytes = (kF8 ? 256.0 : 512.0) * fp.Skv / (fp.Hq / fp.Hkv);
-        const double budget = 32.0 * 1024 * 1024;
-        const int half = fp.n_qtiles / 2 < 16 ? fp.n_qtiles / 2 : 16;
-        const int cap = (fp.causal && fp.n_qtiles < 16) ? 1 : half;
-        while ((grid >> cls_log2) * head_bytes > budget && (2 << cls_log2) <= cap) ++cls_log2;
-#endif
-        while (cls_log2 > 0 && (1 << cls_log2) > fp.n_qtiles) --cls_log2;
-    }
-    // From three rounds per head on (56K keys on 148 SMs) and once a head's K and V are past what
-    // L2 keeps, the head-by-head order with whole rounds per head (see PpItems); the empty slots of
-    // a head's last round cost little there because its items are the head's shortest.
-    const double kv_bytes_per_head = 2.0 * fp.Skv * 128 * (kF8 ? 1 : 2);
-    if (!varlen && fp.n_qtiles >= 3 * grid && kv_bytes_per_head > 24.0 * 1024 * 1024) {
-        fpc.rounds_per_head = (fp.n_qtiles + grid - 1) / grid;
-        fpc.by_rph.set(fpc.rounds_per_head);
-    }
-    fpc.cls_log2 = cls_log2;
-    const long long class_items = ((long long)fp.B * fp.Hq) << cls_log2;  // > total only for a single class
-    fpc.by_class.set(class_items > 0x7fffffffll ? 0x7fffffff : (int)class_items);
-    const int last = fp.n_qtiles & ((1 << cls_log2) - 1);
-    fpc.by_lastcls.set(last ? last : 1);
+    const FwdParams fpc = pp_plan_items(fp, grid, kF8 ? 256.0 : 512.0);
     kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, to, fpc, (int)total);
     e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = (int)e; return -7; }

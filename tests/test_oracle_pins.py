@@ -378,6 +378,38 @@ def test_e4m3_values_and_fp8_decode():
     assert torch.allclose(O3, O, rtol=1e-12, atol=1e-14) and torch.allclose(L3, LSE, rtol=1e-12, atol=1e-14)
 
 
+def test_projection_after_attention():
+    # hand example: scores 0 and ln 3 give P = (1/4, 3/4); V = 4 I gives O = (1, 3); W = [[1, 2], [3, 4]]
+    # gives out = (1*1 + 3*3, 1*2 + 3*4) = (10, 14)
+    q = torch.tensor([[[[1.0, 0.0]]]], dtype=torch.float64)
+    k = torch.tensor([[[[0.0, 0.0]], [[math.log(3.0), 0.0]]]], dtype=torch.float64)
+    v = torch.tensor([[[[4.0, 0.0]], [[0.0, 4.0]]]], dtype=torch.float64)
+    w = torch.tensor([[1.0, 2.0], [3.0, 4.0]], dtype=torch.float64)
+    O, LSE, out = oracle.attention_proj(q, k, v, w, False, 1.0)
+    assert torch.allclose(O[0, 0, 0], torch.tensor([1.0, 3.0], dtype=torch.float64), atol=1e-14)
+    assert torch.allclose(out[0, 0], torch.tensor([10.0, 14.0], dtype=torch.float64), atol=1e-13)
+    # W = I returns O (rounded to the operands' type: the projection reads the 16-bit output), in the
+    # order (head, d) of a row; a permutation matrix picks columns; linear in W
+    B, Sq, Skv, Hq, Hkv, d = 2, 5, 9, 4, 2, 8
+    qh, kh, vh = rnd((B, Sq, Hq, d), 81).half(), rnd((B, Skv, Hkv, d), 82).half(), rnd((B, Skv, Hkv, d), 83).half()
+    K = Hq * d
+    O, LSE, out = oracle.attention_proj(qh, kh, vh, torch.eye(K, dtype=torch.float64), True, 0.3)
+    O2, L2 = oracle.attention_full(qh, kh, vh, True, 0.3)
+    assert torch.equal(O, O2) and torch.equal(LSE, L2)
+    assert torch.equal(out, O.half().double().reshape(B, Sq, K))
+    perm = torch.randperm(K, generator=torch.Generator().manual_seed(5))
+    P = torch.zeros(K, K, dtype=torch.float64); P[perm, torch.arange(K)] = 1.0       # out[:, n] = O[:, perm[n]]
+    assert torch.equal(oracle.attention_proj(qh, kh, vh, P, True, 0.3)[2], O.half().double().reshape(B, Sq, K)[..., perm])
+    w1, w2 = rnd((K, 6), 84).double(), rnd((K, 6), 85).double()
+    o1 = oracle.attention_proj(qh, kh, vh, w1, False, 0.3)[2]
+    o2 = oracle.attention_proj(qh, kh, vh, w2, False, 0.3)[2]
+    o12 = oracle.attention_proj(qh, kh, vh, w1 + 2 * w2, False, 0.3)[2]
+    assert torch.allclose(o12, o1 + 2 * o2, rtol=1e-12, atol=1e-12)
+    # float64 operands are not rounded in between
+    O64, _, out64 = oracle.attention_proj(qh.double(), kh.double(), vh.double(), w1, False, 0.3)
+    assert torch.allclose(out64, O64.reshape(B, Sq, K) @ w1, rtol=1e-13, atol=1e-13)
+
+
 def test_fp8_attention_is_attention_on_the_widened_operands():
     # 8-bit operands: the definition on Q = q_scale * value(bits) etc.  Pins: torch's own widening and
     # softmax.matmul in float64 (library routines the oracle does not use); the factors of q and k

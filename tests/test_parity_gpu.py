@@ -551,6 +551,93 @@ def test_fp8_prefill_bench_sizes_sampled(fa):
         print(f"fp8 {cfg.name}: max|dO| {worst:.2e} (largest allowance {allow:.2e})")
 
 
+# ------------------------------------------------------------------ attention + output projection
+def proj_allowance(o_ref, out_ref, w, ulp):
+    """Sound bound on |d out| from the attention gate: every element of the 16-bit O the projection
+    reads is within TOL_O + 2 ulp |O| of the oracle's rounded O (the gate plus the two roundings),
+    which the weights carry into out as sum_k |W_kn| (...); the stored 16-bit out adds ulp |out|."""
+    B, Sq, Hq, d = o_ref.shape
+    per_k = (TOL_O + 2 * ulp * o_ref.abs()).reshape(B, Sq, Hq * d)
+    return torch.matmul(per_k, w.abs()) + ulp * out_ref.abs()
+
+
+def proj_case(fa, B, Hq, Hkv, Sq, Skv, d_model, causal, dtype, seed, w_kind="dense", rows=None):
+    cfg = synth.PrefillConfig("proj", B, Hq, Hkv, Sq, Skv, dtype=dtype, causal=causal, seed=seed)
+    q, k, v = synth.prefill_inputs(cfg, "cpu" if rows is None else DEV)
+    K = Hq * 128
+    gen = torch.Generator().manual_seed(seed + 1)
+    if w_kind == "dense":
+        w = (torch.randn(K, d_model, generator=gen) / math.sqrt(K)).to(q.dtype)
+    else:   # every column has exactly one entry, +-2^e: out[:, n] = +-2^e O[:, src[n]], exact in the accumulator
+        src = torch.randint(0, K, (d_model,), generator=gen)
+        val = torch.tensor([1.0, -1.0, 0.5, -2.0])[torch.randint(0, 4, (d_model,), generator=gen)]
+        w = torch.zeros(K, d_model)
+        w[src, torch.arange(d_model)] = val
+        w = w.to(q.dtype)
+    qd, kd, vd, wd = q.to(DEV), k.to(DEV), v.to(DEV), w.to(DEV)
+    ws = torch.empty(max(4, fa.fa_forward_proj_workspace_bytes(B, Sq)), dtype=torch.uint8, device=DEV)
+    res = []
+    for fused in (True, False):
+        o, chk_o = guard_alloc((B, Sq, Hq, 128), q.dtype, DEV)
+        lse, chk_l = guard_alloc((B, Hq, Sq), torch.float32, DEV)
+        out, chk_out = guard_alloc((B, Sq, d_model), q.dtype, DEV)
+        fa.fa_forward_proj(qd, kd, vd, wd, o, lse, out, causal, cfg.scale, fused, ws)
+        torch.cuda.synchronize()
+        check_status(fa)
+        chk_o(); chk_l(); chk_out()
+        assert not torch.isnan(o).any() and not torch.isnan(lse).any() and not torch.isnan(out).any()
+        res.append((o, lse, out))
+    # one launch or two: the same kernels on the same data in the same order
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1]) and torch.equal(res[0][2], res[1][2])
+    o, lse, out = res[0]
+    ulp = 2.0 ** -8 if dtype == "bf16" else 2.0 ** -11
+    what = f"proj B{B} Hq{Hq} Hkv{Hkv} Sq{Sq} Skv{Skv} N{d_model} causal{int(causal)} {dtype} {w_kind}"
+    if rows is None:
+        o_ref, l_ref, out_ref = oracle.attention_proj(q, k, v, w, causal, cfg.scale)
+        absv = oracle.attention_full(q, k, v.abs(), causal, cfg.scale)[0] if dtype == "bf16" else None
+        assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv, what=what)
+        got = out.double().cpu()
+    else:
+        # sampled (b, i): the oracle on those batch entries' rows, all heads
+        got_l, ref_l, oref_l = [], [], []
+        for (b, i) in rows:
+            r3 = [(0, h, i) for h in range(Hq)]
+            orow, _ = oracle.attention_rows(q[b:b + 1].cpu(), k[b:b + 1].cpu(), v[b:b + 1].cpu(), causal, cfg.scale, r3)
+            o16 = orow.to(q.dtype).double()
+            ref_l.append(o16.reshape(1, K) @ w.double())
+            oref_l.append(orow.reshape(1, 1, Hq, 128))
+            got_l.append(out[b, i].double().cpu().reshape(1, d_model))
+        got, out_ref, o_ref = torch.cat(got_l).unsqueeze(0), torch.cat(ref_l).unsqueeze(0), torch.cat(oref_l, dim=1)
+    diff = (got - out_ref).abs()
+    allow = proj_allowance(o_ref, out_ref, w.double(), ulp)
+    assert float((diff - allow).max()) <= 0.0, f"{what}: max(|d out| - bound) = {float((diff - allow).max()):.3e}"
+    # the bound is sound but wide for a dense weight; a dropped head or k-block shows in the row norms
+    rel = float(((got - out_ref).norm(dim=-1) / out_ref.norm(dim=-1).clamp_min(1e-30)).max())
+    assert rel <= (2e-2 if dtype == "bf16" else 5e-3), f"{what}: relative row error {rel:.3e}"
+    return float(diff.max()), rel
+
+
+@pytest.mark.parametrize("w_kind", ["select", "dense"])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_attention_with_output_projection_small(fa, dtype, w_kind):
+    proj_case(fa, 1, 2, 2, 512, 512, 256, True, dtype, seed=120, w_kind=w_kind)          # C1's attention
+    proj_case(fa, 2, 4, 2, 300, 300, 512, True, dtype, seed=121, w_kind=w_kind)          # 4 heads, 512 columns, ragged rows
+    proj_case(fa, 1, 4, 1, 130, 1300, 768, False, dtype, seed=122, w_kind=w_kind)
+
+
+def test_attention_with_output_projection_many_blocks(fa):
+    # more projection items than CTAs, several per CTA through both accumulators and around the ring
+    proj_case(fa, 3, 8, 8, 700, 700, 1024, True, "fp16", seed=123, w_kind="select")
+    proj_case(fa, 3, 8, 8, 700, 700, 1024, True, "fp16", seed=124, w_kind="dense")
+
+
+def test_attention_with_output_projection_c2_sampled(fa):
+    c = synth.C2
+    rows = [(0, 0), (0, 127), (0, 128), (1, 1000), (2, 2047), (3, 5), (3, 1029), (1, 255)]
+    worst, rel = proj_case(fa, c.B, c.Hq, c.Hkv, c.Sq, c.Skv, 4096, True, "fp16", seed=125, w_kind="dense", rows=rows)
+    print(f"C2 + projection to 4096 columns: max|d out| {worst:.2e}, relative row error {rel:.2e}")
+
+
 # ------------------------------------------------------------------ packed variable-length batches
 def varlen_case(fa, cfg, what):
     q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
