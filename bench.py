@@ -37,6 +37,17 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def load_traffic():
+    """DRAM bytes per launch of the two roofline kernels, from the ncu captures kept under
+    profiles/ (the file records the commit each figure was captured at)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return {}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -53,7 +64,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -101,7 +112,8 @@ class ClockSampler:
             self._thread.join()
         med = statistics.median(self.samples) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "sm_mhz_min": min(self.samples) if self.samples else None,
+                "sm_mhz_max_seen": max(self.samples) if self.samples else None, "period_ms": self.period * 1e3}
 
 
 # --------------------------------------------------------------------------- workload
@@ -228,6 +240,10 @@ def run_product(args, rank, world, local_rank):
         "gpu_launches": args.steps * (1 + 2 * len(dec)),
         "clocks": clocks,
     }
+    if clocks.get("sm_mhz"):
+        # prefill time in SM clocks (ms x median MHz over the timed region): lets runs on boxes whose
+        # clocks settled differently be compared; approximate, since the samples cover whole steps
+        out["prefill"]["kclocks_at_median_mhz"] = round(part_ms[0] * clocks["sm_mhz"], 1)
     for i, d in enumerate(dec):
         gbs = whole_job_rate(d["bytes"], world, part_ms[1 + i]) / 1e9
         out["decode_" + ("mha" if i == 0 else "gqa")] = {
@@ -239,7 +255,10 @@ def run_product(args, rank, world, local_rank):
     # `traffic`: DRAM bytes per launch from one ncu capture (profiles/): the C2 prefill launch
     # itself, and for decode a 4.3 GB case of the same kernel whose dram bytes were 1.007 x its
     # algorithmic bytes, scaled to this launch by the cache bytes it scans
-    c2_traffic = 304.0e6 if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
+    traffic = load_traffic()
+    c2_rec = traffic.get("prefill_c2", {})
+    c2_traffic = c2_rec.get("dram_bytes_per_launch") if (pc.B, pc.Hq, pc.Sq) == (4, 32, 2048) else None
+    dec_ratio = traffic.get("decode_split", {}).get("dram_bytes_over_algorithmic")
     algo_prefill_bytes = (2.0 * pc.B * pc.Sq * pc.Hq + 2.0 * pc.B * pc.Skv * pc.Hkv) * pc.d * 2 + 4.0 * pc.B * pc.Hq * pc.Sq
     out["roofline"] = {"kernel": "fa_fwd_pingpong_kernel (prefill C2, the kernel behind `value`; the library picks it for Skv >= 1024)", "bound": "tensor",
                        "achieved": round(tflops / world, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -247,14 +266,16 @@ def run_product(args, rank, world, local_rank):
                        "peak_source": peaks["source"] + " bf16 GEMM burst (of measured; fp16 has the same nominal rate)",
                        "frac_nominal": round(tflops / world / NOMINAL_TENSOR_TFLOPS, 4),
                        "algorithmic_flops": pc.flops(), "algorithmic_bytes": algo_prefill_bytes,
-                       "traffic": c2_traffic}
+                       "traffic": c2_traffic, "traffic_source": c2_rec.get("source")}
     g0 = out["decode_mha"]["gbs"] / world
     out["roofline_decode"] = {"kernel": "fa_decode_split_mma_kernel (decode Hkv=32, the dominant kernel by time)",
                               "bound": "hbm", "achieved": round(g0, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": round(g0 / peaks["hbm_gbs"], 4),
                               "peak_source": peaks["source"] + " copy bandwidth (of measured; the scan only reads)",
                               "frac_nominal": round(g0 / NOMINAL_HBM_GBS, 4),
-                              "algorithmic_bytes": dec[0]["bytes"], "traffic": round(1.007 * dec[0]["bytes"])}
+                              "algorithmic_bytes": dec[0]["bytes"],
+                              "traffic": round(dec_ratio * dec[0]["bytes"]) if dec_ratio else None,
+                              "traffic_source": traffic.get("decode_split", {}).get("source")}
 
     if rank == 0:
         # the same prefill launch back to back, without the decode passes in between: inside the
@@ -279,6 +300,8 @@ def run_product(args, rank, world, local_rank):
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
         out["prefill_d256"] = run_d256(fa, dev, peaks, small=args.small)
+        out["prefill_fp8"] = run_prefill_fp8(fa, dev, peaks, small=args.small)
+        out["prefill_proj"] = run_prefill_proj(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
         out["cpu_baseline"] = run_cpu_baseline(pc, budget_s=args.cpu_seconds)
         print(json.dumps(out), flush=True)
@@ -289,11 +312,11 @@ def run_long_context(fa, dev, peaks):
     configurations (bf16, causal), which the library serves with its ping-pong kernel.  Inputs
     are larger than L2 (>= 192 MiB per launch); CUDA events around back-to-back launches."""
     res = {"kernel": "fa_fwd_pingpong_kernel (the same kernel as for C2)", "dtype": "bf16", "cases": {}}
-    for cfg, iters in ((synth.C3[8192], 10), (synth.C3[32768], 3), (synth.C4, 5)):
+    for cfg, iters in ((synth.C3[8192], 10), (synth.C3[32768], 3), (synth.C4, 5), (synth.C3[131072], 2), (synth.C3[262144], 1)):
         q, k, v = synth.prefill_inputs(cfg, device=dev)
         o = torch.empty_like(q)
         lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
-        for _ in range(3):
+        for _ in range(3 if cfg.Sq <= 32768 else 1):
             fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -312,6 +335,71 @@ def run_long_context(fa, dev, peaks):
     if rc != 0:
         raise SystemExit(f"device status {rc} at {where} block {blk}")
     return res
+
+
+def _time_launches(fa, run, warm, iters):
+    for _ in range(warm):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    return e0.elapsed_time(e1) / iters
+
+
+def run_prefill_fp8(fa, dev, peaks, small=False):
+    """The headline shape and the 8K long-context shape with 8-bit operands (fa_forward_fp8: Q, K, V
+    and the probabilities as FP8 e4m3 on the tensor cores), next to the 16-bit kernel on the same
+    numbers in the same process, outside the timed steps.  The fp8 tensor peak is twice the 16-bit
+    one; the fractions below are against that."""
+    res = {"kernel": "fa_fwd_pingpong_kernel, 8-bit operand instantiation (tcgen05 kind::f8f6f4)", "cases": {}}
+    cfgs = [synth.PrefillConfig("C2-small", 1, 8, 8, 1024, 1024, seed=5)] if small else [synth.C2, synth.C3[8192]]
+    for cfg in cfgs:
+        c16 = synth.PrefillConfig(cfg.name, cfg.B, cfg.Hq, cfg.Hkv, cfg.Sq, cfg.Skv, dtype="fp16", causal=True, seed=cfg.seed)
+        q, k, v = synth.prefill_inputs(c16, device=dev)
+        q8, k8, v8 = synth.fp8_operands(q, k, v, 0.125, 0.25, 0.0625)
+        o = torch.empty_like(q)
+        lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+        ms16 = _time_launches(fa, lambda: fa.fa_forward(q, k, v, o, lse, True, c16.scale), 20, 20)
+        ms8 = _time_launches(fa, lambda: fa.fa_forward_fp8(q8, k8, v8, o, lse, True, c16.scale, 0.125, 0.25, 0.0625), 20, 20)
+        tf8 = c16.flops() / (ms8 * 1e-3) / 1e12
+        res["cases"][cfg.name] = {"ms_fp8": round(ms8, 4), "tflops_fp8": round(tf8, 1), "ms_fp16": round(ms16, 4),
+                                  "tflops_fp16": round(c16.flops() / (ms16 * 1e-3) / 1e12, 1),
+                                  "speedup": round(ms16 / ms8, 3),
+                                  "frac_nominal_fp8_tensor": round(tf8 / (2 * NOMINAL_TENSOR_TFLOPS), 4)}
+        del q, k, v, q8, k8, v8, o, lse
+    return res
+
+
+def run_prefill_proj(fa, dev, peaks, small=False):
+    """Attention followed by the output projection to d_model = Hq * 128 columns (fa_forward_proj) on
+    the headline shape: one launch against the same two kernels as two launches, outside the timed
+    steps; torch.matmul on the same operands for the size of the projection itself."""
+    cfg = synth.PrefillConfig("C2-small", 1, 8, 8, 1024, 1024, seed=5) if small else synth.C2
+    q, k, v = synth.prefill_inputs(cfg, device=dev)
+    K = cfg.Hq * cfg.d
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + 31)
+    w = (torch.randn(K, K, generator=gen, device=dev) / math.sqrt(K)).to(q.dtype)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+    out = torch.empty(cfg.B, cfg.Sq, K, dtype=q.dtype, device=dev)
+    ws = torch.empty(max(4, fa.fa_forward_proj_workspace_bytes(cfg.B, cfg.Sq)), dtype=torch.uint8, device=dev)
+    ms_att = _time_launches(fa, lambda: fa.fa_forward_ex(q, k, v, o, lse, True, cfg.scale, variant=3), 20, 20)
+    ms_two = _time_launches(fa, lambda: fa.fa_forward_proj(q, k, v, w, o, lse, out, True, cfg.scale, False, ws), 20, 20)
+    ms_one = _time_launches(fa, lambda: fa.fa_forward_proj(q, k, v, w, o, lse, out, True, cfg.scale, True, ws), 20, 20)
+    ms_mm = _time_launches(fa, lambda: torch.matmul(o.view(cfg.B, cfg.Sq, K), w, out=out), 20, 20)
+    fl = cfg.flops() + 2.0 * cfg.B * cfg.Sq * K * K
+    return {"workload": f"{cfg.name} + projection [{K} x {K}], fp16", "ms_one_launch": round(ms_one, 4),
+            "ms_two_launches": round(ms_two, 4), "ms_attention_alone": round(ms_att, 4),
+            "ms_projection_by_difference": round(ms_two - ms_att, 4), "ms_torch_matmul_same_projection": round(ms_mm, 4),
+            "tflops_one_launch": round(fl / (ms_one * 1e-3) / 1e12, 1), "tflops_two_launches": round(fl / (ms_two * 1e-3) / 1e12, 1)}
 
 
 def run_d64(fa, dev, peaks, small=False, iters=10):
@@ -607,6 +695,32 @@ def run_reference(args, rank, world):
         "gpu_launches": 0}), flush=True)
 
 
+def _free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _spawn_entry(rank, world, port, fn, fn_args):
+    os.environ.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world),
+                       "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    fn(*fn_args)
+
+
+def spawn_ranks(world: int, fn, fn_args=()):
+    """Runs fn(*fn_args) in `world` processes with the environment torchrun would give them
+    (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, MASTER_PORT); returns when all have
+    exited and raises if one failed."""
+    import torch.multiprocessing as mp
+    mp.spawn(_spawn_entry, args=(world, _free_port(), fn, fn_args), nprocs=world, join=True)
+
+
+def _rank_main(argv):
+    sys.argv = [sys.argv[0]] + list(argv)
+    main()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -617,6 +731,10 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
 
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and args.impl == "product":
+        # plain `python bench.py --gpus N`: start the N ranks here (under torchrun they exist already)
+        spawn_ranks(args.gpus, _rank_main, (sys.argv[1:],))
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

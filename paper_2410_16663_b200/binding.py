@@ -169,7 +169,7 @@ def fa_forward_fp8(q, k, v, o, lse, causal: bool, scale: float, q_scale: float, 
     dt = FA_DTYPE_BF16 if o.dtype == torch.bfloat16 else FA_DTYPE_FP16
     rc = lib.fa_forward_fp8(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, Hq, Hkv, Sq, Skv, d, int(bool(causal)),
                             float(scale), float(q_scale), float(k_scale), float(v_scale), dt, _stream())
-    return _check(rc, "fa_forward_fp8", "fa_forward_proj", "fa_forward_proj_workspace_bytes", raise_on_error)
+    return _check(rc, "fa_forward_fp8", raise_on_error)
 
 
 def fa_forward_proj_workspace_bytes(B: int, Sq: int) -> int:

@@ -40,10 +40,6 @@ namespace fa {
 constexpr int kPpNK = FA_PP_NK;   // K ring slots
 constexpr int kPpNV = FA_PP_NV;   // V ring slots
 constexpr int kPpQBufs = 2;
-#ifndef FA_PP_TURNS
-#define FA_PP_TURNS 0
-#endif
-constexpr bool kPpTurns = FA_PP_TURNS != 0;
 static_assert((kPpQBufs + kPpNK + kPpNV) * kTileBytes + 3072 <= 232448, "shared memory budget");
 
 // What changes with FP8 e4m3 operands (kF8; Appendix D.2 evaluates the operator with 8-bit
@@ -220,12 +216,8 @@ __device__ __forceinline__ void pp_exp_chunk(const uint32_t (&s)[128], int c, ui
                 f2_fma(f2_pack(__uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1])), sc2, nm2);
             float x0, x1;
             f2_unpack(x01, x0, x1);
-            if (q < kPolyPairs) {
-                exp2_poly_pair(fmaxf(x0, -125.f), fmaxf(x1, -125.f), pv[2 * q], pv[2 * q + 1]);
-            } else {
-                pv[2 * q] = fast_exp2(x0);
-                pv[2 * q + 1] = fast_exp2(x1);
-            }
+            pv[2 * q] = fast_exp2(x0);
+            pv[2 * q + 1] = fast_exp2(x1);
         }
         la = f2_add(la, f2_pack(pv[0], pv[1]));
         lb = f2_add(lb, f2_pack(pv[2], pv[3]));
@@ -518,10 +510,6 @@ struct PpSoftmax {
         const float neg_ms = -((m_new == -INFINITY) ? 0.f : m_new) * scale_log2 + (kF8 ? kP8ScaleLog2 : 0.f);
         const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
         uint64_t la = f2_pack(0.f, 0.f), lb = la;
-        if (kPpTurns && g >= 1) {
-            // the two warpgroups take turns at the exponentials
-            if (!pp_warp_wait(pp_bar(bar0, ppb::p_full + (1 - w)), ((g - 1) >> 1) & 1, abort_flag, 122 + w)) return false;
-        }
         {
             uint32_t pk[Op::kPCols];
             const bool p_free = g < 2 || mbar_test(pp_bar(bar0, ppb::pv_done + w), ((g >> 1) - 1) & 1);

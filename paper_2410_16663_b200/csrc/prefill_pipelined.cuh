@@ -1,4 +1,4 @@
-// Prefill forward, pipelined variant (the default kernel).
+// Prefill forward, paired-tile pipelined variant (the library's choice below 1024 keys).
 //
 // A persistent CTA (one per SM, 384 threads) walks a static list of work items, longest
 // first, in boustrophedon order over the CTAs.  An item is a pair of adjacent 128-row query
@@ -40,10 +40,6 @@ constexpr int kPipeSoftmaxRegs = 224, kPipeOtherRegs = 56;
 static_assert(256 * (kPipeSoftmaxRegs - kPipeLaunchRegs) <= 128 * (kPipeLaunchRegs - kPipeOtherRegs),
               "setmaxnreg.inc would wait for registers nobody releases");
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
-#ifndef FA_POLY_PAIRS
-#define FA_POLY_PAIRS 0
-#endif
-constexpr int kPolyPairs = FA_POLY_PAIRS;   // of every 4 column pairs, how many take the polynomial exp2
 
 // Work item taken by this CTA in its k-th round.  Items are listed longest first; rounds
 // alternate direction across the CTAs (boustrophedon) so that every CTA gets nearly the same
@@ -160,9 +156,7 @@ __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, ui
         }
         l_run += l0 + l1;
     } else {
-        // packed f32x2 arithmetic: one FMA and one add per pair of columns.  Of every four pairs,
-        // kPolyPairs take the polynomial exp2 on the FMA pipe and the rest the special-function
-        // unit, so that neither pipe alone bounds the softmax.
+        // packed f32x2 arithmetic: one FMA and one add per pair of columns
         const uint64_t sc2 = f2_pack(scale_log2, scale_log2), nm2 = f2_pack(neg_ms, neg_ms);
         uint64_t la = f2_pack(0.f, 0.f), lb = la;
 #pragma unroll
@@ -178,12 +172,8 @@ __device__ __forceinline__ void softmax_step(uint32_t (&s)[128], uint32_t tS, ui
                         f2_fma(f2_pack(__uint_as_float(s[e + 2 * q]), __uint_as_float(s[e + 2 * q + 1])), sc2, nm2);
                     float x0, x1;
                     f2_unpack(x01, x0, x1);
-                    if (q < kPolyPairs) {
-                        exp2_poly_pair(fmaxf(x0, -125.f), fmaxf(x1, -125.f), pv[2 * q], pv[2 * q + 1]);
-                    } else {
-                        pv[2 * q] = fast_exp2(x0);
-                        pv[2 * q + 1] = fast_exp2(x1);
-                    }
+                    pv[2 * q] = fast_exp2(x0);
+                    pv[2 * q + 1] = fast_exp2(x1);
                 }
                 la = f2_add(la, f2_pack(pv[0], pv[1]));
                 lb = f2_add(lb, f2_pack(pv[2], pv[3]));

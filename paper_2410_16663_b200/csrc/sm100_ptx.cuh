@@ -372,29 +372,6 @@ __device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
     asm("mul.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
-// 2^x for a pair of values on the FMA pipe instead of the special-function unit: round x to
-// the nearest integer with the 1.5*2^23 trick, evaluate a cubic for 2^frac on [-0.5, 0.5]
-// (relative error 7.5e-5, below the rounding of the 16-bit probabilities it feeds), and add the
-// integer part to the exponent field.  Inputs must be >= -125 (callers clamp).
-__device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float& r0, float& r1) {
-    const uint64_t magic = f2_pack(12582912.f, 12582912.f), neg_magic = f2_pack(-12582912.f, -12582912.f);
-    const uint64_t neg_one = f2_pack(-1.f, -1.f);
-    const uint64_t c0 = f2_pack(0.9999280572f, 0.9999280572f), c1 = f2_pack(0.6932609677f, 0.6932609677f);
-    const uint64_t c2 = f2_pack(0.2426111251f, 0.2426111251f), c3 = f2_pack(0.0551716462f, 0.0551716462f);
-    const uint64_t x = f2_pack(x0, x1);
-    const uint64_t t = f2_add(x, magic);                 // integer part lands in the low mantissa bits
-    const uint64_t xi = f2_add(t, neg_magic);
-    const uint64_t xf = f2_fma(xi, neg_one, x);          // x - round(x)
-    uint64_t pl = f2_fma(c3, xf, c2);
-    pl = f2_fma(pl, xf, c1);
-    pl = f2_fma(pl, xf, c0);
-    float t0, t1, p0, p1;
-    f2_unpack(t, t0, t1);
-    f2_unpack(pl, p0, p1);
-    r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-    r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
-
 // Register reallocation between warpgroups (all four warps of a warpgroup execute it).
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {

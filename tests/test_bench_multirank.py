@@ -45,3 +45,27 @@ def test_single_rank_is_identity():
     import bench
     assert bench.max_over_ranks([3.0, 1.5], 1, torch.device("cpu")) == [3.0, 1.5]
     assert bench.whole_job_rate(10.0, 1, 2.0) == 5000.0
+
+
+def _spawned_rank(result_dir):
+    # what `python bench.py --gpus 2` starts per rank (bench.spawn_ranks), here with the gloo backend
+    sys.path.insert(0, ROOT)
+    import bench
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]) == rank
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    red = bench.max_over_ranks([10.0 * (rank + 1), 1.0], world, torch.device("cpu"))
+    with open(os.path.join(result_dir, f"rank{rank}.txt"), "w") as f:
+        f.write(repr((world, red)))
+    dist.destroy_process_group()
+
+
+def test_gpus_flag_spawns_its_own_ranks(tmp_path):
+    # `--gpus N` without torchrun goes through bench.spawn_ranks: N processes with torchrun's
+    # environment that find each other on 127.0.0.1
+    sys.path.insert(0, ROOT)
+    import bench
+    bench.spawn_ranks(2, _spawned_rank, (str(tmp_path),))
+    for r in range(2):
+        world, red = eval(open(tmp_path / f"rank{r}.txt").read())
+        assert world == 2 and red == [20.0, 1.0]
