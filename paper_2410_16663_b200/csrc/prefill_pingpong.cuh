@@ -892,6 +892,16 @@ inline FwdParams pp_plan_items(const FwdParams& fp, int grid, double bytes_per_k
         while ((grid >> cls_log2) * head_bytes > budget && (2 << cls_log2) <= cap) ++cls_log2;
         while (cls_log2 > 0 && (1 << cls_log2) > fp.n_qtiles) --cls_log2;
     }
+    if (varlen) {
+        // Packed batches: sequence by sequence and head by head, a head's tiles longest first (a
+        // single class).  The lengths differ from sequence to sequence, so classes of tiles across
+        // heads would mix long and short items in a round; head by head a round holds the tiles
+        // of two or three neighbouring heads, which are of a size and share their K and V
+        // (measured on 32 requests of 256 to 8192 tokens: 6.0 ms against 6.8 to 7.7 ms with
+        // classes of 1 to 16 tiles).
+        cls_log2 = 0;
+        while ((1 << cls_log2) < fp.n_qtiles) ++cls_log2;
+    }
     // From three rounds per head on (56K keys on 148 SMs) and once a head's K and V are past what
     // L2 keeps, the head-by-head order with whole rounds per head (see PpItems); the empty slots of
     // a head's last round cost little there because its items are the head's shortest.

@@ -13,8 +13,8 @@
 //                         boxes of 64 columns) -- 48 KiB;
 //   warp 8  (one thread): per stage four tcgen05.mma 128 x 256 x 16 into one of two 256-column
 //                         accumulators in tensor memory;
-//   warps 0-7           : warpgroup a drains accumulator a: one thread per row, 128 columns at a
-//                         time, rounded to 16 bits and written with whole-line stores.
+//   warps 0-7           : warpgroup a drains accumulator a: one thread per row, 32 columns at a
+//                         time, rounded to 16 bits and stored.
 // In the fused launch a row block may be loaded only after every head's attention output for it
 // has reached global memory: the attention epilogue counts its completed TMA stores per row block
 // in `done`, and the loading thread waits (bounded) for the count before the block's first load.
@@ -150,26 +150,28 @@ __device__ __forceinline__ void proj_phase(const CUtensorMap* tm_a, const CUtens
             ++mine;
             tc_fence_after();
             const int row = qt * kTile + r;
-            const int rows_live = min(32, pp.Sq - (qt * kTile + (warp & 3) * 32));   // of this warp's 32 rows
             T* row_ptr = static_cast<T*>(pp.out) + ((long long)b * pp.Sq + row) * pp.N + (long long)cb * 256;
+            // 32 columns at a time: few registers, and a thread's eight stores of a chunk fill
+            // whole 64-byte pieces of its row (the lines are completed in L2 before they go to HBM)
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                uint32_t acc[128];
-                const uint32_t ta = tmem + lane_sel + 256 * a + 128 * half;
-                tmem_ld_x32(ta, *reinterpret_cast<uint32_t(*)[32]>(&acc[0]));
-                tmem_ld_x32(ta + 32, *reinterpret_cast<uint32_t(*)[32]>(&acc[32]));
-                tmem_ld_x32(ta + 64, *reinterpret_cast<uint32_t(*)[32]>(&acc[64]));
-                tmem_ld_x32(ta + 96, *reinterpret_cast<uint32_t(*)[32]>(&acc[96]));
+            for (int c = 0; c < 8; ++c) {
+                uint32_t acc[32];
+                tmem_ld_x32(tmem + lane_sel + 256 * a + 32 * c, acc);
                 tmem_wait_ld();
-                if (half == 1) {
-                    // the whole accumulator is in registers: the next item may overwrite it
+                if (c == 7) {
+                    // the whole accumulator has been read: the next item may overwrite it
                     tc_fence_before();
                     mbar_arrive(pp_bar(bar0, prb::acc_empty + a));
                 }
-                uint32_t w[64];
+                if (row < pp.Sq) {
+                    uint4* dst = reinterpret_cast<uint4*>(row_ptr + 32 * c);
 #pragma unroll
-                for (int i = 0; i < 64; ++i) w[i] = pack2<T>(__uint_as_float(acc[2 * i]), __uint_as_float(acc[2 * i + 1]));
-                if (rows_live > 0) store_rows_coalesced<T>(row_ptr + half * 128, pp.N, rows_live, w);
+                    for (int i = 0; i < 4; ++i)
+                        dst[i] = make_uint4(pack2<T>(__uint_as_float(acc[8 * i]), __uint_as_float(acc[8 * i + 1])),
+                                            pack2<T>(__uint_as_float(acc[8 * i + 2]), __uint_as_float(acc[8 * i + 3])),
+                                            pack2<T>(__uint_as_float(acc[8 * i + 4]), __uint_as_float(acc[8 * i + 5])),
+                                            pack2<T>(__uint_as_float(acc[8 * i + 6]), __uint_as_float(acc[8 * i + 7])));
+                }
             }
         }
     }
@@ -203,9 +205,6 @@ fa_proj_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_holder;
-    // the epilogue holds 128 accumulator columns and their packed form per thread
-    if (warp < 8) setmaxnreg_inc<kPipeSoftmaxRegs>();
-    else setmaxnreg_dec<kPipeOtherRegs>();
     proj_phase<T>(&tm_a, &tm_w, pp, bar0, smem_base, tmem_base, &abort_word);
     tc_fence_before();
     __syncthreads();
