@@ -3,6 +3,8 @@
 Meant for profilers (ncu wraps this command) and quick timing:
   python -m paper_2410_16663_b200.run_case prefill --B 1 --H 32 --Hkv 32 --S 8192 --dtype bf16 --iters 3
   python -m paper_2410_16663_b200.run_case decode  --B 16 --H 32 --Hkv 8 --Smax 16384 --iters 3
+  python -m paper_2410_16663_b200.run_case prefill --B 1 --H 32 --S 8192 --fp8           (8-bit operands)
+  python -m paper_2410_16663_b200.run_case proj    --B 4 --H 32 --S 2048 --fused 1       (attention + projection)
 """
 from __future__ import annotations
 
@@ -17,7 +19,7 @@ from . import inputs as synth
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["prefill", "decode"])
+    ap.add_argument("kind", choices=["prefill", "decode", "proj"])
     ap.add_argument("--B", type=int, default=1)
     ap.add_argument("--H", type=int, default=32)
     ap.add_argument("--Hkv", type=int, default=0)
@@ -27,7 +29,9 @@ def main():
     ap.add_argument("--d", type=int, default=128, choices=[64, 128, 256], help="head dimension (prefill only)")
     ap.add_argument("--dtype", default="fp16", choices=["fp16", "bf16"])
     ap.add_argument("--noncausal", action="store_true")
-    ap.add_argument("--fp8", action="store_true", help="decode: the cache as FP8 e4m3 (factors 1/4 and 1/8)")
+    ap.add_argument("--fp8", action="store_true", help="decode: the cache as FP8 e4m3 (factors 1/4 and 1/8); "
+                                                       "prefill: q, k, v as FP8 e4m3 (fa_forward_fp8)")
+    ap.add_argument("--fused", type=int, default=1, help="proj: one launch (1) or two (0)")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
@@ -41,7 +45,23 @@ def main():
         o = torch.empty_like(q)
         lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
         run = lambda: fa.fa_forward_ex(q, k, v, o, lse, cfg.causal, cfg.scale, variant=a.variant)
+        if a.fp8:
+            q8, k8, v8 = synth.fp8_operands(q, k, v, 0.125, 0.25, 0.0625)
+            o = torch.empty(q.shape, dtype=torch.float16, device=dev)
+            run = lambda: fa.fa_forward_fp8(q8, k8, v8, o, lse, cfg.causal, cfg.scale, 0.125, 0.25, 0.0625)
         work, unit = cfg.flops() / 1e12, "TFLOPS"
+    elif a.kind == "proj":
+        cfg = synth.PrefillConfig("case", a.B, a.H, hkv, a.S, a.Skv or a.S, d=128, dtype=a.dtype,
+                                  causal=not a.noncausal, seed=7)
+        q, k, v = synth.prefill_inputs(cfg, dev)
+        K = a.H * 128
+        w = (torch.randn(K, K, device=dev) / math.sqrt(K)).to(q.dtype)
+        o = torch.empty_like(q)
+        lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+        out = torch.empty(cfg.B, cfg.Sq, K, dtype=q.dtype, device=dev)
+        ws = torch.empty(max(4, fa.fa_forward_proj_workspace_bytes(cfg.B, cfg.Sq)), dtype=torch.uint8, device=dev)
+        run = lambda: fa.fa_forward_proj(q, k, v, w, o, lse, out, cfg.causal, cfg.scale, bool(a.fused), ws)
+        work, unit = (cfg.flops() + 2.0 * cfg.B * cfg.Sq * K * K) / 1e12, "TFLOPS"
     else:
         cfg = synth.DecodeConfig("case", a.B, a.H, hkv, a.Smax, max(1, a.Smax // 32), a.Smax, seed=8)
         q, k, v, sl = synth.decode_inputs(cfg, dev, poison=True)
