@@ -297,3 +297,28 @@ def test_forward_fp8_validation(fa):
     assert call(scale=-0.1) == fa.FA_ERR_UNSUPPORTED
     assert call(qp=None) == fa.FA_ERR_NULL and call(op=None) == fa.FA_ERR_NULL and call(kp=None) == fa.FA_ERR_NULL
     assert call(qp=P(q) + 4) == fa.FA_ERR_ALIGN and call(op=P(o) + 2) == fa.FA_ERR_ALIGN
+
+
+def test_forward_proj_validation(fa):
+    q = torch.zeros(1, 4, 4, 128, dtype=torch.float16)
+    w = torch.zeros(512, 256, dtype=torch.float16)
+    out = torch.zeros(1, 4, 256, dtype=torch.float16)
+    ws = torch.zeros(64, dtype=torch.uint8)
+    P = lambda t: t.data_ptr()
+    L = fa.lib.fa_forward_proj
+    def call(qp=P(q), wp=P(w), op=P(q), outp=P(out), wsp=P(ws), wsn=64, **kw):
+        a = dict(B=1, Hq=4, Hkv=2, Sq=4, Skv=4, d=128, dm=256, causal=1, scale=0.1, dt=fa.FA_DTYPE_FP16, fused=1)
+        a.update(kw)
+        return L(qp, P(q), P(q), wp, op, None, outp, a["B"], a["Hq"], a["Hkv"], a["Sq"], a["Skv"], a["d"], a["dm"],
+                 a["causal"], a["scale"], a["dt"], a["fused"], wsp, wsn, None)
+    assert fa.lib.fa_forward_proj_workspace_bytes(1, 4) == 4 and fa.lib.fa_forward_proj_workspace_bytes(3, 300) == 36
+    assert fa.lib.fa_forward_proj_workspace_bytes(0, 4) == 0
+    assert call(B=0) == fa.FA_OK and call(Sq=0) == fa.FA_OK
+    assert call(Hq=3) == fa.FA_ERR_SHAPE and call(dm=0) == fa.FA_ERR_SHAPE
+    assert call(dm=200) == fa.FA_ERR_UNSUPPORTED and call(d=64) == fa.FA_ERR_UNSUPPORTED
+    assert call(dt=fa.FA_DTYPE_FP32) == fa.FA_ERR_UNSUPPORTED and call(Sq=5) == fa.FA_ERR_UNSUPPORTED
+    assert call(scale=float("nan")) == fa.FA_ERR_UNSUPPORTED
+    assert call(qp=None) == fa.FA_ERR_NULL and call(wp=None) == fa.FA_ERR_NULL and call(outp=None) == fa.FA_ERR_NULL
+    assert call(outp=P(out) + 16) == fa.FA_ERR_ALIGN and call(wp=P(w) + 2) == fa.FA_ERR_ALIGN
+    assert call(wsp=None) == fa.FA_ERR_WORKSPACE and call(wsn=2) == fa.FA_ERR_WORKSPACE
+    assert call(wsp=P(ws) + 1) == fa.FA_ERR_ALIGN
