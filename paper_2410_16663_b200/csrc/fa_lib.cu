@@ -202,6 +202,7 @@ fa::FwdParams dense_fwd_params(const fa_params& p) {
     fp.seqlens_k = nullptr;
     fp.table_stride = 0;
     fp.page_size = 1;
+    fp.by_tiles_per_page.set(1);
     fp.d = p.d;
     fp.o_align32 = ((reinterpret_cast<uintptr_t>(p.o) & 31u) == 0 && (p.o_stride[0] & 15) == 0 &&
                     (p.o_stride[1] & 15) == 0 && (p.o_stride[2] & 15) == 0) ? 1 : 0;
@@ -448,6 +449,7 @@ int fa_forward_fp8(const void* q, const void* k, const void* v, void* o, float* 
     fp.seqlens_k = nullptr;
     fp.table_stride = 0;
     fp.page_size = 1;
+    fp.by_tiles_per_page.set(1);
     fp.d = 128;
     if (Skv == 0) {
         const long long rows = (long long)B * Sq * Hq;
@@ -612,6 +614,7 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     fp.seqlens_k = block_table ? cu_seqlens_k : nullptr;   // per-sequence key counts in the paged form
     fp.table_stride = table_stride;
     fp.page_size = block_table ? page_size : 1;
+    fp.by_tiles_per_page.set(block_table ? page_size / fa::kTile : 1);
 
     if (total_k == 0 || max_seqlen_k == 0) {
         // no keys anywhere: O = 0, LSE = -inf over the packed rows, seen as one sequence

@@ -354,7 +354,7 @@ __device__ __forceinline__ int pp_page_of(const FwdParams& p, int b, int j, int 
         int page;
         asm volatile("ld.global.nc.s32 %0, [%1];"
                      : "=r"(page)
-                     : "l"(p.block_table + (long long)b * p.table_stride + (j * kTile) / p.page_size));
+                     : "l"(p.block_table + (long long)b * p.table_stride + p.by_tiles_per_page.div(j)));
         return page;
     }
     return 0;
@@ -363,7 +363,7 @@ template <bool kVarlen>
 __device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int page, int j, int& row, int& slab) {
     if (kVarlen && p.block_table != nullptr) {
         slab = page;
-        row = (j * kTile) % p.page_size;
+        row = (j - p.by_tiles_per_page.div(j) * (int)p.by_tiles_per_page.d) * kTile;
     }
 }
 

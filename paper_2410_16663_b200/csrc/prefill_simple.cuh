@@ -68,6 +68,7 @@ struct FwdParams {
     const int* block_table;
     const int* seqlens_k;
     int table_stride, page_size;
+    FastDiv by_tiles_per_page;  // page_size / 128: kv tile j lies in table entry j / that, at tile j % that of the page
     int d;  // head dimension: 128, or 64 (its own kernel)
     float out_scale;  // factor on O (FP8 operands: the factor of V; 1 otherwise)
 };
