@@ -201,7 +201,8 @@ size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d);
  * v_pages [num_pages, page_size, Hkv, d]; page_size a positive multiple of 128; max_seqlen_k an
  * upper bound of seqlens_k, at most max_pages * page_size.  The causal mask is aligned
  * bottom-right per sequence (the queries are the sequence's LAST rows).  Only the table entries
- * that cover keys [0, seqlens_k[b]) are read (none for a sequence without keys).  Rows of a page
+ * that cover keys [0, seqlens_k[b]) are used; the first entry of every sequence's row is always
+ * read (it exists: table_stride >= 1) and ignored when the sequence has no keys.  Rows of a page
  * past the end of its sequence, and unused pages, may hold anything (NaN too).
  * Errors: as fa_forward_varlen; FA_ERR_SHAPE also for a page_size that is not a multiple of 128,
  * table_stride < max_pages or max_seqlen_k > max_pages * page_size.

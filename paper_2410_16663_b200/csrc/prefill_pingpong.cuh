@@ -94,6 +94,7 @@ struct PpItem {
     // packed variable-length batches only: first row of the sequence in q/o and in k/v, and
     // the sequence's own lengths
     int q_base, k_base, Sq, Skv;
+    int page0;   // paged K/V: the sequence's first table entry (-1 for a sequence without keys)
 };
 
 // Work item `idx`.  The query tiles of a head are taken in classes of C = 2^cls_log2 consecutive
@@ -133,7 +134,12 @@ __device__ __forceinline__ PpItem pp_decode_item(const FwdParams& p, int bh, int
         it.Sq = p.cu_q[it.b + 1] - it.q_base;
         if (p.block_table) {   // paged K/V: the keys are reached through the table
             it.k_base = 0;
+            // the first table entry is fetched together with the lengths, so that a loader does
+            // not start an item with two dependent global loads (the entry exists for every
+            // sequence; its value is ignored when the sequence has no keys)
+            const int first_page = __ldg(p.block_table + (long long)it.b * p.table_stride);
             it.Skv = p.seqlens_k[it.b];
+            it.page0 = it.Skv > 0 ? first_page : -1;
         } else {
             it.k_base = p.cu_k[it.b];
             it.Skv = p.cu_k[it.b + 1] - it.k_base;
@@ -395,7 +401,7 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), PpOperands<kF8>::kQBytes);
         pp_load_tile<kF8>(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
                        kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
-        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n, it.Skv);
+        int page = (kVarlen && p.block_table != nullptr) ? it.page0 : 0;
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
@@ -419,7 +425,7 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
     while (items.next(p, total_items)) {
         const int ord = items.ord;
         const PpItem& it = items.it;
-        int page = pp_page_of<kVarlen>(p, it.b, 0, it.n, it.Skv);
+        int page = (kVarlen && p.block_table != nullptr) ? it.page0 : 0;
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
