@@ -366,8 +366,14 @@ def run_prefill_fp8(fa, dev, peaks, small=False):
         q8, k8, v8 = synth.fp8_operands(q, k, v, 0.125, 0.25, 0.0625)
         o = torch.empty_like(q)
         lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
-        ms16 = _time_launches(fa, lambda: fa.fa_forward(q, k, v, o, lse, True, c16.scale), 20, 20)
-        ms8 = _time_launches(fa, lambda: fa.fa_forward_fp8(q8, k8, v8, o, lse, True, c16.scale, 0.125, 0.25, 0.0625), 20, 20)
+        # alternately, twice each, and the faster of the two: the launches are long enough for the
+        # board's power state to move between them
+        run16 = lambda: fa.fa_forward(q, k, v, o, lse, True, c16.scale)
+        run8 = lambda: fa.fa_forward_fp8(q8, k8, v8, o, lse, True, c16.scale, 0.125, 0.25, 0.0625)
+        ms16 = _time_launches(fa, run16, 20, 20)
+        ms8 = _time_launches(fa, run8, 20, 20)
+        ms16 = min(ms16, _time_launches(fa, run16, 5, 20))
+        ms8 = min(ms8, _time_launches(fa, run8, 5, 20))
         tf8 = c16.flops() / (ms8 * 1e-3) / 1e12
         res["cases"][cfg.name] = {"ms_fp8": round(ms8, 4), "tflops_fp8": round(tf8, 1), "ms_fp16": round(ms16, 4),
                                   "tflops_fp16": round(c16.flops() / (ms16 * 1e-3) / 1e12, 1),
