@@ -433,7 +433,7 @@ def run_d64(fa, dev, peaks, small=False, iters=10):
     tf = cfg.flops() / (ms * 1e-3) / 1e12
     nbytes = 4.0 * q.numel() * 2 + lse.numel() * 4
     gbs = nbytes / (ms * 1e-3) / 1e9
-    return {"workload": f"{cfg.name}: non-causal B={cfg.B} H={cfg.Hq} S={cfg.Sq} d=64 fp16", "kernel": "fa_fwd_d64_short_kernel",
+    return {"workload": f"{cfg.name}: non-causal B={cfg.B} H={cfg.Hq} S={cfg.Sq} d=64 fp16", "kernel": "fa_fwd_d64_stream_kernel",
             "ms": round(ms, 4), "tflops": round(tf, 1), "gbs": round(gbs, 1), "algorithmic_bytes": nbytes,
             "bound": "hbm", "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
             "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}

@@ -15,6 +15,7 @@
 #include "prefill_pingpong.cuh"
 #include "proj_gemm.cuh"
 #include "prefill_d64.cuh"
+#include "prefill_d64_stream.cuh"
 #include "prefill_d256.cuh"
 #include "decode_fp8.cuh"
 #include "prefill_pipelined.cuh"
@@ -258,15 +259,9 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     if (rc) return rc;
 
     if (p.d == 64 && p.Skv > 128 && p.Skv <= 256) {
-        // short sequences: all keys are one 256-wide tile, one CTA per (batch, head, two query tiles)
-        auto kern = bf16 ? fa::fa_fwd_d64_short_kernel<__nv_bfloat16> : fa::fa_fwd_d64_short_kernel<__half>;
-        int sm_count = 0;
-        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), fa::kD64ShortSmem, &sm_count))
-            return cuda_fail(static_cast<cudaError_t>(ce));
-        dim3 grid((fp.n_qtiles + 1) / 2, fp.Hq, fp.B);
-        kern<<<grid, fa::kD64ShortThreads, fa::kD64ShortSmem, st>>>(tq, tk, tv, fp);
-        cudaError_t e = cudaGetLastError();
-        return e == cudaSuccess ? FA_OK : cuda_fail(e);
+        // short sequences: all keys are one tile; a persistent pipeline over (batch, head, two query tiles)
+        return bf16 ? fa::launch_d64_stream<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
+                    : fa::launch_d64_stream<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
     }
     if (p.d == 64) {  // one CTA per (batch, head, query tile), four CTAs per SM
         auto kern = bf16 ? fa::fa_fwd_d64_slim_kernel<__nv_bfloat16> : fa::fa_fwd_d64_slim_kernel<__half>;

@@ -385,13 +385,26 @@ def test_d64_shape_grid(fa, sq, skv, causal):
 
 
 def test_d64_short_sequence_kernel(fa):
-    # 128 < Skv <= 256: all keys as one 256-wide tile.  More CTAs than fit at once, with one or
-    # two query tiles each, many query tiles over few keys, causal with fewer queries than keys
+    # 128 < Skv <= 256: all keys as one tile, a persistent pipeline over (batch, head, two query
+    # tiles).  More items than CTAs, with one or two query tiles each, many query tiles over few
+    # keys, causal with fewer queries than keys
     full_case_d64(fa, 30, 12, 12, 197, 197, False, "fp16", seed=81)
     full_case_d64(fa, 40, 6, 2, 100, 130, False, "bf16", seed=82)
     full_case_d64(fa, 3, 4, 4, 700, 256, False, "fp16", seed=83)
     full_case_d64(fa, 5, 8, 8, 150, 255, True, "fp16", seed=84)
     full_case_d64(fa, 2, 2, 1, 256, 256, True, "bf16", seed=85)
+    # an odd number of query tiles: the last item of a head has one tile, and the tiles change pairs
+    full_case_d64(fa, 7, 9, 3, 300, 200, False, "fp16", seed=86)
+    full_case_d64(fa, 50, 4, 4, 190, 197, True, "fp16", seed=87)
+    full_case_d64(fa, 9, 4, 4, 640, 197, False, "fp16", seed=88)
+
+
+@pytest.mark.parametrize("skv", [129, 144, 145, 160, 176, 193, 208, 209, 224, 240, 241])
+def test_d64_short_sequence_every_split_of_the_keys(fa, skv):
+    # the keys go to the two halves of a row in chunks of 16: every count of chunks from 9 to 16,
+    # with and without a ragged last chunk; enough items for every CTA to take several
+    full_case_d64(fa, 13, 12, 4, 197, skv, False, "fp16", seed=900 + skv)
+    full_case_d64(fa, 2, 3, 3, skv, skv, True, "bf16", seed=700 + skv)
 
 
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
