@@ -480,24 +480,48 @@ def run_varlen(fa, dev, peaks, small=False, iters=10):
     o = torch.empty_like(q)
     lse = torch.empty(cfg.Hq, q.shape[0], dtype=torch.float32, device=dev)
     mq, mk = max(cfg.seqlens_q), max(cfg.seqlens_k)
+    # the same keys and values behind a block table (256-key pages in a seeded random order), for
+    # the packed-batch prefill over a paged cache: the two forms are timed in alternation, because
+    # the box's power state moves either one by more than they differ
+    page = 128 if small else 256
+    kp, vp, table = synth.paged_from_packed(k, v, cfg.seqlens_k, page, seed=cfg.seed + 5)
+    table = table.to(dev)
+    sk = torch.tensor(cfg.seqlens_k, dtype=torch.int32, device=dev)
+    o2 = torch.empty_like(q)
+    lse2 = torch.empty_like(lse)
+    packed = lambda: fa.fa_forward_varlen(q, k, v, o, lse, cu_q, cu_k, mq, mk, cfg.causal, cfg.scale)
+    paged = lambda: fa.fa_forward_varlen_paged(q, kp, vp, table, o2, lse2, cu_q, sk, mq, mk, cfg.causal, cfg.scale)
+    times = {"packed": [], "paged": []}
     for _ in range(3):
-        fa.fa_forward_varlen(q, k, v, o, lse, cu_q, cu_k, mq, mk, cfg.causal, cfg.scale)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(iters):
-        fa.fa_forward_varlen(q, k, v, o, lse, cu_q, cu_k, mq, mk, cfg.causal, cfg.scale)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / iters
+        for name, run in (("packed", packed), ("paged", paged)):
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                run()
+            e1.record()
+            torch.cuda.synchronize()
+            times[name].append(e0.elapsed_time(e1) / iters)
     rc, where, blk = fa.fa_device_status()
     if rc != 0:
         raise SystemExit(f"device status {rc} at {where} block {blk}")
+    same = bool(torch.equal(o, o2) and torch.equal(lse, lse2))
+    ms = sorted(times["packed"])[1]
+    ms_paged = sorted(times["paged"])[1]
     tf = cfg.flops() / (ms * 1e-3) / 1e12
     return {"workload": f"{len(cfg.seqlens_q)} causal requests, lengths {min(cfg.seqlens_q)}..{mq} "
                         f"(sum {int(q.shape[0])}), Hq=Hkv={cfg.Hq}, bf16, packed", "ms": round(ms, 4),
             "tflops": round(tf, 1), "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4),
-            "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4)}
+            "frac_measured_tensor": round(tf / peaks["bf16_tflops"], 4),
+            "ms_all": [round(x, 4) for x in times["packed"]],
+            "paged": {"workload": f"the same requests with K and V in {page}-key pages in random order "
+                                  "(fa_forward_varlen_paged)", "ms": round(ms_paged, 4),
+                      "tflops": round(cfg.flops() / (ms_paged * 1e-3) / 1e12, 1),
+                      "ms_all": [round(x, 4) for x in times["paged"]],
+                      "paged_over_packed": round(ms_paged / ms, 4), "bit_identical_to_packed": same},
+            "note": "medians of three alternating measurements of each form"}
 
 
 def run_decode_append(fa, d, dev, peaks, Sq=4, iters=5):

@@ -255,6 +255,38 @@ def paged_cache(k, v, seqlens, page_size: int, seed: int, spare_pages: int = 3, 
     return k_pages, v_pages, table
 
 
+def paged_from_packed(k, v, seqlens, page_size: int, seed: int, spare_pages: int = 3, poison: bool = True):
+    """The packed keys and values of ``varlen_inputs`` (``[total_k, Hkv, d]``, sequences back to back)
+    laid out in pages: returns ``(k_pages, v_pages, block_table)`` as ``paged_cache`` does, pages
+    handed out in a seeded random order, unused rows and pages holding NaN bit patterns when
+    ``poison`` is set.  Layout only: no arithmetic."""
+    need = [(int(n) + page_size - 1) // page_size for n in seqlens]
+    num_pages = sum(need) + spare_pages
+    order = torch.randperm(num_pages, generator=_gen(seed, "cpu")).tolist()
+    bits = FP16_NAN_BITS if k.dtype == torch.float16 else BF16_NAN_BITS
+    k_pages = torch.empty(num_pages, page_size, k.shape[1], k.shape[2], dtype=k.dtype, device=k.device)
+    v_pages = torch.empty_like(k_pages)
+    if poison:
+        k_pages.view(torch.int16).fill_(bits)
+        v_pages.view(torch.int16).fill_(bits)
+    else:
+        k_pages.zero_()
+        v_pages.zero_()
+    table = torch.full((len(need), max(1, max(need))), -1, dtype=torch.int32)
+    nxt, base = 0, 0
+    for b, n in enumerate(int(x) for x in seqlens):
+        for pg in range(need[b]):
+            page = order[nxt]
+            nxt += 1
+            table[b, pg] = page
+            lo = pg * page_size
+            rows = min(page_size, n - lo)
+            k_pages[page, :rows] = k[base + lo:base + lo + rows]
+            v_pages[page, :rows] = v[base + lo:base + lo + rows]
+        base += n
+    return k_pages, v_pages, table
+
+
 def sample_rows(cfg: PrefillConfig, n_random: int, seed: int, pairs=None, tile: int = 128):
     """Rows (b, h, i) for row-sampled checks: the first four and the last row, both sides of
     tile boundaries near the start, middle and end, and uniformly random rows, over a few
