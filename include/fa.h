@@ -273,12 +273,27 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
                   const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
                   float k_scale, float v_scale, void* workspace, size_t workspace_bytes, void* stream);
 
+/* fa_decode_fp8 with q and o in bf16 (the models of the evaluation section run in either 16-bit
+ * type; the 8-bit cache is the same).  The products still run in fp16, the type the cache bytes
+ * widen to exactly: q is converted on load, which is exact for magnitudes in fp16's normal range
+ * (6.1e-5 to 65504; larger ones become infinities), the probabilities are rounded to fp16, and o
+ * is rounded to bf16 when it is stored.  Everything else as for fa_decode_fp8. */
+int fa_decode_fp8_bf16(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                       const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,
+                       float k_scale, float v_scale, void* workspace, size_t workspace_bytes, void* stream);
+
 /* fa_decode_fp8 over a paged cache: k_pages, v_pages [num_pages, page_size, Hkv, d] of e4m3 bytes;
  * block_table, page_size, max_pages, table_stride as for fa_decode_paged, scales as for fa_decode_fp8. */
 int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
                         void* o, float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages,
                         int page_size, int max_pages, int table_stride, int d, float scale, float k_scale,
                         float v_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/* fa_decode_fp8_paged with q and o in bf16 (see fa_decode_fp8_bf16). */
+int fa_decode_fp8_paged_bf16(const void* q, const void* k_pages, const void* v_pages, const int* block_table,
+                             void* o, float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages,
+                             int page_size, int max_pages, int table_stride, int d, float scale, float k_scale,
+                             float v_scale, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Decode over a paged cache: the same computation as fa_decode (Appendix C), with the cached
@@ -333,7 +348,8 @@ int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, v
 /*
  * Host-buffer form of fa_forward for callers whose tensors live in host memory (pinned memory
  * makes the copies asynchronous): copies q, k, v to the device staging area, runs the forward,
- * copies o and lse back.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16.
+ * copies o and lse back.  dtype is FA_DTYPE_FP16 or FA_DTYPE_BF16; d is 64, 128 or 256, as for
+ * fa_forward (FA_ERR_UNSUPPORTED otherwise, and fa_forward_host_staging_bytes then returns 0).
  * staging is a DEVICE buffer of at least fa_forward_host_staging_bytes(...) bytes, 1024-byte
  * aligned, owned by the caller.  The call is ordered after the work already on `stream`, and the
  * results are in o_host / lse_host once `stream` is idle.  Inside, the batch is cut into up to

@@ -70,6 +70,10 @@ lib.fa_decode_fp8.restype = _i
 lib.fa_decode_fp8.argtypes = [_p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
 lib.fa_decode_fp8_paged.restype = _i
 lib.fa_decode_fp8_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _f, _f, _f, _p, _sz, _p]
+lib.fa_decode_fp8_bf16.restype = _i
+lib.fa_decode_fp8_bf16.argtypes = lib.fa_decode_fp8.argtypes
+lib.fa_decode_fp8_paged_bf16.restype = _i
+lib.fa_decode_fp8_paged_bf16.argtypes = lib.fa_decode_fp8_paged.argtypes
 lib.fa_forward_varlen_paged.restype = _i
 lib.fa_forward_varlen_paged.argtypes = [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f,
                                         _i, _p]
@@ -93,7 +97,7 @@ lib.fa_last_cuda_error.restype = _i
 FA_DECODE_NOALLOC_BYTES = 4 << 20
 
 EXPORTS = ["fa_forward", "fa_forward_bf16", "fa_forward_ex", "fa_forward_fp8", "fa_forward_proj", "fa_forward_proj_workspace_bytes", "fa_decode", "fa_decode_workspace_bytes",
-           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
+           "fa_decode_noalloc", "fa_decode_paged", "fa_forward_varlen", "fa_decode_fp8", "fa_decode_fp8_paged", "fa_decode_fp8_bf16", "fa_decode_fp8_paged_bf16", "fa_decode_append", "fa_decode_append_workspace_bytes", "fa_decode_ex", "fa_forward_varlen_paged",
            "fa_forward_host", "fa_forward_host_staging_bytes", "fa_device_status", "fa_selftest_wait", "fa_strerror",
            "fa_version", "fa_last_cuda_error"]
 
@@ -285,6 +289,17 @@ def fa_decode_fp8(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, k_scale:
     return _check(rc, "fa_decode_fp8", raise_on_error)
 
 
+def fa_decode_fp8_bf16(q, k_cache, v_cache, o, lse, seqlens_k, scale: float, k_scale: float, v_scale: float, workspace,
+                       raise_on_error: bool = True) -> int:
+    """``fa_decode_fp8_bf16``: as ``fa_decode_fp8`` with q and o in bf16."""
+    B, _, Hq, d = q.shape
+    _, Smax, Hkv, _ = k_cache.shape
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_fp8_bf16(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse), _ptr(seqlens_k), B, Hq, Hkv,
+                                Smax, d, float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
+    return _check(rc, "fa_decode_fp8_bf16", raise_on_error)
+
+
 def fa_decode_fp8_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, k_scale: float,
                         v_scale: float, workspace, max_pages: int = None, raise_on_error: bool = True) -> int:
     """``fa_decode_fp8_paged``: as ``fa_decode_paged`` with pools of FP8 e4m3 bytes and one factor per tensor."""
@@ -298,6 +313,21 @@ def fa_decode_fp8_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, sca
                                  _ptr(seqlens_k), B, Hq, Hkv, num_pages, page_size, int(max_pages), int(stride), d,
                                  float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
     return _check(rc, "fa_decode_fp8_paged", raise_on_error)
+
+
+def fa_decode_fp8_paged_bf16(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, k_scale: float,
+                             v_scale: float, workspace, max_pages: int = None, raise_on_error: bool = True) -> int:
+    """``fa_decode_fp8_paged_bf16``: as ``fa_decode_fp8_paged`` with q and o in bf16."""
+    B, _, Hq, d = q.shape
+    num_pages, page_size, Hkv, _ = k_pages.shape
+    stride = block_table.stride(0) if block_table.dim() == 2 else block_table.numel() // max(1, B)
+    if max_pages is None:
+        max_pages = block_table.shape[1]
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.fa_decode_fp8_paged_bf16(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(o), _ptr(lse),
+                                      _ptr(seqlens_k), B, Hq, Hkv, num_pages, page_size, int(max_pages), int(stride), d,
+                                      float(scale), float(k_scale), float(v_scale), _ptr(workspace), wbytes, _stream())
+    return _check(rc, "fa_decode_fp8_paged_bf16", raise_on_error)
 
 
 def fa_decode_paged(q, k_pages, v_pages, block_table, o, lse, seqlens_k, scale: float, workspace,

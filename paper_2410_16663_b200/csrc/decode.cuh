@@ -38,6 +38,7 @@ struct DecodeParams {
     // the result itself and no merge kernel runs (nullptr otherwise)
     void* o_final;
     float* lse_final;
+    int bf16_io = 0;      // 8-bit cache kernel only: q and o are bf16 (fp16 otherwise)
 };
 
 

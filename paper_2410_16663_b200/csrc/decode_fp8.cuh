@@ -27,6 +27,14 @@ __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t in, uint32_t& lo, uin
         : "r"(in));
 }
 
+// A pair of bf16 values as a pair of fp16 values: exact for magnitudes in fp16's normal range
+// (bf16 carries 8 significant bits, fp16 11); larger ones become infinities, smaller ones lose bits.
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
+    const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+    const __half2 h = __floats2half2_rn(f.x, f.y);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
 // grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
 template <int NB>
 __global__ void __launch_bounds__(kDec8Threads, 2)
@@ -57,6 +65,7 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     if (k_begin >= k_end) {  // uniform for the CTA
         if (p.o_final != nullptr && tid < 128) {   // a sequence without keys, and nobody else writes its rows
             for (int r = 0; r < G; ++r) {
+                // (sixteen zero bits are 0.0 in fp16 and in bf16)
                 static_cast<__half*>(p.o_final)[((long long)b * p.Hq + h0 + r) * 128 + tid] = __half(0.f);
                 if (tid == 0 && p.lse_final) p.lse_final[(long long)b * p.Hq + h0 + r] = -INFINITY;
             }
@@ -149,6 +158,10 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     const int d0 = ks * 16 + 4 * t4;
                     qb[nbk][ks][0] = (head < G) ? *reinterpret_cast<const uint32_t*>(qp + head * 128 + d0) : 0u;
                     qb[nbk][ks][1] = (head < G) ? *reinterpret_cast<const uint32_t*>(qp + head * 128 + d0 + 2) : 0u;
+                    if (p.bf16_io) {   // the products run in fp16 (the widened cache is fp16): q goes there too
+                        qb[nbk][ks][0] = bf16x2_to_f16x2(qb[nbk][ks][0]);
+                        qb[nbk][ks][1] = bf16x2_to_f16x2(qb[nbk][ks][1]);
+                    }
                 }
             }
         }
@@ -354,7 +367,8 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 const float lse = (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f;
                 if (p.o_final != nullptr) {   // the only chunk: this is the result
                     const long long row = (long long)b * p.Hq + h0 + r;
-                    static_cast<__half*>(p.o_final)[row * 128 + col] = __half(out);
+                    if (p.bf16_io) static_cast<__nv_bfloat16*>(p.o_final)[row * 128 + col] = __nv_bfloat16(out);
+                    else static_cast<__half*>(p.o_final)[row * 128 + col] = __half(out);
                     if (col == 0 && p.lse_final) p.lse_final[row] = lse;
                 } else {
                     const long long slot = ((long long)b * p.Hq + h0 + r) * p.n_chunks + c;

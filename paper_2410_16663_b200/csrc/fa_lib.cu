@@ -775,7 +775,7 @@ int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, 
 static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
                            const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale,
                            float v_scale, void* workspace, size_t workspace_bytes, void* stream, const int* block_table,
-                           int num_pages, int page_size, int table_stride) {
+                           int num_pages, int page_size, int table_stride, bool bf16 = false) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0) return FA_ERR_SHAPE;
     if (Hq % Hkv) return FA_ERR_SHAPE;
     if (d != 128) return FA_ERR_UNSUPPORTED;
@@ -807,6 +807,7 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     dp.table_stride = table_stride;
     dp.v_scale = v_scale;
     dp.Sq = 1;
+    dp.bf16_io = bf16 ? 1 : 0;
     // one chunk per sequence: the split kernel writes O and LSE itself and no merge is launched
     const bool direct = Skv_max > 0 && dp.n_chunks == 1;
     dp.o_final = direct ? o : nullptr;
@@ -834,7 +835,8 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
         if (rc) return rc;
     }
     if (direct) return FA_OK;
-    fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16><<<B * Hq, 128, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
+    else fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
@@ -871,7 +873,14 @@ int fa_decode_fp8(const void* q, const void* k_cache, const void* v_cache, void*
                            workspace, workspace_bytes, stream, nullptr, 0, 0, 0);
 }
 
-int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+int fa_decode_fp8_bf16(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                       const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale, float k_scale,
+                       float v_scale, void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_fp8_impl(q, k_cache, v_cache, o, lse, seqlens_k, B, Hq, Hkv, Skv_max, d, scale, k_scale, v_scale,
+                           workspace, workspace_bytes, stream, nullptr, 0, 0, 0, true);
+}
+
+static int decode_fp8_paged_checked(bool bf16, const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
                         float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
                         int max_pages, int table_stride, int d, float scale, float k_scale, float v_scale,
                         void* workspace, size_t workspace_bytes, void* stream) {
@@ -882,7 +891,25 @@ int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages,
     if (max_pages > 0 && num_pages == 0) return FA_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(block_table) & 3u) return FA_ERR_ALIGN;
     return decode_fp8_impl(q, k_pages, v_pages, o, lse, seqlens_k, B, Hq, Hkv, max_pages * page_size, d, scale, k_scale,
-                           v_scale, workspace, workspace_bytes, stream, block_table, num_pages, page_size, table_stride);
+                           v_scale, workspace, workspace_bytes, stream, block_table, num_pages, page_size, table_stride, bf16);
+}
+
+int fa_decode_fp8_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+                        float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
+                        int max_pages, int table_stride, int d, float scale, float k_scale, float v_scale,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_fp8_paged_checked(false, q, k_pages, v_pages, block_table, o, lse, seqlens_k, B, Hq, Hkv, num_pages,
+                                    page_size, max_pages, table_stride, d, scale, k_scale, v_scale, workspace,
+                                    workspace_bytes, stream);
+}
+
+int fa_decode_fp8_paged_bf16(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
+                             float* lse, const int* seqlens_k, int B, int Hq, int Hkv, int num_pages, int page_size,
+                             int max_pages, int table_stride, int d, float scale, float k_scale, float v_scale,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_fp8_paged_checked(true, q, k_pages, v_pages, block_table, o, lse, seqlens_k, B, Hq, Hkv, num_pages,
+                                    page_size, max_pages, table_stride, d, scale, k_scale, v_scale, workspace,
+                                    workspace_bytes, stream);
 }
 
 int fa_decode_paged(const void* q, const void* k_pages, const void* v_pages, const int* block_table, void* o,
@@ -938,10 +965,10 @@ int fa_decode_noalloc(const void* q, const void* k_cache, const void* v_cache, v
 }
 
 size_t fa_forward_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int d) {
-    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv < 0 || d != 128) return 0;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv < 0 || (d != 64 && d != 128 && d != 256)) return 0;
     auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
-    const size_t qo = up((size_t)B * Sq * Hq * 128 * 2);
-    const size_t kv = up((size_t)B * Skv * Hkv * 128 * 2);
+    const size_t qo = up((size_t)B * Sq * Hq * d * 2);
+    const size_t kv = up((size_t)B * Skv * Hkv * d * 2);
     const size_t l = up((size_t)B * Hq * Sq * 4);
     return 2 * qo + 2 * kv + l;
 }
@@ -950,7 +977,7 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
                     int B, int Hq, int Hkv, int Sq, int Skv, int d, int causal, float scale, int dtype,
                     void* staging, size_t staging_bytes, void* stream) {
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Sq < 0 || Skv < 0 || d <= 0) return FA_ERR_SHAPE;
-    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (d != 64 && d != 128 && d != 256) return FA_ERR_UNSUPPORTED;   // the head dimensions fa_forward takes
     if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (B == 0 || Sq == 0) return FA_OK;
     if (!q_host || !o_host || (Skv > 0 && (!k_host || !v_host))) return FA_ERR_NULL;
@@ -958,7 +985,7 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
     if (!staging || staging_bytes < need) return FA_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(staging) & 1023u) return FA_ERR_ALIGN;
     auto up = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
-    const size_t qo_b = (size_t)B * Sq * Hq * 128 * 2, kv_b = (size_t)B * Skv * Hkv * 128 * 2;
+    const size_t qo_b = (size_t)B * Sq * Hq * d * 2, kv_b = (size_t)B * Skv * Hkv * d * 2;
     char* base = static_cast<char*>(staging);
     char* dq = base;
     char* dk = dq + up(qo_b);
@@ -979,7 +1006,7 @@ int fa_forward_host(const void* q_host, const void* k_host, const void* v_host, 
     if ((e = cudaEventRecord(hp->start, st)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess) return cuda_fail(e);
-    const size_t q1 = (size_t)Sq * Hq * 128 * 2, kv1 = (size_t)Skv * Hkv * 128 * 2, l1 = (size_t)Hq * Sq * 4;
+    const size_t q1 = (size_t)Sq * Hq * d * 2, kv1 = (size_t)Skv * Hkv * d * 2, l1 = (size_t)Hq * Sq * 4;
     for (int c = 0; c < parts; ++c) {
         const int b0 = (int)((long long)B * c / parts), b1 = (int)((long long)B * (c + 1) / parts);
         const size_t nb = (size_t)(b1 - b0);

@@ -182,17 +182,25 @@ def test_fp8_decode_validation(fa):
     ws = torch.zeros(1 << 16, dtype=torch.uint8)
     P = lambda t: t.data_ptr()
     need = fa.fa_decode_workspace_bytes(2, 8, 2, 256, 128)
-    call = lambda **kw: L.fa_decode_fp8(P(q), P(kc), P(kc), P(o), None, kw.get("sl", P(sl)), kw.get("B", 2), 8,
-                                        kw.get("Hkv", 2), 256, kw.get("d", 128), 0.1, kw.get("ks", 1.0), kw.get("vs", 1.0),
-                                        P(ws), kw.get("wbytes", need), None)
-    assert call(Hkv=3) == fa.FA_ERR_SHAPE
-    assert call(d=64) == fa.FA_ERR_UNSUPPORTED
-    assert call(ks=0.0) == fa.FA_ERR_UNSUPPORTED
-    assert call(vs=float("inf")) == fa.FA_ERR_UNSUPPORTED
-    assert call(ks=float("nan")) == fa.FA_ERR_UNSUPPORTED
-    assert call(sl=None) == fa.FA_ERR_NULL
-    assert call(wbytes=need - 1) == fa.FA_ERR_WORKSPACE
-    assert call(B=0) == fa.FA_OK
+    for entry in (L.fa_decode_fp8, L.fa_decode_fp8_bf16):   # the bf16 form shares every check
+        call = lambda **kw: entry(P(q), P(kc), P(kc), P(o), None, kw.get("sl", P(sl)), kw.get("B", 2), 8,
+                                  kw.get("Hkv", 2), 256, kw.get("d", 128), 0.1, kw.get("ks", 1.0), kw.get("vs", 1.0),
+                                  P(ws), kw.get("wbytes", need), None)
+        assert call(Hkv=3) == fa.FA_ERR_SHAPE
+        assert call(d=64) == fa.FA_ERR_UNSUPPORTED
+        assert call(ks=0.0) == fa.FA_ERR_UNSUPPORTED
+        assert call(vs=float("inf")) == fa.FA_ERR_UNSUPPORTED
+        assert call(ks=float("nan")) == fa.FA_ERR_UNSUPPORTED
+        assert call(sl=None) == fa.FA_ERR_NULL
+        assert call(wbytes=need - 1) == fa.FA_ERR_WORKSPACE
+        assert call(B=0) == fa.FA_OK
+    table = torch.zeros(2, 1, dtype=torch.int32)
+    for entry in (L.fa_decode_fp8_paged, L.fa_decode_fp8_paged_bf16):
+        paged = lambda **kw: entry(P(q), P(kc), P(kc), kw.get("table", P(table)), P(o), None, P(sl), 2, 8, 2, 2,
+                                   kw.get("page_size", 256), 1, kw.get("stride", 1), 128, 0.1, 1.0, 1.0, P(ws), need, None)
+        assert paged(page_size=48) == fa.FA_ERR_SHAPE
+        assert paged(stride=0) == fa.FA_ERR_SHAPE
+        assert paged(table=None) == fa.FA_ERR_NULL
 
 
 def test_varlen_paged_validation(fa):
@@ -246,6 +254,13 @@ def test_host_entry_validation(fa):
     assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_WORKSPACE
     assert L.fa_forward_host(None, P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_NULL
     assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 128, 1, 0.1, 5, None, 0, None) == fa.FA_ERR_UNSUPPORTED
+    # head dimensions: the ones fa_forward takes, with a staging area that follows d
+    up = lambda x: (x + 1023) // 1024 * 1024
+    for d in (64, 128, 256):
+        assert fa.fa_forward_host_staging_bytes(2, 4, 2, 5, 7, d) == 2 * up(2 * 5 * 4 * d * 2) + 2 * up(2 * 7 * 2 * d * 2) + up(2 * 4 * 5 * 4)
+    assert fa.fa_forward_host_staging_bytes(1, 4, 4, 4, 4, 96) == 0
+    assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 96, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_UNSUPPORTED
+    assert L.fa_forward_host(P(q), P(q), P(q), P(q), None, 1, 4, 4, 4, 4, 64, 1, 0.1, 0, None, 0, None) == fa.FA_ERR_WORKSPACE
 
 
 def test_binding_fails_loudly_without_the_library(tmp_path, monkeypatch):

@@ -1042,6 +1042,56 @@ def test_c5_decode_fp8_full_size_sampled(fa, cfg):
                                    what=f"{cfg.name} fp8 b{b} h{h} n{n}")
 
 
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 2), (17, 1), (40, 2)])
+def test_decode_fp8_bf16_queries(fa, hq, hkv):
+    # the same 8-bit cache with q and o in bf16: q widens to fp16 exactly (N(0,1) values), the
+    # probabilities are fp16 as in the fp16 form, so only the stored bf16 output adds a rounding
+    # (2^-8 |O|, allowed with its exact bound); contiguous and paged forms agree bit for bit;
+    # a sequence without keys and ragged lengths around the tile size are included
+    cfg = synth.DecodeConfig("t", 6, hq, hkv, 2304, 1, 2304, seed=960 + hq)
+    q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    q = q.to(torch.bfloat16)
+    sl[0], sl[1], sl[2], sl[3] = 2304, 0, 1, 257
+    k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+    B, _, Hq, d = q.shape
+    o, chk_o = guard_alloc((B, 1, Hq, d), torch.bfloat16, DEV)
+    lse, chk_l = guard_alloc((B, Hq), torch.float32, DEV)
+    ws, chk_w = guard_alloc((max(fa.fa_decode_workspace_bytes(B, Hq, cfg.Hkv, cfg.Smax, d) // 4, 4),), torch.float32, DEV)
+    fa.fa_decode_fp8_bf16(q.to(DEV), k8.to(DEV), v8.to(DEV), o, lse, sl.to(DEV), cfg.scale, 0.25, 0.125, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, 0.25, 0.125)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, stored_bf16=True, what=f"fp8 decode, bf16 q/o, {hq}/{hkv}")
+    page = 256
+    kp, vp, table = synth.paged_cache(k8, v8, sl, page, seed=11, spare_pages=2, poison=False)
+    o2 = torch.full((B, 1, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse2 = torch.full((B, Hq), float("nan"), device=DEV)
+    ws2 = torch.empty(fa.fa_decode_workspace_bytes(B, Hq, cfg.Hkv, table.shape[1] * page, d), dtype=torch.uint8, device=DEV)
+    fa.fa_decode_fp8_paged_bf16(q.to(DEV), kp.to(DEV), vp.to(DEV), table.to(DEV), o2, lse2, sl.to(DEV), cfg.scale, 0.25, 0.125, ws2)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)
+
+
+def test_decode_fp8_bf16_single_chunk_writes_the_result_itself(fa):
+    # short caches: one chunk per sequence, the split kernel stores the bf16 result without a merge launch
+    cfg = synth.DecodeConfig("t", 5, 8, 2, 640, 1, 640, seed=977)
+    q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    q = q.to(torch.bfloat16)
+    sl[0], sl[1] = 640, 0
+    k8, v8 = synth.fp8_cache(k, v, sl, 0.25, 0.125, poison=True)
+    B, _, Hq, d = q.shape
+    o = torch.full((B, 1, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, Hq), float("nan"), device=DEV)
+    ws = torch.empty(max(16, fa.fa_decode_workspace_bytes(B, Hq, cfg.Hkv, cfg.Smax, d)), dtype=torch.uint8, device=DEV)
+    fa.fa_decode_fp8_bf16(q.to(DEV), k8.to(DEV), v8.to(DEV), o, lse, sl.to(DEV), cfg.scale, 0.25, 0.125, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    o_ref, l_ref = oracle.decode_fp8(q, k8, v8, sl, cfg.scale, 0.25, 0.125)
+    assert_close_to_oracle(o[:, 0], lse, o_ref, l_ref, stored_bf16=True, what="fp8 decode, bf16 q/o, one chunk")
+
+
 @pytest.mark.parametrize("page", [256, 16, 64])
 def test_decode_fp8_paged_equals_contiguous_fp8_decode(fa, page):
     # the 8-bit cache in pages: bit for bit what fa_decode_fp8 gives on the same keys stored
@@ -1185,6 +1235,23 @@ def test_forward_host_entry(fa):
     check_status(fa)
     o_ref, l_ref = oracle.attention_full(q, k, v, c.causal, c.scale)
     assert_close_to_oracle(o, lse, o_ref, l_ref, what="host entry")
+
+
+@pytest.mark.parametrize("d", [64, 256])
+def test_forward_host_entry_other_head_dimensions(fa, d):
+    # the host entry takes the head dimensions fa_forward takes: the staging layout follows d
+    cfg = synth.PrefillConfig("t", 3, 4, 2, 150, 300, d=d, dtype="fp16", causal=True, seed=90 + d)
+    q, k, v = (t.pin_memory() for t in synth.prefill_inputs(cfg, "cpu"))
+    o = torch.full_like(q, float("nan")).pin_memory()
+    lse = torch.full((cfg.B, cfg.Hq, cfg.Sq), float("nan"), dtype=torch.float32).pin_memory()
+    n = fa.fa_forward_host_staging_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Sq, cfg.Skv, cfg.d)
+    st = torch.empty(n + 1024, dtype=torch.uint8, device=DEV)
+    off = (-st.data_ptr()) % 1024
+    fa.fa_forward_host(q, k, v, o, lse, True, cfg.scale, st[off:off + n])
+    torch.cuda.synchronize()
+    check_status(fa)
+    o_ref, l_ref = oracle.attention_full(q, k, v, True, cfg.scale)
+    assert_close_to_oracle(o, lse, o_ref, l_ref, what=f"host entry d={d}")
 
 
 @pytest.mark.parametrize("B", [2, 5])
