@@ -186,6 +186,9 @@ int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, floa
  *   outside [0, Skv_max] are clamped.
  *   workspace: at least fa_decode_workspace_bytes(...) bytes, 16-byte aligned, contents
  *   need no initialisation and are overwritten.
+ *   d is 128 or 64 (FA_ERR_UNSUPPORTED otherwise; fa_decode_workspace_bytes then returns 0); the
+ *   same holds for fa_decode_paged, fa_decode_append, fa_decode_ex and fa_decode_noalloc, which
+ *   run the same kernel.  The 8-bit cache forms (fa_decode_fp8...) take d = 128 only.
  */
 int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
               const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,

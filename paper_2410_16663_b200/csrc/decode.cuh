@@ -13,14 +13,23 @@
 namespace fa {
 
 constexpr int kDecTile = 128;                 // keys per shared-memory tile
-constexpr int kDecStages = 3;                 // ring depth (K and V tiles each 32 KiB)
-constexpr int kDecTileBytes = 32768;
-constexpr int kDecHalfBytes = 16384;
+constexpr int kDecStages = 3;                 // ring depth for d = 128 (K and V tiles each 32 KiB)
+constexpr int kDecTileBytes = 32768;          // a tile of d = 128
+constexpr int kDecHalfBytes = 16384;          // one 128-key x 64-element box
+// Head dimension D (128 or 64): a tile is 128 keys x D 16-bit elements, one or two swizzled
+// boxes, and the ring holds the same 96 KiB per operand either way (six 16 KiB slots for D = 64).
+template <int D>
+struct DecShape {
+    static_assert(D == 64 || D == 128, "head dimensions of the 16-bit decode kernel");
+    static constexpr int kTileBytes = kDecTile * D * 2;
+    static constexpr int kStages = kDecStages * 128 / D;
+    static constexpr int kSmem = 1024 + 2 * kStages * kTileBytes;
+};
 
 struct DecodeParams {
-    const void* q;        // [B,1,Hq,128] 16-bit
+    const void* q;        // [B,1,Hq,d] 16-bit
     const int* seqlens;   // [B] device
-    float* o_part;        // [B,Hq,NC,128]
+    float* o_part;        // [B,Hq,NC,d]
     float* lse_part;      // [B,Hq,NC]
     int B, Hq, Hkv, Smax;
     int chunk;            // keys per chunk (multiple of kDecTile)
@@ -86,15 +95,17 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // position len - Sq + t.  q is [B,Sq,Hq,128], the partials [B,Sq,Hq,NC,...].
 // grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
 // T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
-template <bool kMulti, typename T = __half>
+// D: the head dimension, 128 or 64.
+template <bool kMulti, typename T = __half, int D = 128>
 __global__ void __launch_bounds__(kDecMmaThreads, 1)
 fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr int kStages = DecShape<D>::kStages, kTileB = DecShape<D>::kTileBytes;
     const uint32_t sK = smem_base;
-    const uint32_t sV = smem_base + kDecStages * kDecTileBytes;
-    __shared__ __align__(8) uint64_t bars[3 * kDecStages];  // K full, V full, slot empty
+    const uint32_t sV = smem_base + kStages * kTileB;
+    __shared__ __align__(8) uint64_t bars[3 * kStages];  // K full, V full, slot empty
     __shared__ volatile uint32_t abort_flag;
 
     const int tid = threadIdx.x;
@@ -125,9 +136,9 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         return ((long long)b * p.Hq + hk * g_all + (kMulti ? R % g_all : R)) * Sq + row_token(r);
     };
     if (k_begin >= k_end) {  // uniform for the CTA
-        if (p.o_final != nullptr && tid < 128) {   // a sequence without keys, and nobody else writes its rows
+        if (p.o_final != nullptr && tid < D) {   // a sequence without keys, and nobody else writes its rows
             for (int r = 0; r < G; ++r) {
-                static_cast<T*>(p.o_final)[row_index(r) * 128 + tid] = T(0.f);
+                static_cast<T*>(p.o_final)[row_index(r) * D + tid] = T(0.f);
                 if (tid == 0 && p.lse_final) p.lse_final[lse_index(r)] = -INFINITY;
             }
         }
@@ -136,8 +147,8 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     const int n_tiles = (k_end - k_begin + kDecTile - 1) / kDecTile;
 
     if (tid == 0) {
-        for (int i = 0; i < 2 * kDecStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
-        for (int i = 0; i < kDecStages; ++i) mbar_init(smem_u32(&bars[2 * kDecStages + i]), 4);  // one arrival per consumer warp
+        for (int i = 0; i < 2 * kStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(&bars[2 * kStages + i]), 4);  // one arrival per consumer warp
         abort_flag = 0;
         fence_mbar_init();
     }
@@ -159,33 +170,33 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             };
             int pg_next = lookup(k_begin);
             for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kDecStages;
-                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                const int st = t % kStages;
+                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kStages + st]);
                 const int row0 = k_begin + t * kDecTile;
                 const int cur = pg_next;
                 if (t + 1 < n_tiles) pg_next = lookup(row0 + kDecTile);
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22);
+                if (lane == 0) ok = mbar_wait(smem_u32(&bars[2 * kStages + st]), ((t / kStages) & 1) ^ 1, &abort_flag, 22);
                 if (!__shfl_sync(0xffffffffu, ok, 0)) break;
                 const int live = min(n_sub, (k_end - row0 + ps - 1) / ps);   // pages of this tile that hold keys
                 if (lane == 0) {
-                    mbar_expect_tx(bk, (uint32_t)(live * ps) * 256u);
-                    mbar_expect_tx(bv, (uint32_t)(live * ps) * 256u);
+                    mbar_expect_tx(bk, (uint32_t)(live * ps) * (2u * D));
+                    mbar_expect_tx(bv, (uint32_t)(live * ps) * (2u * D));
                 }
                 __syncwarp();
                 if (lane < live) {
                     const uint32_t offs = (uint32_t)(lane * ps) * 128u;
-                    tma_load_4d(sK + st * kDecTileBytes + offs, &tm_k, bk, 0, hk, 0, cur);
-                    tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur);
-                    tma_load_4d(sV + st * kDecTileBytes + offs, &tm_v, bv, 0, hk, 0, cur);
-                    tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur);
+                    tma_load_4d(sK + st * kTileB + offs, &tm_k, bk, 0, hk, 0, cur);
+                    if (D == 128) tma_load_4d(sK + st * kTileB + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur);
+                    tma_load_4d(sV + st * kTileB + offs, &tm_v, bv, 0, hk, 0, cur);
+                    if (D == 128) tma_load_4d(sV + st * kTileB + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur);
                 }
             }
         } else if (lane == 0) {
             int page_next = table ? table[k_begin / p.page_size] : 0;
             for (int t = 0; t < n_tiles; ++t) {
-                const int st = t % kDecStages;
-                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kDecStages + st]);
+                const int st = t % kStages;
+                const uint32_t bk = smem_u32(&bars[st]), bv = smem_u32(&bars[kStages + st]);
                 int row0 = k_begin + t * kDecTile;  // first key of the tile within the sequence
                 int slab = b;                        // outermost coordinate: the sequence, or the page
                 if (table) {
@@ -193,26 +204,26 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     if (t + 1 < n_tiles) page_next = table[(row0 + kDecTile) / p.page_size];
                     row0 %= p.page_size;
                 }
-                if (!mbar_wait(smem_u32(&bars[2 * kDecStages + st]), ((t / kDecStages) & 1) ^ 1, &abort_flag, 22)) break;
-                mbar_expect_tx(bk, kDecTileBytes);
-                tma_load_4d(sK + st * kDecTileBytes, &tm_k, bk, 0, hk, row0, slab);
-                tma_load_4d(sK + st * kDecTileBytes + kDecHalfBytes, &tm_k, bk, 64, hk, row0, slab);
-                mbar_expect_tx(bv, kDecTileBytes);
-                tma_load_4d(sV + st * kDecTileBytes, &tm_v, bv, 0, hk, row0, slab);
-                tma_load_4d(sV + st * kDecTileBytes + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
+                if (!mbar_wait(smem_u32(&bars[2 * kStages + st]), ((t / kStages) & 1) ^ 1, &abort_flag, 22)) break;
+                mbar_expect_tx(bk, kTileB);
+                tma_load_4d(sK + st * kTileB, &tm_k, bk, 0, hk, row0, slab);
+                if (D == 128) tma_load_4d(sK + st * kTileB + kDecHalfBytes, &tm_k, bk, 64, hk, row0, slab);
+                mbar_expect_tx(bv, kTileB);
+                tma_load_4d(sV + st * kTileB, &tm_v, bv, 0, hk, row0, slab);
+                if (D == 128) tma_load_4d(sV + st * kTileB + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
             }
         }
         __syncwarp();
     } else {
         // ---------------------------------------------------------------- consumers
         const int g = lane >> 2, t4 = lane & 3;  // fragment row (query head g and g + 8) and column pair
-        // Q as A fragments for the eight k-steps of d = 128 (rows >= G are zero)
-        uint32_t qa[8][4];
+        // Q as A fragments for the D / 16 k-steps (rows >= G are zero)
+        uint32_t qa[D / 16][4];
         {
-            const __half* q_lo = static_cast<const __half*>(p.q) + row_index(g) * 128;
-            const __half* q_hi = static_cast<const __half*>(p.q) + row_index(g + 8) * 128;
+            const __half* q_lo = static_cast<const __half*>(p.q) + row_index(g) * D;
+            const __half* q_hi = static_cast<const __half*>(p.q) + row_index(g + 8) * D;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+            for (int ks = 0; ks < D / 16; ++ks) {
                 const int k0 = ks * 16 + 2 * t4;
                 qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_lo + k0) : 0u;
                 qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q_hi + k0) : 0u;
@@ -223,16 +234,16 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         // keys an earlier query token must not see: the last Sq - 1 - t of the sequence
         const int hide_lo = kMulti ? Sq - 1 - row_token(g) : 0;
         const int hide_hi = kMulti ? Sq - 1 - row_token(min(g + 8, G - 1)) : 0;
-        float o[16][4];
+        float o[D / 8][4];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
         float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;  // rows g and g + 8
         const int key_w = warp * 32;  // this warp's keys inside a tile
         bool ok = true;
 
         for (int t = 0; t < n_tiles; ++t) {
-            const int st = t % kDecStages;
-            const uint32_t parity = (t / kDecStages) & 1;
+            const int st = t % kStages;
+            const uint32_t parity = (t / kStages) & 1;
             const int valid = min(kDecTile, k_end - (k_begin + t * kDecTile)) - key_w;  // valid keys of this warp's 32
             ok = mbar_wait(smem_u32(&bars[st]), parity, &abort_flag, 20);
             ok = __all_sync(0xffffffffu, ok);
@@ -240,13 +251,13 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             float sc[4][4];
             if (valid > 0) {
                 // ---- S = Q K^T for this warp's four blocks of 8 keys
-                const uint32_t kt = sK + st * kDecTileBytes;
+                const uint32_t kt = sK + st * kTileB;
 #pragma unroll
                 for (int nb = 0; nb < 4; ++nb) {
                     sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
                     const int key = key_w + nb * 8 + (lane & 7);
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {  // 4 d-chunks of 8 per ldmatrix.x4 = two k-steps
+                    for (int c4 = 0; c4 < D / 32; ++c4) {  // 4 d-chunks of 8 per ldmatrix.x4 = two k-steps
                         const int chunk = c4 * 4 + (lane >> 3);
                         const uint32_t addr = kt + (chunk >> 3) * kDecHalfBytes + key * 128 + (((chunk & 7) ^ (key & 7)) << 4);
                         uint32_t b0, b1, b2, b3;
@@ -303,28 +314,28 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 l_lo = l_lo * a_lo + s_lo;  // per-thread partial of the row sum (the quad is summed at the end)
                 l_hi = l_hi * a_hi + s_hi;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < D / 8; ++i) {
                     o[i][0] *= a_lo;
                     o[i][1] *= a_lo;
                     o[i][2] *= a_hi;
                     o[i][3] *= a_hi;
                 }
             }
-            ok = mbar_wait(smem_u32(&bars[kDecStages + st]), parity, &abort_flag, 21);
+            ok = mbar_wait(smem_u32(&bars[kStages + st]), parity, &abort_flag, 21);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (valid > 0) {
-                const uint32_t vt = sV + st * kDecTileBytes;
+                const uint32_t vt = sV + st * kTileB;
                 if (valid < 32) {
                     // rows past the sequence may hold NaN bits: zero them (0 * NaN would poison O)
-                    for (int i = lane; i < (32 - valid) * 16; i += 32) {
-                        const int key = key_w + valid + (i >> 4), ch = i & 15;
+                    for (int i = lane; i < (32 - valid) * (D / 8); i += 32) {
+                        const int key = key_w + valid + i / (D / 8), ch = i % (D / 8);
                         const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
                         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                     }
                     __syncwarp();
                 }
-                // ---- O += P V: two k-steps of 16 keys, sixteen blocks of 8 output columns
+                // ---- O += P V: two k-steps of 16 keys, D / 8 blocks of 8 output columns
 #pragma unroll
                 for (int k2 = 0; k2 < 2; ++k2) {
                     uint32_t pa[4];
@@ -334,7 +345,7 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     pa[3] = pack2<T>(sc[2 * k2 + 1][2], sc[2 * k2 + 1][3]);
                     const int key = key_w + k2 * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
 #pragma unroll
-                    for (int n2 = 0; n2 < 8; ++n2) {  // two output blocks per ldmatrix.x4.trans
+                    for (int n2 = 0; n2 < D / 16; ++n2) {  // two output blocks per ldmatrix.x4.trans
                         const int ch = n2 * 2 + (lane >> 4);
                         const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
                         uint32_t b0, b1, b2, b3;
@@ -350,7 +361,7 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kDecStages + st]));
+            if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kStages + st]));
         }
 
         // ---- merge the four warps' states and write this chunk's partial result
@@ -360,15 +371,15 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][128]
-        float* ml = mo + 4 * 16 * 128;                                                       // [4][16][2]: m, l
+        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][D]
+        float* ml = mo + 4 * 16 * D;                                                         // [4][16][2]: m, l
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ok) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
+            for (int i = 0; i < D / 8; ++i) {
                 const int col = i * 8 + 2 * t4;
-                *reinterpret_cast<float2*>(&mo[(warp * 16 + g) * 128 + col]) = make_float2(o[i][0], o[i][1]);
-                *reinterpret_cast<float2*>(&mo[(warp * 16 + g + 8) * 128 + col]) = make_float2(o[i][2], o[i][3]);
+                *reinterpret_cast<float2*>(&mo[(warp * 16 + g) * D + col]) = make_float2(o[i][0], o[i][1]);
+                *reinterpret_cast<float2*>(&mo[(warp * 16 + g + 8) * D + col]) = make_float2(o[i][2], o[i][3]);
             }
             if (t4 == 0) {
                 ml[(warp * 16 + g) * 2] = m_lo;
@@ -378,7 +389,7 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
             }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (ok) {
+        if (ok && tid < D) {
             for (int r = 0; r < G; ++r) {  // thread `tid` owns output column `tid` of every row
                 float M = -INFINITY;
 #pragma unroll
@@ -389,17 +400,17 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                     const float mw = ml[(w * 16 + r) * 2];
                     const float sw = (mw == -INFINITY) ? 0.f : fast_exp2((mw - M) * p.scale_log2);
                     l += sw * ml[(w * 16 + r) * 2 + 1];
-                    acc += sw * mo[(w * 16 + r) * 128 + tid];
+                    acc += sw * mo[(w * 16 + r) * D + tid];
                 }
                 // (l == 0: a query token that sees none of this chunk's keys)
                 const float out = (l > 0.f) ? acc / l : 0.f;
                 const float lse = (l > 0.f) ? (M * p.scale_log2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
                 if (p.o_final != nullptr) {   // the only chunk: this is the result
-                    static_cast<T*>(p.o_final)[row_index(r) * 128 + tid] = T(out);
+                    static_cast<T*>(p.o_final)[row_index(r) * D + tid] = T(out);
                     if (tid == 0 && p.lse_final) p.lse_final[lse_index(r)] = lse;
                 } else {
                     const long long slot = row_index(r) * p.n_chunks + c;
-                    p.o_part[slot * 128 + tid] = out;
+                    p.o_part[slot * D + tid] = out;
                     if (tid == 0) p.lse_part[slot] = lse;
                 }
             }
@@ -409,8 +420,8 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
 // Merge of the per-chunk partials (rowmax/rowsum recurrence applied across chunks):
 //   M = max_c LSE_c, w_c = exp(LSE_c - M), O = sum_c w_c O_c / sum_c w_c, LSE = M + ln sum_c w_c.
-// grid: B * Sq * Hq blocks of 128 threads (row = (b, token, head)), thread t owns output dim t.
-template <typename T>
+// grid: B * Sq * Hq blocks of D threads (row = (b, token, head)), thread t owns output dim t.
+template <typename T, int D = 128>
 __global__ void __launch_bounds__(128)
 fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
     const int bh = blockIdx.x;
@@ -422,11 +433,11 @@ fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
     len = max(0, min(len, p.Smax));
     const int nc = (len + p.chunk - 1) / p.chunk;
     const float* lp = p.lse_part + (long long)bh * p.n_chunks;
-    const float* op = p.o_part + (long long)bh * p.n_chunks * 128;
+    const float* op = p.o_part + (long long)bh * p.n_chunks * D;
     float M = -INFINITY;
     for (int c = 0; c < nc; ++c) M = fmaxf(M, lp[c]);
     if (nc == 0 || M == -INFINITY) {   // no keys, or (several query rows) a token that sees none
-        o[(long long)bh * 128 + tid] = T(0.f);
+        o[(long long)bh * D + tid] = T(0.f);
         if (lse && tid == 0) lse[lse_at] = -INFINITY;
         return;
     }
@@ -434,9 +445,9 @@ fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
     for (int c = 0; c < nc; ++c) {
         const float w = __expf(lp[c] - M);
         wsum += w;
-        acc = fmaf(w, op[(long long)c * 128 + tid], acc);
+        acc = fmaf(w, op[(long long)c * D + tid], acc);
     }
-    o[(long long)bh * 128 + tid] = T(acc / wsum);
+    o[(long long)bh * D + tid] = T(acc / wsum);
     if (lse && tid == 0) lse[lse_at] = M + logf(wsum);
 }
 

@@ -662,10 +662,10 @@ int fa_forward_varlen_paged(const void* q, const void* k_pages, const void* v_pa
 }
 
 size_t fa_decode_workspace_bytes(int B, int Hq, int Hkv, int Skv_max, int d) {
-    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Skv_max <= 0 || d != 128) return 0;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Skv_max <= 0 || (d != 128 && d != 64)) return 0;
     const int chunk = decode_chunk(B, Hkv, Skv_max);
     const size_t nc = (size_t)((Skv_max + chunk - 1) / chunk);
-    return (size_t)B * Hq * nc * (128 + 1) * sizeof(float);
+    return (size_t)B * Hq * nc * ((size_t)d + 1) * sizeof(float);
 }
 
 size_t fa_decode_append_workspace_bytes(int B, int Sq, int Hq, int Hkv, int Skv_max, int d) {
@@ -683,7 +683,7 @@ int decode_check_args(const void* q, const void* k_cache, const void* v_cache, c
     if (B < 0 || Hq <= 0 || Hkv <= 0 || Skv_max < 0 || d <= 0 || Sq < 1) return FA_ERR_SHAPE;
     if (Sq > 64 || Sq > Skv_max) return FA_ERR_UNSUPPORTED;   // several query rows are the LAST rows of the cache
     if (Hq % Hkv) return FA_ERR_SHAPE;
-    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (d != 128 && d != 64) return FA_ERR_UNSUPPORTED;
     if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
     if (B > 65535 || Hq > 65535) return FA_ERR_UNSUPPORTED;
     if (B == 0) return FA_OK;
@@ -693,8 +693,34 @@ int decode_check_args(const void* q, const void* k_cache, const void* v_cache, c
     return FA_OK;
 }
 
-// Decode over a contiguous cache (block_table == nullptr; k_cache, v_cache [B,Skv_max,Hkv,128])
-// or over pages (k_cache, v_cache [num_pages,page_size,Hkv,128]; Skv_max = max_pages * page_size).
+// Launch of the split kernel and of the merge for one head dimension.
+template <int D>
+int decode_launch(const CUtensorMap& tk, const CUtensorMap& tv, const fa::DecodeParams& dp, void* o, float* lse, int g,
+                  bool bf16, bool direct, bool have_keys, cudaStream_t st) {
+    const int B = dp.B, Sq = dp.Sq, Hq = dp.Hq, Hkv = dp.Hkv;
+    if (have_keys) {
+        constexpr int smem = fa::DecShape<D>::kSmem;
+        int sm_count = 0;
+        auto kern = bf16 ? ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __nv_bfloat16, D>
+                                     : fa::fa_decode_split_mma_kernel<false, __nv_bfloat16, D>)
+                         : ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __half, D>
+                                     : fa::fa_decode_split_mma_kernel<false, __half, D>);
+        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
+            return cuda_fail(static_cast<cudaError_t>(ce));
+        dim3 grid(dp.n_chunks, Hkv * ((g * Sq + 15) / 16), B);   // 16 (token, head) rows per CTA
+        kern<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (direct) return FA_OK;
+    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16, D><<<B * Sq * Hq, D, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
+    else fa::fa_decode_combine_kernel<__half, D><<<B * Sq * Hq, D, 0, st>>>(dp, static_cast<__half*>(o), lse);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+}
+
+// Decode over a contiguous cache (block_table == nullptr; k_cache, v_cache [B,Skv_max,Hkv,d])
+// or over pages (k_cache, v_cache [num_pages,page_size,Hkv,d]; Skv_max = max_pages * page_size).
 int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, const int* seqlens_k,
                 int B, int Hq, int Hkv, int Skv_max, int d, float scale, void* workspace, size_t workspace_bytes,
                 void* stream, const int* block_table, int num_pages, int page_size, int table_stride, int Sq = 1,
@@ -717,7 +743,7 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max) : 256;
     dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
     dp.o_part = static_cast<float*>(workspace);
-    dp.lse_part = dp.o_part + (size_t)B * Sq * Hq * dp.n_chunks * 128;
+    dp.lse_part = dp.o_part + (size_t)B * Sq * Hq * dp.n_chunks * d;
     dp.scale_log2 = scale * 1.4426950408889634f;
     dp.block_table = block_table;
     dp.page_size = block_table ? page_size : 1;
@@ -729,36 +755,21 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.lse_final = direct ? lse : nullptr;
     const int g = Hq / Hkv;
 
+    CUtensorMap tk, tv;
     if (Skv_max > 0) {
         // the outermost dimension of the maps is the sequence, or the page
         const int slabs = block_table ? num_pages : B;
         const int slab_rows = block_table ? page_size : Skv_max;
-        CUtensorMap tk, tv;
         const int box_rows = (block_table && page_size < fa::kDecTile) ? page_size : fa::kDecTile;
-        rc = encode_map(&tk, k_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        box_rows, bf16);
+        rc = encode_map(&tk, k_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * d, (int64_t)Hkv * d, d,
+                        box_rows, bf16, d);
         if (rc) return rc;
-        rc = encode_map(&tv, v_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128,
-                        box_rows, bf16);
-        if (rc) return rc;
-        constexpr int smem = 1024 + 2 * fa::kDecStages * fa::kDecTileBytes;
-        int sm_count = 0;
-        auto kern = bf16 ? ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __nv_bfloat16>
-                                     : fa::fa_decode_split_mma_kernel<false, __nv_bfloat16>)
-                         : ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __half> : fa::fa_decode_split_mma_kernel<false, __half>);
-        if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
-            return cuda_fail(static_cast<cudaError_t>(ce));
-        dim3 grid(dp.n_chunks, Hkv * ((g * Sq + 15) / 16), B);   // 16 (token, head) rows per CTA
-        kern<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
-        cudaError_t e = cudaGetLastError();
-        rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
+        rc = encode_map(&tv, v_cache, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * d, (int64_t)Hkv * d, d,
+                        box_rows, bf16, d);
         if (rc) return rc;
     }
-    if (direct) return FA_OK;
-    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
-    else fa::fa_decode_combine_kernel<__half><<<B * Sq * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
-    cudaError_t e = cudaGetLastError();
-    return e == cudaSuccess ? FA_OK : cuda_fail(e);
+    return d == 64 ? decode_launch<64>(tk, tv, dp, o, lse, g, bf16, direct, Skv_max > 0, st)
+                   : decode_launch<128>(tk, tv, dp, o, lse, g, bf16, direct, Skv_max > 0, st);
 }
 }  // namespace
 

@@ -94,7 +94,8 @@ def test_decode_validation_and_workspace_size(fa):
     P = lambda t: t.data_ptr()
     need = fa.fa_decode_workspace_bytes(2, 8, 2, 256, 128)
     assert need == 2 * 8 * 1 * 129 * 4
-    assert fa.fa_decode_workspace_bytes(2, 8, 2, 256, 64) == 0
+    assert fa.fa_decode_workspace_bytes(2, 8, 2, 256, 64) == 2 * 8 * 1 * 65 * 4    # head dimension 64: its own partials
+    assert fa.fa_decode_workspace_bytes(2, 8, 2, 256, 256) == 0 and fa.fa_decode_workspace_bytes(2, 8, 2, 256, 96) == 0
     # large problems use 2048-key chunks
     assert fa.fa_decode_workspace_bytes(64, 32, 32, 32768, 128) == 64 * 32 * 16 * 129 * 4
     args = lambda **kw: None

@@ -950,6 +950,68 @@ def test_decode_with_a_single_chunk_per_sequence(fa, sq, dtype):
                                what=f"single-chunk decode B{B} sq{sq} {dtype}")
 
 
+# ------------------------------------------------------------------ decode with head dimension 64
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("form", ["plain", "append", "paged", "paged16", "one-chunk"])
+def test_decode_head_dimension_64(fa, form, dtype):
+    # The 16-bit decode kernel with d = 64 (tiles of one 64-column box, six ring slots): one query
+    # row and five (append), contiguous and paged caches (256-key and 16-key pages), many chunks and
+    # a single one; lengths: full, empty, one key, ragged around the tile size; NaN past every end.
+    sq = 5 if form == "append" else 1
+    smax = 640 if form == "one-chunk" else 2560
+    cfg = synth.DecodeConfig("t", 6, 8, 2, smax, 1, smax, d=64, dtype=dtype, seed=1400 + len(form))
+    _, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=False)
+    sl[0], sl[1], sl[2], sl[3] = smax, 0, max(1, sq), 129 + sq
+    for b in range(cfg.B):
+        k[b, int(sl[b]):] = float("nan")
+        v[b, int(sl[b]):] = float("nan")
+    gen = torch.Generator().manual_seed(cfg.seed + 1)
+    q = torch.randn(cfg.B, sq, cfg.Hq, 64, generator=gen).to(k.dtype)
+    kz, vz = k.nan_to_num(0.0), v.nan_to_num(0.0)
+    o_ref, l_ref = oracle.decode_append(q, kz, vz, sl, cfg.scale)
+    absv = oracle.decode_append(q, kz, vz.abs(), sl, cfg.scale)[0] if dtype == "bf16" else None
+    o, chk_o = guard_alloc((cfg.B, sq, cfg.Hq, 64), k.dtype, DEV)
+    lse, chk_l = guard_alloc((cfg.B, cfg.Hq, sq), torch.float32, DEV)
+    nbytes = fa.fa_decode_append_workspace_bytes(cfg.B, sq, cfg.Hq, cfg.Hkv, smax, 64)
+    assert nbytes > 0
+    ws, chk_w = guard_alloc((nbytes // 4,), torch.float32, DEV)
+    table = None
+    kd, vd = k, v
+    if form.startswith("paged"):
+        page = 16 if form == "paged16" else 256
+        kd, vd, table = synth.paged_cache(k, v, sl, page, seed=9, spare_pages=2, poison=True)
+        table = table.to(DEV)
+    fa.fa_decode_ex(q.to(DEV), kd.to(DEV), vd.to(DEV), o, lse, sl.to(DEV), cfg.scale, ws, block_table=table)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    assert_close_to_oracle(o, lse, o_ref, l_ref, stored_bf16=(dtype == "bf16"), p_absv=absv,
+                           what=f"decode d=64 {form} {dtype}")
+    assert float(o[1].float().abs().max()) == 0.0 and torch.isneginf(lse[1]).all()
+
+
+def test_decode_head_dimension_64_large_batch_sampled(fa):
+    # a batch that fills the GPU (2048-key chunks, 64 sequences of up to 16K keys, GQA): sampled rows
+    cfg = synth.DecodeConfig("t", 64, 32, 8, 16384, 1024, 16384, d=64, dtype="fp16", seed=1450)
+    q, k, v, sl = synth.decode_inputs(cfg, DEV, poison=True)
+    o, chk_o = guard_alloc((cfg.B, 1, cfg.Hq, 64), torch.float16, DEV)
+    lse, chk_l = guard_alloc((cfg.B, cfg.Hq), torch.float32, DEV)
+    ws, chk_w = guard_alloc((fa.fa_decode_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Smax, 64) // 4,), torch.float32, DEV)
+    fa.fa_decode(q, k, v, o, lse, sl.to(DEV), cfg.scale, ws)
+    torch.cuda.synchronize()
+    check_status(fa)
+    chk_o(); chk_l(); chk_w()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    g = cfg.Hq // cfg.Hkv
+    for b in (0, 17, cfg.B - 1, int(torch.argmax(sl)), int(torch.argmin(sl))):
+        n = int(sl[b])
+        for h in (0, g - 1, cfg.Hq - 1):
+            hk = h // g
+            o_ref, l_ref = oracle.decode(q[b:b + 1, :, h:h + 1].cpu(), k[b:b + 1, :n, hk:hk + 1].contiguous().cpu(),
+                                         v[b:b + 1, :n, hk:hk + 1].contiguous().cpu(), [n], cfg.scale)
+            assert_close_to_oracle(o[b, 0, h].view(1, 1, -1), lse[b, h].view(1, 1), o_ref, l_ref, what=f"decode d=64 b{b} h{h}")
+
+
 # ------------------------------------------------------------------ decode over an FP8 cache
 def run_decode_fp8(fa, q, k8, v8, seqlens_dev, scale, k_scale, v_scale):
     B, _, Hq, d = q.shape
