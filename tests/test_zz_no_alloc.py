@@ -49,7 +49,8 @@ def test_noalloc_checks_its_arguments_like_fa_decode_before_any_cuda_call(fa):
         dict(scale=float("inf")),
         dict(scale=float("nan")),
         dict(Hq=6, Hkv=4),
-        dict(d=64),
+        dict(d=96),                                # a head dimension other than 128 and 64
+        dict(d=256),
         dict(B=70000),
         dict(Skv_max=0),
     ]
