@@ -68,9 +68,10 @@ def test_noalloc_checks_its_arguments_like_fa_decode_before_any_cuda_call(fa):
 
 
 @pytest.mark.gpu
-def test_noalloc_matches_fa_decode_on_two_calls_in_a_row(fa):
+@pytest.mark.parametrize("d", [128, 64])
+def test_noalloc_matches_fa_decode_on_two_calls_in_a_row(fa, d):
     dev = "cuda"
-    cfg = synth.DecodeConfig("noalloc", 6, 8, 2, 5000, 1, 5000, seed=808)
+    cfg = synth.DecodeConfig("noalloc", 6, 8, 2, 5000, 1, 5000, d=d, seed=808)
     q, k, v, sl = synth.decode_inputs(cfg, dev, poison=False)  # the second call reads other lengths
     assert fa.fa_decode_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Smax, cfg.d) <= fa.FA_DECODE_NOALLOC_BYTES
     ws = torch.empty(fa.fa_decode_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.Smax, cfg.d), dtype=torch.uint8,
