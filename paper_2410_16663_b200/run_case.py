@@ -3,6 +3,7 @@
 Meant for profilers (ncu wraps this command) and quick timing:
   python -m paper_2410_16663_b200.run_case prefill --B 1 --H 32 --Hkv 32 --S 8192 --dtype bf16 --iters 3
   python -m paper_2410_16663_b200.run_case decode  --B 16 --H 32 --Hkv 8 --Smax 16384 --iters 3
+  python -m paper_2410_16663_b200.run_case decode  --B 16 --H 32 --Hkv 8 --Smax 16384 --d 64    (head dimension 64)
   python -m paper_2410_16663_b200.run_case prefill --B 1 --H 32 --S 8192 --fp8           (8-bit operands)
   python -m paper_2410_16663_b200.run_case proj    --B 4 --H 32 --S 2048 --fused 1       (attention + projection)
 """
@@ -26,7 +27,7 @@ def main():
     ap.add_argument("--S", type=int, default=8192)
     ap.add_argument("--Skv", type=int, default=0)
     ap.add_argument("--Smax", type=int, default=16384)
-    ap.add_argument("--d", type=int, default=128, choices=[64, 128, 256], help="head dimension (prefill only)")
+    ap.add_argument("--d", type=int, default=128, choices=[64, 128, 256], help="head dimension (prefill: 64, 128, 256; decode: 64, 128)")
     ap.add_argument("--dtype", default="fp16", choices=["fp16", "bf16"])
     ap.add_argument("--noncausal", action="store_true")
     ap.add_argument("--fp8", action="store_true", help="decode: the cache as FP8 e4m3 (factors 1/4 and 1/8); "
@@ -63,7 +64,9 @@ def main():
         run = lambda: fa.fa_forward_proj(q, k, v, w, o, lse, out, cfg.causal, cfg.scale, bool(a.fused), ws)
         work, unit = (cfg.flops() + 2.0 * cfg.B * cfg.Sq * K * K) / 1e12, "TFLOPS"
     else:
-        cfg = synth.DecodeConfig("case", a.B, a.H, hkv, a.Smax, max(1, a.Smax // 32), a.Smax, seed=8)
+        if a.d == 256 or (a.fp8 and a.d != 128):
+            raise SystemExit("decode takes d = 128 or 64 (the 8-bit cache form d = 128 only)")
+        cfg = synth.DecodeConfig("case", a.B, a.H, hkv, a.Smax, max(1, a.Smax // 32), a.Smax, d=a.d, seed=8)
         q, k, v, sl = synth.decode_inputs(cfg, dev, poison=True)
         o = torch.empty_like(q)
         lse = torch.empty(cfg.B, cfg.Hq, dtype=torch.float32, device=dev)
