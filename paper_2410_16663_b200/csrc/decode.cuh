@@ -13,7 +13,7 @@
 namespace fa {
 
 constexpr int kDecTile = 128;                 // keys per shared-memory tile
-constexpr int kDecStages = 3;                 // ring depth for d = 128 (K and V tiles each 32 KiB)
+constexpr int kDecStages = 3;                 // ring depth (K and V tiles each)
 constexpr int kDecTileBytes = 32768;          // a tile of d = 128
 constexpr int kDecHalfBytes = 16384;          // one 128-key x 64-element box
 // Head dimension D (128 or 64): a tile is 128 keys x D 16-bit elements, one or two swizzled
@@ -42,7 +42,7 @@ struct DecodeParams {
     float scale_log2;
     // paged cache (block_table != nullptr): key j of sequence b is row j % page_size of page
     // block_table[b * table_stride + j / page_size]; the tensor maps then run over
-    // [pages, page_size, Hkv, 128]; page_size is a multiple of kDecTile, or 16, 32 or 64 (then a
+    // [pages, page_size, Hkv, d]; page_size is a multiple of kDecTile, or 16, 32 or 64 (then a
     // tile is several pages and the TMA box is one page high)
     const int* block_table;
     int page_size, table_stride;
@@ -97,7 +97,7 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // kMulti: Sq > 1 query rows per sequence, the last Sq positions of its cache (decoding after
 // several tokens were appended, Appendix C with more than one new token): the 16 MMA rows of a
 // CTA are then (token, head) pairs of one kv head, and query token t sees the keys up to
-// position len - Sq + t.  q is [B,Sq,Hq,128], the partials [B,Sq,Hq,NC,...].
+// position len - Sq + t.  q is [B,Sq,Hq,d], the partials [B,Sq,Hq,NC,...].
 // grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
 // T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
 // D: the head dimension, 128 or 64.
