@@ -60,8 +60,9 @@ extern "C" {
  * Prefill / general forward, fp16 inputs and output (Section 5.1 operator; Section 4.1 method).
  *   q [B,Sq,Hq,d], k,v [B,Skv,Hkv,d], o [B,Sq,Hq,d] fp16, contiguous; lse [B,Hq,Sq] float or NULL.
  *   d must be 128, 64 (the short vision workload of the evaluation section) or 256; 64 and 256
- *   have kernels of their own and are taken by fa_forward, fa_forward_bf16 and fa_forward_ex
- *   with variant 0 only; every other entry point wants 128.
+ *   have kernels of their own and are taken by fa_forward, fa_forward_bf16, fa_forward_host and
+ *   fa_forward_ex (variant 0; d = 64 also variant 3).  The packed-batch and the 16-bit decode
+ *   entry points take 128 and 64; the 8-bit and projection entry points want 128.
  *   B == 0 or Sq == 0 is a successful no-op.  Skv == 0 gives O = 0, LSE = -inf.
  *   o and lse must not alias the inputs.
  */
@@ -158,8 +159,8 @@ size_t fa_forward_proj_workspace_bytes(int B, int Sq);
  * fa_forward, sequence by sequence.  Sequence b owns rows [cu_seqlens_q[b], cu_seqlens_q[b+1])
  * of q and o and rows [cu_seqlens_k[b], cu_seqlens_k[b+1]) of k and v; with the causal mask its
  * diagonal is aligned bottom-right, as in fa_forward, sequence by sequence.
- *   q, o [total_q, Hq, d]; k, v [total_k, Hkv, d], contiguous, 16-byte aligned, dtype as given
- *   (FA_DTYPE_FP16 or FA_DTYPE_BF16; o has the same type); lse [Hq, total_q] float or NULL;
+ *   q, o [total_q, Hq, d]; k, v [total_k, Hkv, d], d = 128 or 64, contiguous, 16-byte aligned,
+ *   dtype as given (FA_DTYPE_FP16 or FA_DTYPE_BF16; o has the same type); lse [Hq, total_q] float or NULL;
  *   cu_seqlens_q, cu_seqlens_k: int32 [B + 1] on the DEVICE, non-decreasing, first entry 0, last
  *   entry total_q / total_k; max_seqlen_q / max_seqlen_k: upper bounds of the sequence lengths
  *   (they size the launch: a longer sequence would be cut off at the bound).

@@ -210,13 +210,22 @@ fa::FwdParams dense_fwd_params(const fa_params& p) {
     return fp;
 }
 
+// Head dimension 64: keys from which the ping-pong kernel is used (128 < Skv <= 256 has the
+// short-sequence pipeline of its own; up to 128 keys the kernel with four small CTAs per SM, which
+// the ping-pong kernel ties there and beats by 3 to 37 % from 300 keys on).
+#ifndef FA_D64_PINGPONG_FROM
+#define FA_D64_PINGPONG_FROM 257
+#endif
+constexpr int kD64PingPongFrom = FA_D64_PINGPONG_FROM;
+
 int forward_impl(const fa_params& in, cudaStream_t st) {
     fa_params p = in;
     // ---- validation (no CUDA call before it passes)
     if (p.B < 0 || p.Hq <= 0 || p.Hkv <= 0 || p.Sq < 0 || p.Skv < 0 || p.d <= 0) return FA_ERR_SHAPE;
     if (p.Hq % p.Hkv) return FA_ERR_SHAPE;
     if (p.d != 128 && p.d != 64 && p.d != 256) return FA_ERR_UNSUPPORTED;
-    if (p.d != 128 && p.variant != 0) return FA_ERR_UNSUPPORTED;  // d = 64 and d = 256 have kernels of their own
+    // d = 64 and d = 256 have kernels of their own (d = 64 also takes variant 3, the ping-pong kernel)
+    if (p.d != 128 && p.variant != 0 && !(p.d == 64 && p.variant == 3)) return FA_ERR_UNSUPPORTED;
     if (p.dtype != FA_DTYPE_FP16 && p.dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (p.o_dtype != p.dtype && p.o_dtype != FA_DTYPE_FP32) return FA_ERR_UNSUPPORTED;
     if (!(p.scale >= 0.f) || isinf(p.scale)) return FA_ERR_UNSUPPORTED;
@@ -262,6 +271,16 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         // short sequences: all keys are one tile; a persistent pipeline over (batch, head, two query tiles)
         return bf16 ? fa::launch_d64_stream<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
                     : fa::launch_d64_stream<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
+    }
+    if (p.d == 64 && (p.variant == 3 || (p.variant == 0 && p.Skv >= kD64PingPongFrom))) {
+        // long sequences: the ping-pong kernel with tiles of one 64-element box (see PpOperands)
+        CUtensorMap to = tq;
+        if (!fp.o_fp32) {  // the output leaves through TMA stores of 32 rows x 64 columns
+            rc = encode_map(&to, p.o, p.B, p.Sq, p.Hq, p.o_stride[0], p.o_stride[1], p.o_stride[2], 32, bf16, 64);
+            if (rc) return rc;
+        }
+        return bf16 ? fa::launch_pingpong<__nv_bfloat16, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
+                    : fa::launch_pingpong<__half, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
     }
     if (p.d == 64) {  // one CTA per (batch, head, query tile), four CTAs per SM
         auto kern = bf16 ? fa::fa_fwd_d64_slim_kernel<__nv_bfloat16> : fa::fa_fwd_d64_slim_kernel<__half>;
@@ -554,8 +573,8 @@ int fa_forward_ex(const fa_params* p, void* stream) {
     return forward_impl(*p, static_cast<cudaStream_t>(stream));
 }
 
-// Packed batch; K and V packed too (block_table == nullptr: k, v [total_k,Hkv,128], cu_seqlens_k) or in
-// pages (k, v [num_pages,page_size,Hkv,128], seqlens_k and the block table; total_k = num_pages * page_size).
+// Packed batch; K and V packed too (block_table == nullptr: k, v [total_k,Hkv,d], cu_seqlens_k) or in
+// pages (k, v [num_pages,page_size,Hkv,d], seqlens_k and the block table; total_k = num_pages * page_size).
 static int varlen_impl(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens_q,
                        const int* cu_seqlens_k, int B, int Hq, int Hkv, int total_q, int total_k, int max_seqlen_q,
                        int max_seqlen_k, int d, int causal, float scale, int dtype, void* stream,
@@ -564,7 +583,7 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
         return FA_ERR_SHAPE;
     if (Hq % Hkv) return FA_ERR_SHAPE;
     if (max_seqlen_q > total_q || (!block_table && max_seqlen_k > total_k)) return FA_ERR_SHAPE;
-    if (d != 128) return FA_ERR_UNSUPPORTED;
+    if (d != 128 && d != 64) return FA_ERR_UNSUPPORTED;
     if (dtype != FA_DTYPE_FP16 && dtype != FA_DTYPE_BF16) return FA_ERR_UNSUPPORTED;
     if (!(scale >= 0.f) || isinf(scale)) return FA_ERR_UNSUPPORTED;
     if (Hq > 65535 || B > 65535) return FA_ERR_UNSUPPORTED;
@@ -586,7 +605,7 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     fp.B = B; fp.Hq = Hq; fp.Hkv = Hkv; fp.Sq = max_seqlen_q; fp.Skv = max_seqlen_k;
     fp.causal = causal ? 1 : 0;
     fp.scale_log2 = fmaxf(scale * 1.4426950408889634f, 1e-30f);
-    fp.o_sb = 0; fp.o_ss = (long long)Hq * 128; fp.o_sh = 128;
+    fp.o_sb = 0; fp.o_ss = (long long)Hq * d; fp.o_sh = d;
     fp.o_fp32 = 0;
     fp.o_align32 = 0;
     fp.n_qtiles = (max_seqlen_q + fa::kTile - 1) / fa::kTile;
@@ -604,7 +623,7 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     fp.cu_q = cu_seqlens_q;
     fp.cu_k = cu_seqlens_k;
     fp.total_q = total_q;
-    fp.d = 128;
+    fp.d = d;
     fp.block_table = block_table;
     fp.seqlens_k = block_table ? cu_seqlens_k : nullptr;   // per-sequence key counts in the paged form
     fp.table_stride = table_stride;
@@ -624,16 +643,19 @@ static int varlen_impl(const void* q, const void* k, const void* v, void* o, flo
     }
     // the packed tensors as one batch entry; a sequence's rows are reached through the prefix sums
     CUtensorMap tq, tk, tv, to;
-    rc = encode_map(&tq, q, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 128, bf16);
+    rc = encode_map(&tq, q, 1, total_q, Hq, (int64_t)total_q * Hq * d, (int64_t)Hq * d, d, 128, bf16, d);
     if (rc) return rc;
     // K and V: one batch entry with every sequence back to back, or one entry per page
     const int slabs = block_table ? num_pages : 1, slab_rows = block_table ? page_size : total_k;
-    rc = encode_map(&tk, k, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    rc = encode_map(&tk, k, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * d, (int64_t)Hkv * d, d, 128, bf16, d);
     if (rc) return rc;
-    rc = encode_map(&tv, v, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * 128, (int64_t)Hkv * 128, 128, 128, bf16);
+    rc = encode_map(&tv, v, slabs, slab_rows, Hkv, (int64_t)slab_rows * Hkv * d, (int64_t)Hkv * d, d, 128, bf16, d);
     if (rc) return rc;
-    rc = encode_map(&to, o, 1, total_q, Hq, (int64_t)total_q * Hq * 128, (int64_t)Hq * 128, 128, 32, bf16);
+    rc = encode_map(&to, o, 1, total_q, Hq, (int64_t)total_q * Hq * d, (int64_t)Hq * d, d, 32, bf16, d);
     if (rc) return rc;
+    if (d == 64)
+        return bf16 ? fa::launch_pingpong<__nv_bfloat16, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
+                    : fa::launch_pingpong<__half, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
     return bf16 ? fa::launch_pingpong<__nv_bfloat16>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
                 : fa::launch_pingpong<__half>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
 }

@@ -2,11 +2,12 @@
 // evaluation section: DeiT-like, 197 tokens, 12 heads, large batches; causal and longer
 // sequences work too).  The tcgen05 tile shapes of d = 64: Q, K and V tiles are single 128 x 64
 // swizzled TMA boxes; S = Q K^T takes four k-steps of 16; O += P V is an N = 64 MMA with V as the
-// N-major operand.  Two kernels:
+// N-major operand.  Three kernels:
 //   fa_fwd_d64_stream_kernel (prefill_d64_stream.cuh)  128 < Skv <= 256: all keys as one tile,
 //                            single-pass softmax, a persistent pipeline over (batch, head, two query tiles)
-//   fa_fwd_d64_slim_kernel   (here) any Skv: online softmax over 128-key tiles, one thread per
-//                            query row, O kept in registers
+//   fa_fwd_pingpong_kernel   (prefill_pingpong.cuh, D = 64)  longer sequences and packed batches
+//   fa_fwd_d64_slim_kernel   (here) any Skv, used up to 128 keys: online softmax over 128-key
+//                            tiles, one thread per query row, O kept in registers
 #pragma once
 
 #include "prefill_simple.cuh"

@@ -48,12 +48,18 @@ static_assert((kPpQBufs + kPpNK + kPpNV) * kTileBytes + 3072 <= 232448, "shared 
 // contraction, so a product takes four instead of eight; the probabilities are rounded to e4m3
 // four to a 32-bit column of tensor memory, times kP8Scale so that they use the format's range:
 // with the reference max at most 2^kP8Threshold behind the row max they stay below 2^8 < 448.
-template <bool kF8>
+// Head dimension 64 (D; 16-bit operands only) has the same byte layout: a row of a Q, K or V tile
+// is 64 elements = 128 bytes, one box; Q K^T then contracts over four MMAs of 16 elements, P V is
+// eight MMAs of 16 keys with N = 64, and O takes 64 columns of tensor memory.
+template <bool kF8, int D = 128>
 struct PpOperands {
-    static constexpr int kKvSlotBytes = kF8 ? 16384 : kTileBytes;   // one K or V ring slot
-    static constexpr int kQBytes = kF8 ? 16384 : kTileBytes;        // bytes a Q load delivers
-    static constexpr int kSteps = kF8 ? 4 : 8;                      // MMAs per 128 x 128 x 128 product
-    static constexpr int kPCols = kF8 ? 8 : 16;                     // tensor-memory columns of 32 probabilities
+    static_assert(D == 128 || (D == 64 && !kF8), "head dimension 128, or 64 with 16-bit operands");
+    static constexpr bool kOneBox = kF8 || D == 64;                     // a tile row is 128 bytes
+    static constexpr int kKvSlotBytes = kOneBox ? 16384 : kTileBytes;   // one K or V ring slot
+    static constexpr int kQBytes = kOneBox ? 16384 : kTileBytes;        // bytes a Q load delivers
+    static constexpr int kSteps = kOneBox ? 4 : 8;                      // MMAs of Q K^T (32 bytes of every row each)
+    static constexpr int kPvSteps = kF8 ? 4 : 8;                        // MMAs of P V (32 or 16 keys each)
+    static constexpr int kPCols = kF8 ? 8 : 16;                         // tensor-memory columns of 32 probabilities
 };
 constexpr float kP8Threshold = 4.0f;   // log2 units: how far the row max may outgrow the reference (FP8)
 constexpr float kP8ScaleLog2 = 4.0f;   // log2 of the factor on the FP8 probabilities
@@ -270,12 +276,12 @@ struct PpRing {
 };
 
 // The thread that issues S = Q K^T of every step.
-template <typename T, bool kTmaOut, bool kVarlen, bool kF8>
+template <typename T, bool kTmaOut, bool kVarlen, bool kF8, int D>
 __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK, uint32_t tmem, const FwdParams& p,
                                          int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
     constexpr uint32_t idesc = kF8 ? instr_desc_e4m3(128, 128, false, false) : instr_desc_f16(kBf16, 128, 128, false, false);
-    using Op = PpOperands<kF8>;
+    using Op = PpOperands<kF8, D>;
     uint32_t g = 0;
     PpRing<kPpNK> ring;
     PpItems<kVarlen> items;
@@ -296,8 +302,8 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
 #pragma unroll
             for (int ks = 0; ks < Op::kSteps; ++ks) {
                 // one MMA takes 32 bytes of every row: 16 16-bit elements (a row of d = 128 is two
-                // 128-byte boxes) or 32 8-bit ones (one box)
-                const uint32_t koff = kF8 ? (uint32_t)(ks * 32) >> 4 : ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                // 128-byte boxes, one of d = 64 a single one) or 32 8-bit ones (one box)
+                const uint32_t koff = Op::kOneBox ? (uint32_t)(ks * 32) >> 4 : ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
                 if (kF8) mma_ss_lo_f8(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
                 else mma_ss_lo(tmem + 128 + 128 * buf, a_lo + koff, b_lo + koff, idesc, ks > 0 ? 1u : 0u);
             }
@@ -310,12 +316,12 @@ __device__ __forceinline__ void pp_run_s(uint32_t bar0, uint32_t sQ, uint32_t sK
 }
 
 // The thread that issues O += P V of every step.
-template <typename T, bool kVarlen, bool kF8>
+template <typename T, bool kVarlen, bool kF8, int D>
 __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t tmem, const FwdParams& p,
                                           int total_items, volatile uint32_t* abort_flag) {
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
-    constexpr uint32_t idesc = kF8 ? instr_desc_e4m3(128, 128, false, true) : instr_desc_f16(kBf16, 128, 128, false, true);
-    using Op = PpOperands<kF8>;
+    constexpr uint32_t idesc = kF8 ? instr_desc_e4m3(128, 128, false, true) : instr_desc_f16(kBf16, 128, D, false, true);
+    using Op = PpOperands<kF8, D>;
     uint32_t g = 0;
     PpRing<kPpNV> ring;
     PpItems<kVarlen> items;
@@ -329,12 +335,13 @@ __device__ __forceinline__ void pp_run_pv(uint32_t bar0, uint32_t sV, uint32_t t
             if (j == 0 && ord > 0 && !mbar_wait(pp_bar(bar0, ppb::o_free), (ord - 1) & 1, abort_flag, 141)) return;
             if (!mbar_wait(pp_bar(bar0, ppb::p_full + buf), (g >> 1) & 1, abort_flag, 142)) return;
             tc_fence_after();
-            // V is the N-major operand: a key is a row of 128 elements of d.  16-bit: two 128-byte
-            // column blocks kHalfBytes apart, 16 keys (2048 bytes) per MMA; 8-bit: one block, 32 keys
-            // (4096 bytes) per MMA.  Either way an MMA reads 8 columns of P.
-            const uint32_t b_lo = desc_lo(sV + ring.slot * Op::kKvSlotBytes, kHalfBytes);
+            // V is the N-major operand: a key is a row of d elements.  16-bit, d = 128: two 128-byte
+            // column blocks kHalfBytes apart, 16 keys (2048 bytes) per MMA; d = 64: one block, the
+            // same 16 keys per MMA; 8-bit: one block, 32 keys (4096 bytes) per MMA.  Either way an
+            // MMA reads 8 columns of P.
+            const uint32_t b_lo = desc_lo(sV + ring.slot * Op::kKvSlotBytes, D == 64 ? 16 : kHalfBytes);
 #pragma unroll
-            for (int ks = 0; ks < Op::kSteps; ++ks) {
+            for (int ks = 0; ks < Op::kPvSteps; ++ks) {
                 if (kF8) mma_ts_lo_f8(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (4096 >> 4), idesc,
                                       (ks > 0) ? 1u : (j > 0 ? 1u : 0u));
                 else mma_ts_lo(tmem, tmem + 384 + 64 * buf + ks * 8, b_lo + ks * (2048 >> 4), idesc,
@@ -375,15 +382,15 @@ __device__ __forceinline__ void pp_paged_tile(const FwdParams& p, int page, int 
 
 // The thread that loads Q of every item and K of every step.  (Packed batches: the tensor maps
 // have one batch entry that holds every sequence back to back.)
-// One tile: two 64-element boxes of a 16-bit tensor, or one 128-byte box of an 8-bit one.
-template <bool kF8>
+// One tile: two 64-element boxes of a 16-bit tensor of d = 128, or one 128-byte box (8-bit, or d = 64).
+template <bool kOneBox>
 __device__ __forceinline__ void pp_load_tile(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int h, int s0, int b,
                                              uint64_t policy) {
-    if (kF8) tma_load_4d_hint(dst, tm, bar, 0, h, s0, b, policy);
+    if (kOneBox) tma_load_4d_hint(dst, tm, bar, 0, h, s0, b, policy);
     else load_tile_hint(dst, tm, bar, h, s0, b, policy);
 }
 
-template <bool kVarlen, bool kF8>
+template <bool kVarlen, bool kF8, int D>
 __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint32_t sK, const CUtensorMap* tm_q,
                                                const CUtensorMap* tm_k, const FwdParams& p, int total_items,
                                                volatile uint32_t* abort_flag) {
@@ -398,24 +405,24 @@ __device__ __forceinline__ void pp_run_load_qk(uint32_t bar0, uint32_t sQ, uint3
         const uint32_t qb = ord & 1;
         // passes at once the first time each buffer is used
         if (!mbar_wait(pp_bar(bar0, ppb::q_empty + qb), ((ord >> 1) & 1) ^ 1, abort_flag, 150)) return;
-        mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), PpOperands<kF8>::kQBytes);
-        pp_load_tile<kF8>(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
+        mbar_expect_tx(pp_bar(bar0, ppb::q_full + qb), PpOperands<kF8, D>::kQBytes);
+        pp_load_tile<PpOperands<kF8, D>::kOneBox>(sQ + qb * kTileBytes, tm_q, pp_bar(bar0, ppb::q_full + qb), it.h,
                        kVarlen ? it.q_base + it.q0 : it.q0, kVarlen ? 0 : it.b, pol_q);
         int page = (kVarlen && p.block_table != nullptr) ? it.page0 : 0;
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::k_empty + ring.slot), ring.par ^ 1, abort_flag, 151)) return;
-            mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), PpOperands<kF8>::kKvSlotBytes);
+            mbar_expect_tx(pp_bar(bar0, ppb::k_full + ring.slot), PpOperands<kF8, D>::kKvSlotBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
             pp_paged_tile<kVarlen>(p, page, j, row, slab);
             page = page_next;
-            pp_load_tile<kF8>(sK + ring.slot * PpOperands<kF8>::kKvSlotBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
+            pp_load_tile<PpOperands<kF8, D>::kOneBox>(sK + ring.slot * PpOperands<kF8, D>::kKvSlotBytes, tm_k, pp_bar(bar0, ppb::k_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }
 
 // The thread that loads V of every step.
-template <bool kVarlen, bool kF8>
+template <bool kVarlen, bool kF8, int D>
 __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const CUtensorMap* tm_v, const FwdParams& p,
                                               int total_items, volatile uint32_t* abort_flag) {
     tma_prefetch_desc(tm_v);
@@ -429,11 +436,11 @@ __device__ __forceinline__ void pp_run_load_v(uint32_t bar0, uint32_t sV, const 
         for (int j = 0; j < it.n; ++j, ring.next()) {
             const int page_next = pp_page_of<kVarlen>(p, it.b, j + 1, it.n, it.Skv);
             if (!mbar_wait(pp_bar(bar0, ppb::v_empty + ring.slot), ring.par ^ 1, abort_flag, 152)) return;
-            mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), PpOperands<kF8>::kKvSlotBytes);
+            mbar_expect_tx(pp_bar(bar0, ppb::v_full + ring.slot), PpOperands<kF8, D>::kKvSlotBytes);
             int row = kVarlen ? it.k_base + j * kTile : j * kTile, slab = kVarlen ? 0 : it.b;
             pp_paged_tile<kVarlen>(p, page, j, row, slab);
             page = page_next;
-            pp_load_tile<kF8>(sV + ring.slot * PpOperands<kF8>::kKvSlotBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
+            pp_load_tile<PpOperands<kF8, D>::kOneBox>(sV + ring.slot * PpOperands<kF8, D>::kKvSlotBytes, tm_v, pp_bar(bar0, ppb::v_full + ring.slot), it.hk, row, slab, pol_kv);
         }
     }
 }
@@ -447,10 +454,10 @@ __device__ __forceinline__ bool pp_warp_wait(uint32_t bar, uint32_t parity, vola
 }
 
 // One thread of a softmax warpgroup: its state across the steps of an item, and the step.
-template <typename T, bool kVarlen, bool kF8>
+template <typename T, bool kVarlen, bool kF8, int D>
 struct PpSoftmax {
     static_assert(!(kF8 && kVarlen), "packed batches take 16-bit operands");
-    using Op = PpOperands<kF8>;
+    using Op = PpOperands<kF8, D>;
     // fixed for the kernel
     uint32_t bar0;
     volatile uint32_t* abort_flag;
@@ -535,7 +542,7 @@ struct PpSoftmax {
                 tc_fence_after();
                 const float alpha = grow ? ((m_prev == -INFINITY) ? 0.f : fast_exp2((m_prev - mx) * scale_log2)) : 1.f;
 #pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < D / 16; ++c) {
                     uint32_t o[16];
                     tmem_ld_x16(tO + c * 16, o);
                     tmem_wait_ld();
@@ -564,13 +571,13 @@ struct PpSoftmax {
             // Their probabilities are exact zeros, but 0 * NaN would still poison O, so those
             // rows are cleared in shared memory before P V of this step may start (a contiguous
             // tensor gets the same from the zero fill of its TMA loads).  Thread r owns key row r:
-            // its 256 bytes are one 128-byte line in each half of the tile, whatever the swizzle.
+            // its bytes are one 128-byte line in each 64-element half of the tile, whatever the swizzle.
             static_assert(kPpNV == 2, "the V slot of step g is taken to be g & 1");
             if (!pp_warp_wait(pp_bar(bar0, ppb::v_full + w), (g >> 1) & 1, abort_flag, 124 + w)) return false;
             if (r >= Skv - j * kTile) {
-                const uint32_t line = sV + (uint32_t)w * kTileBytes + (uint32_t)r * 128u;
+                const uint32_t line = sV + (uint32_t)w * Op::kKvSlotBytes + (uint32_t)r * 128u;
 #pragma unroll
-                for (int c = 0; c < 16; ++c)
+                for (int c = 0; c < D / 8; ++c)
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(line + (uint32_t)(c >> 3) * kHalfBytes + (uint32_t)(c & 7) * 16u), "r"(0u) : "memory");
             }
             fence_proxy_async_smem();
@@ -599,14 +606,14 @@ struct PpSoftmax {
 // and counts them in done[batch * n_qtiles + query tile]; four warps and Hq heads make a row
 // block of O complete.
 // The whole kernel but for the release of tensor memory; returns false if nothing was set up.
-template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8, bool kProj>
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8, bool kProj, int D = 128>
 __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                              const CUtensorMap& tm_o, const FwdParams& p, const int total_items,
                                              PpStatic& ss, const uint32_t smem_base, unsigned int* done) {
-    static_assert(!kProj || (kTmaOut && !kVarlen), "the projection phase reads a contiguous 16-bit O");
+    static_assert(!kProj || (kTmaOut && !kVarlen && D == 128), "the projection phase reads a contiguous 16-bit O of d = 128");
     const uint32_t sQ = smem_base;
     const uint32_t sK = sQ + kPpQBufs * kTileBytes;
-    const uint32_t sV = sK + kPpNK * PpOperands<kF8>::kKvSlotBytes;
+    const uint32_t sV = sK + kPpNK * PpOperands<kF8, D>::kKvSlotBytes;
     const uint32_t bar0 = smem_u32(&ss.bars[0]);
     volatile uint32_t* abort_flag = &ss.abort_flag;
 
@@ -645,7 +652,7 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
         const uint32_t tS = tmem_base + lane_sel + 128 + 128 * w;
         const uint32_t tP = tmem_base + lane_sel + 384 + 64 * w;
         const float scale_log2 = p.scale_log2;
-        PpSoftmax<T, kVarlen, kF8> sm;
+        PpSoftmax<T, kVarlen, kF8, D> sm;
         sm.sV = sV;
         sm.r = r;
         sm.bar0 = bar0;
@@ -758,8 +765,10 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
                 tc_fence_after();
                 tmem_ld_x32(tO, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                 tmem_ld_x32(tO + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-                tmem_ld_x32(tO + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
-                tmem_ld_x32(tO + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+                if (D == 128) {
+                    tmem_ld_x32(tO + 64, *reinterpret_cast<uint32_t(*)[32]>(&s[64]));
+                    tmem_ld_x32(tO + 96, *reinterpret_cast<uint32_t(*)[32]>(&s[96]));
+                }
                 tmem_wait_ld();
                 // O is in registers: the next item's first P V may overwrite it
                 tc_fence_before();
@@ -778,7 +787,7 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
                     const uint32_t q_buf = sQ + (uint32_t)(ord & 1) * kTileBytes;
                     const uint32_t row_base = q_buf + (uint32_t)r * 128u;
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
+                    for (int c = 0; c < D / 8; ++c) {
                         // 16-byte chunk c & 7 of the row's half c >> 3, at its swizzled place
                         const uint32_t addr = row_base + (uint32_t)(c >> 3) * kHalfBytes + (((uint32_t)(c & 7) ^ ((uint32_t)r & 7u)) << 4);
                         const uint32_t w0 = pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l);
@@ -796,7 +805,7 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
                     if (lane == 0 && box) {
                         const uint32_t src = q_buf + (uint32_t)(warp & 3) * 4096u;
                         tma_store_4d(&tm_o, src, 0, it.h, kVarlen ? it.q_base + row0 : row0, kVarlen ? 0 : it.b);
-                        tma_store_4d(&tm_o, src + kHalfBytes, 64, it.h, kVarlen ? it.q_base + row0 : row0, kVarlen ? 0 : it.b);
+                        if (D == 128) tma_store_4d(&tm_o, src + kHalfBytes, 64, it.h, kVarlen ? it.q_base + row0 : row0, kVarlen ? 0 : it.b);
                         tma_store_commit();
                     }
                     q_back = ord & 1;  // handed back to the loader after this warp's next step
@@ -806,7 +815,7 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
                         // the ragged end of a sequence: each thread writes its own row
                         T* dst = static_cast<T*>(p.o) + obase;
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
+                        for (int c = 0; c < D / 8; ++c)
                             reinterpret_cast<uint4*>(dst)[c] =
                                 make_uint4(pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l),
                                            pack2<T>(__uint_as_float(s[8 * c + 2]) * inv_l, __uint_as_float(s[8 * c + 3]) * inv_l),
@@ -817,14 +826,14 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
                     if (p.o_fp32) {
                         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.o) + obase);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
+                        for (int i = 0; i < D / 4; ++i)
                             dst[i] = make_float4(__uint_as_float(s[4 * i]) * inv_l, __uint_as_float(s[4 * i + 1]) * inv_l,
                                                  __uint_as_float(s[4 * i + 2]) * inv_l,
                                                  __uint_as_float(s[4 * i + 3]) * inv_l);
                     } else {
                         T* dst = static_cast<T*>(p.o) + obase;
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
+                        for (int c = 0; c < D / 8; ++c)
                             reinterpret_cast<uint4*>(dst)[c] =
                                 make_uint4(pack2<T>(__uint_as_float(s[8 * c]) * inv_l, __uint_as_float(s[8 * c + 1]) * inv_l),
                                            pack2<T>(__uint_as_float(s[8 * c + 2]) * inv_l, __uint_as_float(s[8 * c + 3]) * inv_l),
@@ -842,17 +851,17 @@ __device__ __forceinline__ bool pp_attention(const CUtensorMap& tm_q, const CUte
     } else {
         setmaxnreg_dec<kPipeOtherRegs>();
         if (lane == 0) {
-            if (warp == 8) pp_run_s<T, kTmaOut, kVarlen, kF8>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
-            else if (warp == 10) pp_run_pv<T, kVarlen, kF8>(bar0, sV, tmem_base, p, total_items, abort_flag);
-            else if (warp == 9) pp_run_load_qk<kVarlen, kF8>(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
-            else pp_run_load_v<kVarlen, kF8>(bar0, sV, &tm_v, p, total_items, abort_flag);
+            if (warp == 8) pp_run_s<T, kTmaOut, kVarlen, kF8, D>(bar0, sQ, sK, tmem_base, p, total_items, abort_flag);
+            else if (warp == 10) pp_run_pv<T, kVarlen, kF8, D>(bar0, sV, tmem_base, p, total_items, abort_flag);
+            else if (warp == 9) pp_run_load_qk<kVarlen, kF8, D>(bar0, sQ, sK, &tm_q, &tm_k, p, total_items, abort_flag);
+            else pp_run_load_v<kVarlen, kF8, D>(bar0, sV, &tm_v, p, total_items, abort_flag);
         }
         __syncwarp();
     }
     return true;
 }
 
-template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8 = false>
+template <typename T, bool kTmaOut, bool kSingle, bool kVarlen, bool kF8 = false, int D = 128>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -862,8 +871,8 @@ fa_fwd_pingpong_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // plus seven 32 KiB tiles.  The alignment is checked rather than assumed.
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(1024) PpStatic ss;
-    if (!pp_attention<T, kTmaOut, kSingle, kVarlen, kF8, false>(tm_q, tm_k, tm_v, tm_o, p, total_items, ss,
-                                                                smem_u32(smem_raw), nullptr))
+    if (!pp_attention<T, kTmaOut, kSingle, kVarlen, kF8, false, D>(tm_q, tm_k, tm_v, tm_o, p, total_items, ss,
+                                                                   smem_u32(smem_raw), nullptr))
         return;
     tc_fence_before();
     __syncthreads();
@@ -925,28 +934,29 @@ inline FwdParams pp_plan_items(const FwdParams& fp, int grid, double bytes_per_k
 }
 
 // kF8: tq, tk, tv are maps over FP8 e4m3 bytes (boxes of 128 rows x 128 bytes) and T is the output type.
-template <typename T, bool kF8 = false>
+// D: the head dimension, 128, or 64 with 16-bit operands (maps with boxes of 64 elements either way).
+template <typename T, bool kF8 = false, int D = 128>
 int launch_pingpong(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                     const FwdParams& fp, cudaStream_t st, int* cuda_err) {
-    constexpr int smem = kPpQBufs * kTileBytes + (kPpNK + kPpNV) * PpOperands<kF8>::kKvSlotBytes;
+    constexpr int smem = kPpQBufs * kTileBytes + (kPpNK + kPpNV) * PpOperands<kF8, D>::kKvSlotBytes;
     // the single-copy step up to 32 kv tiles per item (timed: ahead by 3 % at 2048 keys, level at
     // 4096, behind by 1 % at 8192)
     const bool single = fp.o_fp32 || fp.Skv <= 32 * kTile;
     const bool varlen = fp.cu_q != nullptr;
     if (varlen && fp.o_fp32) return -3;
     if (kF8 && (varlen || fp.o_fp32)) return -3;
-    auto kern = kF8 ? fa_fwd_pingpong_kernel<T, true, true, false, kF8>
-                    : (varlen ? fa_fwd_pingpong_kernel<T, true, true, kF8 ? false : true>
-                              : (fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true, false>
-                                           : (single ? fa_fwd_pingpong_kernel<T, true, true, false>
-                                                     : fa_fwd_pingpong_kernel<T, true, false, false>)));
+    auto kern = kF8 ? fa_fwd_pingpong_kernel<T, true, true, false, kF8, D>
+                    : (varlen ? fa_fwd_pingpong_kernel<T, true, true, kF8 ? false : true, false, D>
+                              : (fp.o_fp32 ? fa_fwd_pingpong_kernel<T, false, true, false, false, D>
+                                           : (single ? fa_fwd_pingpong_kernel<T, true, true, false, false, D>
+                                                     : fa_fwd_pingpong_kernel<T, true, false, false, false, D>)));
     int sm_count = 0;
     cudaError_t e;
     if (int ce = prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count)) { *cuda_err = ce; return -7; }
     const long long total = (long long)fp.n_qtiles * fp.B * fp.Hq;
     if (total > 0x7fffffffll) return -3;
     const int grid = (int)(total < sm_count ? total : sm_count);
-    const FwdParams fpc = pp_plan_items(fp, grid, kF8 ? 256.0 : 512.0);
+    const FwdParams fpc = pp_plan_items(fp, grid, (kF8 || D == 64) ? 256.0 : 512.0);
     kern<<<grid, kPipeThreads, smem, st>>>(tq, tk, tv, to, fpc, (int)total);
     e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = (int)e; return -7; }

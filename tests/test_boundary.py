@@ -120,7 +120,7 @@ def test_varlen_validation(fa):
     assert call(Hkv=3) == fa.FA_ERR_SHAPE
     assert call(max_q=21) == fa.FA_ERR_SHAPE
     assert call(max_k=31) == fa.FA_ERR_SHAPE
-    assert call(d=64) == fa.FA_ERR_UNSUPPORTED
+    assert call(d=96) == fa.FA_ERR_UNSUPPORTED and call(d=256) == fa.FA_ERR_UNSUPPORTED   # 128 and 64 are taken
     assert call(dtype=fa.FA_DTYPE_FP32) == fa.FA_ERR_UNSUPPORTED
     assert call(scale=float("nan")) == fa.FA_ERR_UNSUPPORTED
     assert call(cu=None) == fa.FA_ERR_NULL

@@ -429,9 +429,31 @@ def test_d64_vision_batch_full_size_sampled(fa):
 
 
 def test_d64_is_refused_where_it_is_not_built(fa):
+    # of the forced kernel variants only the ping-pong kernel (3) exists for d = 64
     q = torch.zeros(1, 4, 2, 64, dtype=torch.float16, device=DEV)
     o = torch.empty_like(q); lse = torch.empty(1, 2, 4, device=DEV)
-    assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=3, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
+    for variant in (1, 2, 4):
+        assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=variant, raise_on_error=False) == fa.FA_ERR_UNSUPPORTED
+    assert fa.fa_forward_ex(q, q, q, o, lse, False, 0.1, variant=3) == fa.FA_OK
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_d64_pingpong_kernel_shape_grid(fa, causal):
+    # From 512 keys on d = 64 takes the ping-pong kernel (tiles of one 64-element box, O in 64
+    # columns of tensor memory).  Its small-item paths are reached by forcing it on short shapes;
+    # ragged tiles on both sides, chunked prefill (Sq < Skv), GQA, more items than CTAs.
+    for (B, hq, hkv, sq, skv) in [(1, 1, 1, 1, 1), (2, 3, 3, 128, 128), (2, 2, 1, 129, 300), (1, 2, 2, 77, 1500)]:
+        full_case_d64(fa, B, hq, hkv, sq, skv, causal, "fp16", seed=sq * 7 + skv, variant=3)
+    for (B, hq, hkv, sq, skv) in [(2, 3, 3, 512, 512), (1, 4, 2, 1100, 1100), (3, 5, 5, 513, 2049), (40, 4, 4, 600, 600)]:
+        full_case_d64(fa, B, hq, hkv, sq, skv, causal, "fp16", seed=sq * 3 + skv)
+    full_case_d64(fa, 1, 4, 1, 2300, 2300, causal, "bf16", seed=97)          # bf16, and its fp32-output mode
+
+
+def test_d64_long_sequences_full_size_sampled(fa):
+    # 8 x 32 heads x 4096 and 2 x 32 x 8192 causal: every element written, sampled rows against the oracle
+    for (B, S, seed) in ((8, 4096, 1071), (2, 8192, 1072)):
+        cfg = synth.PrefillConfig(f"d64-{S}", B, 32, 32, S, S, d=64, dtype="fp16", causal=True, seed=seed)
+        assert sampled_case(fa, cfg, 16, pairs=[(0, 0), (0, 31), (B - 1, 17)]) >= 48
 
 
 # ------------------------------------------------------------------ head dimension 256
@@ -680,6 +702,29 @@ def test_varlen_ragged_batch(fa, causal, dtype):
     lk = (1, 127, 128, 129, 300, 0, 700, 0, 90, 31, 515)
     cfg = synth.VarlenConfig("t", 4, 2, lq, lk, dtype=dtype, causal=causal, seed=600 + int(causal))
     varlen_case(fa, cfg, f"varlen ragged causal{int(causal)} {dtype}")
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_varlen_head_dimension_64(fa, dtype):
+    # packed batches with d = 64 (the same kernel, tiles of one 64-element box): the ragged batch
+    # of the d = 128 test, causal and not, and the same keys behind a block table
+    lq = (1, 127, 128, 129, 300, 0, 40, 33, 200, 31, 260)
+    lk = (1, 127, 128, 129, 300, 0, 700, 0, 90, 31, 515)
+    for causal in (True, False):
+        cfg = synth.VarlenConfig("t", 4, 2, lq, lk, d=64, dtype=dtype, causal=causal, seed=640 + int(causal))
+        varlen_case(fa, cfg, f"varlen d=64 causal{int(causal)} {dtype}")
+    lens = tuple([17, 130, 64, 5] * 30 + [1700])
+    cfg = synth.VarlenConfig("t", 2, 1, lens, lens, d=64, dtype=dtype, causal=True, seed=643)
+    o_packed, l_packed = varlen_case(fa, cfg, f"varlen d=64 many short + one long {dtype}")
+    q, k, v, cu_q, cu_k = synth.varlen_inputs(cfg, "cpu")
+    kp, vp, table = synth.paged_from_packed(k, v, lens, 128, seed=9, spare_pages=2, poison=True)
+    o = torch.full(tuple(q.shape), float("nan"), dtype=q.dtype, device=DEV)
+    lse = torch.full((cfg.Hq, q.shape[0]), float("nan"), dtype=torch.float32, device=DEV)
+    fa.fa_forward_varlen_paged(q.to(DEV), kp.to(DEV), vp.to(DEV), table.to(DEV), o, lse, cu_q.to(DEV),
+                               torch.tensor(lens, dtype=torch.int32, device=DEV), max(lens), max(lens), True, cfg.scale)
+    torch.cuda.synchronize()
+    check_status(fa)
+    assert torch.equal(o, o_packed) and torch.equal(lse, l_packed)      # the paged form: bit for bit the packed one
 
 
 def test_varlen_many_short_sequences_and_one_long(fa):
