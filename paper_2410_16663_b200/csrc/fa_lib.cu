@@ -267,11 +267,6 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
     rc = encode_map(&tv, p.v, p.B, p.Skv, p.Hkv, p.v_stride[0], p.v_stride[1], p.v_stride[2], 128, bf16, p.d);
     if (rc) return rc;
 
-    if (p.d == 64 && p.Skv > 128 && p.Skv <= 256) {
-        // short sequences: all keys are one tile; a persistent pipeline over (batch, head, two query tiles)
-        return bf16 ? fa::launch_d64_stream<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
-                    : fa::launch_d64_stream<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
-    }
     if (p.d == 64 && (p.variant == 3 || (p.variant == 0 && p.Skv >= kD64PingPongFrom))) {
         // long sequences: the ping-pong kernel with tiles of one 64-element box (see PpOperands)
         CUtensorMap to = tq;
@@ -281,6 +276,11 @@ int forward_impl(const fa_params& in, cudaStream_t st) {
         }
         return bf16 ? fa::launch_pingpong<__nv_bfloat16, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error)
                     : fa::launch_pingpong<__half, false, 64>(tq, tk, tv, to, fp, st, &t_last_cuda_error);
+    }
+    if (p.d == 64 && p.Skv > 128 && p.Skv <= 256) {   // (unless the ping-pong kernel was asked for)
+        // short sequences: all keys are one tile; a persistent pipeline over (batch, head, two query tiles)
+        return bf16 ? fa::launch_d64_stream<__nv_bfloat16>(tq, tk, tv, fp, st, &t_last_cuda_error)
+                    : fa::launch_d64_stream<__half>(tq, tk, tv, fp, st, &t_last_cuda_error);
     }
     if (p.d == 64) {  // one CTA per (batch, head, query tile), four CTAs per SM
         auto kern = bf16 ? fa::fa_fwd_d64_slim_kernel<__nv_bfloat16> : fa::fa_fwd_d64_slim_kernel<__half>;
