@@ -300,6 +300,7 @@ def run_product(args, rank, world, local_rank):
         out["prefill_varlen"] = run_varlen(fa, dev, peaks, small=args.small)
         out["prefill_d64"] = run_d64(fa, dev, peaks, small=args.small)
         out["prefill_d256"] = run_d256(fa, dev, peaks, small=args.small)
+        out["d64_long_and_decode"] = run_d64_long(fa, dev, peaks, small=args.small)
         out["prefill_fp8"] = run_prefill_fp8(fa, dev, peaks, small=args.small)
         out["prefill_proj"] = run_prefill_proj(fa, dev, peaks, small=args.small)
         out["e2e"] = run_e2e(args, fa, pc, dec, dev)
@@ -437,6 +438,58 @@ def run_d64(fa, dev, peaks, small=False, iters=10):
             "ms": round(ms, 4), "tflops": round(tf, 1), "gbs": round(gbs, 1), "algorithmic_bytes": nbytes,
             "bound": "hbm", "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
             "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}
+
+
+def run_d64_long(fa, dev, peaks, small=False, iters=5):
+    """Head dimension 64 on long sequences and in the decode stage, outside the timed steps: causal
+    fp16 self-attention, B = 8, 32 heads, 4096 tokens (the ping-pong kernel's d = 64 instantiation),
+    and the GQA decode configuration's lengths with d = 64 caches (the split-KV kernel's)."""
+    cfg = (synth.PrefillConfig("d64-4K", 8, 32, 32, 4096, 4096, d=64, dtype="fp16", causal=True, seed=1060)
+           if not small else
+           synth.PrefillConfig("d64-small", 1, 4, 4, 1024, 1024, d=64, dtype="fp16", causal=True, seed=1061))
+    q, k, v = synth.prefill_inputs(cfg, device=dev)
+    o = torch.empty_like(q)
+    lse = torch.empty(cfg.B, cfg.Hq, cfg.Sq, dtype=torch.float32, device=dev)
+    for _ in range(10):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fa.fa_forward(q, k, v, o, lse, cfg.causal, cfg.scale)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    tf = cfg.flops() / (ms * 1e-3) / 1e12
+    del q, k, v, o
+    dc = (synth.DecodeConfig("C5-gqa-d64", 64, 32, 8, 32768, 1024, 32768, d=64, dtype="fp16", seed=1021)
+          if not small else synth.DecodeConfig("C5-small-d64", 8, 8, 2, 4096, 512, 4096, d=64, dtype="fp16", seed=1062))
+    dq, dk, dv, sl = synth.decode_inputs(dc, dev, poison=True)
+    do = torch.empty_like(dq)
+    dl = torch.empty(dc.B, dc.Hq, dtype=torch.float32, device=dev)
+    ws = torch.empty(max(16, fa.fa_decode_workspace_bytes(dc.B, dc.Hq, dc.Hkv, dc.Smax, dc.d)), dtype=torch.uint8, device=dev)
+    sld = sl.to(dev)
+    for _ in range(3):
+        fa.fa_decode(dq, dk, dv, do, dl, sld, dc.scale, ws)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        fa.fa_decode(dq, dk, dv, do, dl, sld, dc.scale, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    dms = e0.elapsed_time(e1) / iters
+    rc, where, blk = fa.fa_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} at {where} block {blk}")
+    nbytes = float(sl.sum()) * dc.Hkv * dc.d * 2 * 2
+    gbs = nbytes / (dms * 1e-3) / 1e9
+    return {"prefill": {"workload": f"{cfg.name}: causal B={cfg.B} H={cfg.Hq} S={cfg.Sq} d=64 fp16",
+                        "kernel": "fa_fwd_pingpong_kernel, d = 64 instantiation", "ms": round(ms, 4), "tflops": round(tf, 1),
+                        "frac_nominal_tensor": round(tf / NOMINAL_TENSOR_TFLOPS, 4)},
+            "decode": {"workload": f"{dc.name}: B={dc.B} Hq={dc.Hq} Hkv={dc.Hkv} Skv~U[{dc.len_lo},{dc.len_hi}] d=64 fp16",
+                       "kernel": "fa_decode_split_mma_kernel, d = 64 instantiation", "ms": round(dms, 4), "gbs": round(gbs, 1),
+                       "kv_bytes": nbytes, "frac_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4),
+                       "frac_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)}}
 
 
 def run_d256(fa, dev, peaks, small=False, iters=5):
