@@ -128,7 +128,7 @@ __device__ __forceinline__ void tc_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-// ------------------------------------------------------------------ TMA (no multicast anywhere)
+// ------------------------------------------------------------------ TMA (every load goes to the issuing CTA only)
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
 }
