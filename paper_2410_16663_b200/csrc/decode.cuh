@@ -94,6 +94,171 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// The consumer warps' work in the keys-as-rows form (one query token, at most 8 query heads per
+// kv head).  A warp-level MMA has 16 rows and 8 columns: with the query heads as rows, as in the
+// general form below, a kv head with 1 to 8 query heads leaves half or more of every MMA to
+// padding.  Here the KEYS are the rows: S^T = K q^T (A = 16 keys x 16 elements of K by plain
+// ldmatrix, B = q^T, the 8 columns are the heads), and O^T += V^T P^T (A = 16 output columns x 16
+// keys of V by transposing ldmatrix, B = P^T, which is the accumulator layout of S^T transposed
+// 8 x 8 with movmatrix).  A tile then takes half the MMAs, a thread holds half the scores and
+// half the accumulators, and the row maxima and sums run over the lanes that share a column.
+// Leaves each warp's (max, sum, O) in mo / ml in the layout the merge expects; returns false
+// after a wait that gave up.
+template <typename T, int D>
+__device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint64_t* bars, volatile uint32_t* abort_flag,
+                                                     uint32_t sK, uint32_t sV, float* mo, float* ml, int warp, int lane,
+                                                     const T* q_rows, int G, int k_begin, int k_end, int n_tiles) {
+    constexpr int kStages = DecShape<D>::kStages, kTileB = DecShape<D>::kTileBytes;
+    constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
+    const int g = lane >> 2, t4 = lane & 3;
+    // q^T as B fragments: column g is head g, rows 2 t4, 2 t4 + 1 (and + 8) of every 16-element step
+    uint32_t qb[D / 16][2];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        const int d0 = ks * 16 + 2 * t4;
+        qb[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_rows + g * D + d0) : 0u;
+        qb[ks][1] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_rows + g * D + d0 + 8) : 0u;
+    }
+    // O^T: block i holds output columns 16 i + g (values 0, 1) and 16 i + 8 + g (values 2, 3) of heads 2 t4, 2 t4 + 1
+    float o[D / 16][4];
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};  // heads 2 t4 and 2 t4 + 1
+    const int key_w = warp * 32;  // this warp's keys inside a tile
+    bool ok = true;
+
+    for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % kStages;
+        const uint32_t parity = (t / kStages) & 1;
+        const int valid = min(kDecTile, k_end - (k_begin + t * kDecTile)) - key_w;  // valid keys of this warp's 32
+        ok = mbar_wait(smem_u32(&bars[st]), parity, abort_flag, 20);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint32_t pt[2][2];   // P^T as B fragments, per block of 16 keys
+        if (valid > 0) {
+            // ---- S^T = K q^T: two blocks of 16 keys
+            float sc[2][4];  // (key 16 mb + g | heads 2 t4, 2 t4 + 1), (key 16 mb + g + 8 | the same heads)
+            const uint32_t kt = sK + st * kTileB;
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                sc[mb][0] = sc[mb][1] = sc[mb][2] = sc[mb][3] = 0.f;
+                const int key = key_w + mb * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    // matrices: (keys 0-7, chunk 2 ks), (keys 8-15, chunk 2 ks), (keys 0-7, chunk 2 ks + 1), (keys 8-15, ...)
+                    const int chunk = 2 * ks + (lane >> 4);
+                    const uint32_t addr = kt + (chunk >> 3) * kDecHalfBytes + key * 128 + (((chunk & 7) ^ (key & 7)) << 4);
+                    uint32_t a[4];
+                    ldsm_x4(addr, a[0], a[1], a[2], a[3]);
+                    if (kBf16) mma_16816_bf16(sc[mb], a, qb[ks][0], qb[ks][1]);
+                    else mma_16816(sc[mb], a, qb[ks][0], qb[ks][1]);
+                }
+            }
+            // ---- mask, running max, probabilities
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                const int k_lo = mb * 16 + g;
+                if (k_lo >= valid) sc[mb][0] = sc[mb][1] = -INFINITY;
+                if (k_lo + 8 >= valid) sc[mb][2] = sc[mb][3] = -INFINITY;
+                mx0 = fmaxf(mx0, fmaxf(sc[mb][0], sc[mb][2]));
+                mx1 = fmaxf(mx1, fmaxf(sc[mb][1], sc[mb][3]));
+            }
+#pragma unroll
+            for (int sh = 4; sh <= 16; sh <<= 1) {  // over the lanes that hold other keys of the same heads
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+            }
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);  // finite: key 0 of the warp is valid
+            const float a0 = (m_run[0] == -INFINITY) ? 0.f : fast_exp2((m_run[0] - mn0) * p.scale_log2);
+            const float a1 = (m_run[1] == -INFINITY) ? 0.f : fast_exp2((m_run[1] - mn1) * p.scale_log2);
+            m_run[0] = mn0;
+            m_run[1] = mn1;
+            const float nm0 = -mn0 * p.scale_log2, nm1 = -mn1 * p.scale_log2;
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                const int k_lo = mb * 16 + g;
+                float* e = sc[mb];
+                e[0] = (k_lo < valid) ? fast_exp2(fmaf(e[0], p.scale_log2, nm0)) : 0.f;
+                e[1] = (k_lo < valid) ? fast_exp2(fmaf(e[1], p.scale_log2, nm1)) : 0.f;
+                e[2] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[2], p.scale_log2, nm0)) : 0.f;
+                e[3] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[3], p.scale_log2, nm1)) : 0.f;
+                s0 += e[0] + e[2];
+                s1 += e[1] + e[3];
+                // (key g | heads 2 t4, 2 t4 + 1) -> transposed: (head g | keys 2 t4, 2 t4 + 1), the B fragment
+                const uint32_t lo = pack2<T>(e[0], e[1]), hi = pack2<T>(e[2], e[3]);
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pt[mb][0]) : "r"(lo));
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pt[mb][1]) : "r"(hi));
+            }
+            l_run[0] = l_run[0] * a0 + s0;  // per-thread partial of the sum over keys (reduced at the end)
+            l_run[1] = l_run[1] * a1 + s1;
+#pragma unroll
+            for (int i = 0; i < D / 16; ++i) {
+                o[i][0] *= a0;
+                o[i][1] *= a1;
+                o[i][2] *= a0;
+                o[i][3] *= a1;
+            }
+        }
+        ok = mbar_wait(smem_u32(&bars[kStages + st]), parity, abort_flag, 21);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (valid > 0) {
+            const uint32_t vt = sV + st * kTileB;
+            if (valid < 32) {
+                // rows past the sequence may hold NaN bits: zero them (0 * NaN would poison O)
+                for (int i = lane; i < (32 - valid) * (D / 8); i += 32) {
+                    const int key = key_w + valid + i / (D / 8), ch = i % (D / 8);
+                    const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                }
+                __syncwarp();
+            }
+            // ---- O^T += V^T P^T: two steps of 16 keys, D / 16 blocks of 16 output columns
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                // matrices: (keys 0-7, chunk 2 i), (keys 0-7, chunk 2 i + 1), (keys 8-15, chunk 2 i), (keys 8-15, chunk 2 i + 1)
+                const int key = key_w + mb * 16 + (lane >> 4) * 8 + (lane & 7);
+#pragma unroll
+                for (int i = 0; i < D / 16; ++i) {
+                    const int ch = 2 * i + ((lane >> 3) & 1);
+                    const uint32_t addr = vt + (ch >> 3) * kDecHalfBytes + key * 128 + (((ch & 7) ^ (key & 7)) << 4);
+                    uint32_t a[4];
+                    ldsm_x4_trans(addr, a[0], a[1], a[2], a[3]);
+                    if (kBf16) mma_16816_bf16(o[i], a, pt[mb][0], pt[mb][1]);
+                    else mma_16816(o[i], a, pt[mb][0], pt[mb][1]);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars[2 * kStages + st]));
+    }
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // every warp is through with the ring: it becomes the merge buffer
+    if (ok) {
+        const int h0 = warp * 16 + 2 * t4;
+#pragma unroll
+        for (int i = 0; i < D / 16; ++i) {
+            mo[h0 * D + 16 * i + g] = o[i][0];
+            mo[(h0 + 1) * D + 16 * i + g] = o[i][1];
+            mo[h0 * D + 16 * i + 8 + g] = o[i][2];
+            mo[(h0 + 1) * D + 16 * i + 8 + g] = o[i][3];
+        }
+        if (g == 0) {
+            ml[h0 * 2] = m_run[0];
+            ml[h0 * 2 + 1] = l_run[0];
+            ml[(h0 + 1) * 2] = m_run[1];
+            ml[(h0 + 1) * 2 + 1] = l_run[1];
+        }
+    }
+    return ok;
+}
+
 // kMulti: Sq > 1 query rows per sequence, the last Sq positions of its cache (decoding after
 // several tokens were appended, Appendix C with more than one new token): the 16 MMA rows of a
 // CTA are then (token, head) pairs of one kv head, and query token t sees the keys up to
@@ -101,10 +266,13 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
 // T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
 // D: the head dimension, 128 or 64.
-template <bool kMulti, typename T = __half, int D = 128>
+// kKeyRows (one query token, at most 8 query heads per kv head): the consumers work in the
+// keys-as-rows form (dec_consume_key_rows).
+template <bool kMulti, typename T = __half, int D = 128, bool kKeyRows = false>
 __global__ void __launch_bounds__(kDecMmaThreads, DecShape<D>::kCtasPerSm)
 fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
+    static_assert(!(kKeyRows && kMulti), "keys as rows: one query token");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr int kStages = DecShape<D>::kStages, kTileB = DecShape<D>::kTileBytes;
@@ -222,6 +390,13 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
     } else {
         // ---------------------------------------------------------------- consumers
         const int g = lane >> 2, t4 = lane & 3;  // fragment row (query head g and g + 8) and column pair
+        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][D]
+        float* ml = mo + 4 * 16 * D;                                                         // [4][16][2]: m, l
+        bool ok = true;
+        if constexpr (kKeyRows) {
+            ok = dec_consume_key_rows<T, D>(p, bars, &abort_flag, sK, sV, mo, ml, warp, lane,
+                                            static_cast<const T*>(p.q) + row_index(0) * D, G, k_begin, k_end, n_tiles);
+        } else {
         // Q as A fragments for the D / 16 k-steps (rows >= G are zero)
         uint32_t qa[D / 16][4];
         {
@@ -244,7 +419,6 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
         float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;  // rows g and g + 8
         const int key_w = warp * 32;  // this warp's keys inside a tile
-        bool ok = true;
 
         for (int t = 0; t < n_tiles; ++t) {
             const int st = t % kStages;
@@ -376,8 +550,6 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
         l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-        float* mo = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));  // [4 warps][16 rows][D]
-        float* ml = mo + 4 * 16 * D;                                                         // [4][16][2]: m, l
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ok) {
 #pragma unroll
@@ -392,6 +564,7 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 ml[(warp * 16 + g + 8) * 2] = m_hi;
                 ml[(warp * 16 + g + 8) * 2 + 1] = l_hi;
             }
+        }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (ok && tid < D) {
