@@ -329,6 +329,8 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     if (warp == 4) {
         // ---------------------------------------------------------------- producer
+        // the cache is read once: its lines go first when L2 needs room (q and the partial results stay)
+        const uint64_t stream_policy = l2_policy_evict_first();
         // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
         // the table read is not on the path that refills a freed slot
         const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
@@ -359,10 +361,10 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 __syncwarp();
                 if (lane < live) {
                     const uint32_t offs = (uint32_t)(lane * ps) * 128u;
-                    tma_load_4d(sK + st * kTileB + offs, &tm_k, bk, 0, hk, 0, cur);
-                    if (D == 128) tma_load_4d(sK + st * kTileB + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur);
-                    tma_load_4d(sV + st * kTileB + offs, &tm_v, bv, 0, hk, 0, cur);
-                    if (D == 128) tma_load_4d(sV + st * kTileB + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur);
+                    tma_load_4d_hint(sK + st * kTileB + offs, &tm_k, bk, 0, hk, 0, cur, stream_policy);
+                    if (D == 128) tma_load_4d_hint(sK + st * kTileB + kDecHalfBytes + offs, &tm_k, bk, 64, hk, 0, cur, stream_policy);
+                    tma_load_4d_hint(sV + st * kTileB + offs, &tm_v, bv, 0, hk, 0, cur, stream_policy);
+                    if (D == 128) tma_load_4d_hint(sV + st * kTileB + kDecHalfBytes + offs, &tm_v, bv, 64, hk, 0, cur, stream_policy);
                 }
             }
         } else if (lane == 0) {
@@ -379,11 +381,11 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 }
                 if (!mbar_wait(smem_u32(&bars[2 * kStages + st]), ((t / kStages) & 1) ^ 1, &abort_flag, 22)) break;
                 mbar_expect_tx(bk, kTileB);
-                tma_load_4d(sK + st * kTileB, &tm_k, bk, 0, hk, row0, slab);
-                if (D == 128) tma_load_4d(sK + st * kTileB + kDecHalfBytes, &tm_k, bk, 64, hk, row0, slab);
+                tma_load_4d_hint(sK + st * kTileB, &tm_k, bk, 0, hk, row0, slab, stream_policy);
+                if (D == 128) tma_load_4d_hint(sK + st * kTileB + kDecHalfBytes, &tm_k, bk, 64, hk, row0, slab, stream_policy);
                 mbar_expect_tx(bv, kTileB);
-                tma_load_4d(sV + st * kTileB, &tm_v, bv, 0, hk, row0, slab);
-                if (D == 128) tma_load_4d(sV + st * kTileB + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab);
+                tma_load_4d_hint(sV + st * kTileB, &tm_v, bv, 0, hk, row0, slab, stream_policy);
+                if (D == 128) tma_load_4d_hint(sV + st * kTileB + kDecHalfBytes, &tm_v, bv, 64, hk, row0, slab, stream_policy);
             }
         }
         __syncwarp();

@@ -84,6 +84,8 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     if (warp == kDec8Warps) {
         // ---------------------------------------------------------------- producer
+        // the cache is read once: its lines go first when L2 needs room (q and the partial results stay)
+        const uint64_t stream_policy = l2_policy_evict_first();
         // paged cache: the page of a tile is looked up one tile ahead of its loads, so that
         // the table read is not on the path that refills a freed slot
         const int* table = p.block_table ? p.block_table + (long long)b * p.table_stride : nullptr;
@@ -114,8 +116,8 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 __syncwarp();
                 if (lane < live) {
                     const uint32_t offs = (uint32_t)(lane * ps) * 128u;
-                    tma_load_4d(sK + st * kDec8TileBytes + offs, &tm_k, bk, 0, hk, 0, cur);
-                    tma_load_4d(sV + st * kDec8TileBytes + offs, &tm_v, bv, 0, hk, 0, cur);
+                    tma_load_4d_hint(sK + st * kDec8TileBytes + offs, &tm_k, bk, 0, hk, 0, cur, stream_policy);
+                    tma_load_4d_hint(sV + st * kDec8TileBytes + offs, &tm_v, bv, 0, hk, 0, cur, stream_policy);
                 }
             }
         } else if (lane == 0) {
@@ -132,9 +134,9 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
                 }
                 if (!mbar_wait(smem_u32(&bars[2 * kDec8Stages + st]), ((t / kDec8Stages) & 1) ^ 1, &abort_flag, 22)) break;
                 mbar_expect_tx(bk, kDec8TileBytes);
-                tma_load_4d(sK + st * kDec8TileBytes, &tm_k, bk, 0, hk, row0, slab);
+                tma_load_4d_hint(sK + st * kDec8TileBytes, &tm_k, bk, 0, hk, row0, slab, stream_policy);
                 mbar_expect_tx(bv, kDec8TileBytes);
-                tma_load_4d(sV + st * kDec8TileBytes, &tm_v, bv, 0, hk, row0, slab);
+                tma_load_4d_hint(sV + st * kDec8TileBytes, &tm_v, bv, 0, hk, row0, slab, stream_policy);
             }
         }
         __syncwarp();
