@@ -94,20 +94,24 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// The consumer warps' work in the keys-as-rows form (one query token, at most 8 query heads per
-// kv head).  A warp-level MMA has 16 rows and 8 columns: with the query heads as rows, as in the
+// The consumer warps' work in the keys-as-rows form (at most 8 rows, i.e. (token, head) pairs,
+// per kv head).  A warp-level MMA has 16 rows and 8 columns: with the query heads as rows, as in the
 // general form below, a kv head with 1 to 8 query heads leaves half or more of every MMA to
 // padding.  Here the KEYS are the rows: S^T = K q^T (A = 16 keys x 16 elements of K by plain
 // ldmatrix, B = q^T, the 8 columns are the heads), and O^T += V^T P^T (A = 16 output columns x 16
 // keys of V by transposing ldmatrix, B = P^T, which is the accumulator layout of S^T transposed
 // 8 x 8 with movmatrix).  A tile then takes half the MMAs, a thread holds half the scores and
 // half the accumulators, and the row maxima and sums run over the lanes that share a column.
+// q_col: the query row that is this thread's column g of q^T (nullptr: padding).  kMulti: hide0,
+// hide1 say how many of the sequence's last keys the rows in this thread's accumulator columns
+// 2 t4, 2 t4 + 1 must not see (they came after the row's token).
 // Leaves each warp's (max, sum, O) in mo / ml in the layout the merge expects; returns false
 // after a wait that gave up.
-template <typename T, int D>
+template <bool kMulti, typename T, int D>
 __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint64_t* bars, volatile uint32_t* abort_flag,
                                                      uint32_t sK, uint32_t sV, float* mo, float* ml, int warp, int lane,
-                                                     const T* q_rows, int G, int k_begin, int k_end, int n_tiles) {
+                                                     const T* q_col, int hide0, int hide1, int len, int k_begin, int k_end,
+                                                     int n_tiles) {
     constexpr int kStages = DecShape<D>::kStages, kTileB = DecShape<D>::kTileBytes;
     constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
     const int g = lane >> 2, t4 = lane & 3;
@@ -116,8 +120,8 @@ __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
         const int d0 = ks * 16 + 2 * t4;
-        qb[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_rows + g * D + d0) : 0u;
-        qb[ks][1] = (g < G) ? *reinterpret_cast<const uint32_t*>(q_rows + g * D + d0 + 8) : 0u;
+        qb[ks][0] = q_col ? *reinterpret_cast<const uint32_t*>(q_col + d0) : 0u;
+        qb[ks][1] = q_col ? *reinterpret_cast<const uint32_t*>(q_col + d0 + 8) : 0u;
     }
     // O^T: block i holds output columns 16 i + g (values 0, 1) and 16 i + 8 + g (values 2, 3) of heads 2 t4, 2 t4 + 1
     float o[D / 16][4];
@@ -155,12 +159,18 @@ __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint
                 }
             }
             // ---- mask, running max, probabilities
+            // keys of this warp's 32 that a row may see: all valid ones, minus (several query
+            // rows) those among the sequence's last that came after the row's token
+            const int seen0 = kMulti ? min(valid, len - hide0 - (k_begin + t * kDecTile) - key_w) : valid;
+            const int seen1 = kMulti ? min(valid, len - hide1 - (k_begin + t * kDecTile) - key_w) : valid;
             float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
                 const int k_lo = mb * 16 + g;
-                if (k_lo >= valid) sc[mb][0] = sc[mb][1] = -INFINITY;
-                if (k_lo + 8 >= valid) sc[mb][2] = sc[mb][3] = -INFINITY;
+                if (k_lo >= seen0) sc[mb][0] = -INFINITY;
+                if (k_lo >= seen1) sc[mb][1] = -INFINITY;
+                if (k_lo + 8 >= seen0) sc[mb][2] = -INFINITY;
+                if (k_lo + 8 >= seen1) sc[mb][3] = -INFINITY;
                 mx0 = fmaxf(mx0, fmaxf(sc[mb][0], sc[mb][2]));
                 mx1 = fmaxf(mx1, fmaxf(sc[mb][1], sc[mb][3]));
             }
@@ -169,21 +179,24 @@ __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint
                 mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
                 mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
             }
-            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);  // finite: key 0 of the warp is valid
+            // finite when key 0 of the warp is visible (always with one query token; an earlier
+            // token of several may see none of the warp's keys: its state then stays empty)
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
             const float a0 = (m_run[0] == -INFINITY) ? 0.f : fast_exp2((m_run[0] - mn0) * p.scale_log2);
             const float a1 = (m_run[1] == -INFINITY) ? 0.f : fast_exp2((m_run[1] - mn1) * p.scale_log2);
             m_run[0] = mn0;
             m_run[1] = mn1;
-            const float nm0 = -mn0 * p.scale_log2, nm1 = -mn1 * p.scale_log2;
+            const float nm0 = (kMulti && mn0 == -INFINITY) ? 0.f : -mn0 * p.scale_log2;
+            const float nm1 = (kMulti && mn1 == -INFINITY) ? 0.f : -mn1 * p.scale_log2;
             float s0 = 0.f, s1 = 0.f;
 #pragma unroll
             for (int mb = 0; mb < 2; ++mb) {
                 const int k_lo = mb * 16 + g;
                 float* e = sc[mb];
-                e[0] = (k_lo < valid) ? fast_exp2(fmaf(e[0], p.scale_log2, nm0)) : 0.f;
-                e[1] = (k_lo < valid) ? fast_exp2(fmaf(e[1], p.scale_log2, nm1)) : 0.f;
-                e[2] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[2], p.scale_log2, nm0)) : 0.f;
-                e[3] = (k_lo + 8 < valid) ? fast_exp2(fmaf(e[3], p.scale_log2, nm1)) : 0.f;
+                e[0] = (k_lo < seen0) ? fast_exp2(fmaf(e[0], p.scale_log2, nm0)) : 0.f;
+                e[1] = (k_lo < seen1) ? fast_exp2(fmaf(e[1], p.scale_log2, nm1)) : 0.f;
+                e[2] = (k_lo + 8 < seen0) ? fast_exp2(fmaf(e[2], p.scale_log2, nm0)) : 0.f;
+                e[3] = (k_lo + 8 < seen1) ? fast_exp2(fmaf(e[3], p.scale_log2, nm1)) : 0.f;
                 s0 += e[0] + e[2];
                 s1 += e[1] + e[3];
                 // (key g | heads 2 t4, 2 t4 + 1) -> transposed: (head g | keys 2 t4, 2 t4 + 1), the B fragment
@@ -266,13 +279,12 @@ __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint
 // grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
 // T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
 // D: the head dimension, 128 or 64.
-// kKeyRows (one query token, at most 8 query heads per kv head): the consumers work in the
-// keys-as-rows form (dec_consume_key_rows).
+// kKeyRows (at most 8 (token, head) rows per kv head): the consumers work in the keys-as-rows
+// form (dec_consume_key_rows).
 template <bool kMulti, typename T = __half, int D = 128, bool kKeyRows = false>
 __global__ void __launch_bounds__(kDecMmaThreads, DecShape<D>::kCtasPerSm)
 fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                            const DecodeParams p) {
-    static_assert(!(kKeyRows && kMulti), "keys as rows: one query token");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr int kStages = DecShape<D>::kStages, kTileB = DecShape<D>::kTileBytes;
@@ -396,8 +408,12 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
         float* ml = mo + 4 * 16 * D;                                                         // [4][16][2]: m, l
         bool ok = true;
         if constexpr (kKeyRows) {
-            ok = dec_consume_key_rows<T, D>(p, bars, &abort_flag, sK, sV, mo, ml, warp, lane,
-                                            static_cast<const T*>(p.q) + row_index(0) * D, G, k_begin, k_end, n_tiles);
+            // column g of q^T is row g of the CTA; accumulator columns 2 t4, 2 t4 + 1 are rows 2 t4, 2 t4 + 1
+            const T* q_col = (g < G) ? static_cast<const T*>(p.q) + row_index(g) * D : nullptr;
+            const int hide0 = kMulti ? Sq - 1 - row_token(min(2 * t4, G - 1)) : 0;
+            const int hide1 = kMulti ? Sq - 1 - row_token(min(2 * t4 + 1, G - 1)) : 0;
+            ok = dec_consume_key_rows<kMulti, T, D>(p, bars, &abort_flag, sK, sV, mo, ml, warp, lane, q_col, hide0, hide1,
+                                                    len, k_begin, k_end, n_tiles);
         } else {
         // Q as A fragments for the D / 16 k-steps (rows >= G are zero)
         uint32_t qa[D / 16][4];

@@ -723,12 +723,14 @@ int decode_launch(const CUtensorMap& tk, const CUtensorMap& tv, const fa::Decode
     if (have_keys) {
         constexpr int smem = fa::DecShape<D>::kSmem;
         int sm_count = 0;
-        // one query token and at most 8 query heads per kv head: the keys-as-rows form of the consumers
-        const bool key_rows = Sq == 1 && g <= 8;
-        auto kern = bf16 ? ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __nv_bfloat16, D>
+        // at most 8 (token, head) rows per kv head: the keys-as-rows form of the consumers
+        const bool key_rows = g * Sq <= 8;
+        auto kern = bf16 ? ((Sq > 1) ? (key_rows ? fa::fa_decode_split_mma_kernel<true, __nv_bfloat16, D, true>
+                                                 : fa::fa_decode_split_mma_kernel<true, __nv_bfloat16, D>)
                                      : (key_rows ? fa::fa_decode_split_mma_kernel<false, __nv_bfloat16, D, true>
                                                  : fa::fa_decode_split_mma_kernel<false, __nv_bfloat16, D>))
-                         : ((Sq > 1) ? fa::fa_decode_split_mma_kernel<true, __half, D>
+                         : ((Sq > 1) ? (key_rows ? fa::fa_decode_split_mma_kernel<true, __half, D, true>
+                                                 : fa::fa_decode_split_mma_kernel<true, __half, D>)
                                      : (key_rows ? fa::fa_decode_split_mma_kernel<false, __half, D, true>
                                                  : fa::fa_decode_split_mma_kernel<false, __half, D>));
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))

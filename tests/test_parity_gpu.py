@@ -885,8 +885,10 @@ def run_decode_append(fa, q, k, v, seqlens_dev, scale):
     return o, lse
 
 
-@pytest.mark.parametrize("sq,hq,hkv", [(2, 4, 4), (4, 8, 2), (5, 8, 1), (8, 8, 8), (16, 4, 1), (17, 6, 2), (3, 40, 2), (64, 2, 1)])
+@pytest.mark.parametrize("sq,hq,hkv", [(2, 4, 4), (4, 8, 2), (5, 8, 1), (8, 8, 8), (16, 4, 1), (17, 6, 2), (3, 40, 2), (64, 2, 1),
+                                       (2, 8, 2), (3, 4, 2), (7, 3, 3)])
 def test_decode_append_small_full(fa, sq, hq, hkv):
+    # (up to 8 (token, head) rows per kv head take the keys-as-rows consumers, more the heads-as-rows ones)
     # sq query rows = the last sq positions of each cache; lengths: long, exactly sq, shorter than
     # sq (its first queries see nothing), sq + 1, around a tile and a chunk boundary; NaN past the end
     cfg = synth.DecodeConfig("t", 7, hq, hkv, 3000, 1, 3000, seed=sq * 53 + hq + hkv)
