@@ -816,8 +816,9 @@ def run_decode(fa, q, k, v, seqlens_dev, scale):
     return o, lse
 
 
-@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (8, 2), (8, 1), (6, 2), (16, 1), (17, 1), (40, 2)])
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (8, 4), (8, 2), (8, 1), (6, 2), (16, 1), (17, 1), (40, 2), (7, 1), (10, 2), (9, 1)])
 def test_decode_small_full(fa, hq, hkv):
+    # (1 to 8 query heads per kv head take the keys-as-rows consumers, 9 and more the heads-as-rows ones)
     cfg = synth.DecodeConfig("t", 5, hq, hkv, 1500, 1, 1500, seed=hq * 31 + hkv)
     q, k, v, sl = synth.decode_inputs(cfg, "cpu", poison=True)
     sl[0], sl[1], sl[2] = 1500, 0, 1          # full, empty, single key
