@@ -628,6 +628,9 @@ fa_decode_combine_kernel(const DecodeParams p, T* o, float* lse) {
     int len = p.seqlens[b];
     len = max(0, min(len, p.Smax));
     const int nc = (len + p.chunk - 1) / p.chunk;
+    // launched as a programmatic dependent of the split kernel: its partial results are
+    // complete and visible from here on (returns at once in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const float* lp = p.lse_part + (long long)bh * p.n_chunks;
     const float* op = p.o_part + (long long)bh * p.n_chunks * D;
     float M = -INFINITY;

@@ -720,6 +720,25 @@ int decode_check_args(const void* q, const void* k_cache, const void* v_cache, c
     return FA_OK;
 }
 
+// Launch of the merge kernel as a programmatic dependent of the split kernel before it in the
+// stream: its launch is processed while the split kernel still runs, and its blocks start (they
+// wait in griddepcontrol.wait) when the last block of the split kernel has finished and its
+// writes are visible.
+template <typename T, int D>
+cudaError_t launch_combine(const fa::DecodeParams& dp, int blocks, void* o, float* lse, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(D);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fa::fa_decode_combine_kernel<T, D>, dp, static_cast<T*>(o), lse);
+}
+
 // Launch of the split kernel and of the merge for one head dimension.
 template <int D>
 int decode_launch(const CUtensorMap& tk, const CUtensorMap& tv, const fa::DecodeParams& dp, void* o, float* lse, int g,
@@ -746,9 +765,9 @@ int decode_launch(const CUtensorMap& tk, const CUtensorMap& tv, const fa::Decode
         if (e != cudaSuccess) return cuda_fail(e);
     }
     if (direct) return FA_OK;
-    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16, D><<<B * Sq * Hq, D, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
-    else fa::fa_decode_combine_kernel<__half, D><<<B * Sq * Hq, D, 0, st>>>(dp, static_cast<__half*>(o), lse);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = bf16 ? launch_combine<__nv_bfloat16, D>(dp, B * Sq * Hq, o, lse, st)
+                         : launch_combine<__half, D>(dp, B * Sq * Hq, o, lse, st);
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
@@ -879,9 +898,9 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
         if (rc) return rc;
     }
     if (direct) return FA_OK;
-    if (bf16) fa::fa_decode_combine_kernel<__nv_bfloat16><<<B * Hq, 128, 0, st>>>(dp, static_cast<__nv_bfloat16*>(o), lse);
-    else fa::fa_decode_combine_kernel<__half><<<B * Hq, 128, 0, st>>>(dp, static_cast<__half*>(o), lse);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = bf16 ? launch_combine<__nv_bfloat16, 128>(dp, B * Hq, o, lse, st)
+                         : launch_combine<__half, 128>(dp, B * Hq, o, lse, st);
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? FA_OK : cuda_fail(e);
 }
 
