@@ -190,6 +190,8 @@ int fa_forward_varlen(const void* q, const void* k, const void* v, void* o, floa
  *   d is 128 or 64 (FA_ERR_UNSUPPORTED otherwise; fa_decode_workspace_bytes then returns 0); the
  *   same holds for fa_decode_paged, fa_decode_append, fa_decode_ex and fa_decode_noalloc, which
  *   run the same kernel.  The 8-bit cache forms (fa_decode_fp8...) take d = 128 only.
+ *   Skv_max may not exceed 65535 chunks of the cache split (chunks are 256 to 4096 keys long, so
+ *   16 million keys always fit; FA_ERR_UNSUPPORTED beyond).
  */
 int fa_decode(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
               const int* seqlens_k, int B, int Hq, int Hkv, int Skv_max, int d, float scale,

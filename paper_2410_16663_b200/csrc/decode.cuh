@@ -276,7 +276,10 @@ __device__ __forceinline__ bool dec_consume_key_rows(const DecodeParams& p, uint
 // several tokens were appended, Appendix C with more than one new token): the 16 MMA rows of a
 // CTA are then (token, head) pairs of one kv head, and query token t sees the keys up to
 // position len - Sq + t.  q is [B,Sq,Hq,d], the partials [B,Sq,Hq,NC,...].
-// grid: (n_chunks, Hkv * ceil(Sq * g / 16), B) with g = Hq / Hkv
+// grid: (Hkv * ceil(Sq * g / 16), n_chunks, B) with g = Hq / Hkv.  The kv head is the fastest
+// index: CTAs that run at the same time then read the same keys' rows of neighbouring heads,
+// which are contiguous in the cache (a key's Hkv * D elements), instead of key ranges whole
+// chunks apart (64 sequences of 1K to 32K keys, 32 kv heads: 2.39 against 2.48 ms).
 // T: the 16-bit type of q, the cache and the probabilities (__half or __nv_bfloat16).
 // D: the head dimension, 128 or 64.
 // kKeyRows (at most 8 (token, head) rows per kv head): the consumers work in the keys-as-rows
@@ -295,14 +298,14 @@ fa_decode_split_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int c = blockIdx.x;
+    const int c = blockIdx.y;
     const int b = blockIdx.z;
     const int g_all = p.Hq / p.Hkv;
     const int Sq = kMulti ? p.Sq : 1;
     const int rows_all = g_all * Sq;               // (token, head) rows that share a kv head
     const int n_sub = (rows_all + 15) / 16;        // CTAs per kv head when there are more than 16
-    const int hk = blockIdx.y / n_sub;
-    const int sub = blockIdx.y % n_sub;
+    const int hk = blockIdx.x / n_sub;
+    const int sub = blockIdx.x % n_sub;
     const int G = min(16, rows_all - sub * 16);    // rows of this CTA
     // row r of the CTA: token and head, and its row in q and in the partial results
     auto row_token = [&](int r) { return kMulti ? (sub * 16 + r) / g_all : 0; };

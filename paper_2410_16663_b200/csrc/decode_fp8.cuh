@@ -35,7 +35,7 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-// grid: (n_chunks, Hkv * ceil(g / 16), B) with g = Hq / Hkv
+// grid: (Hkv * ceil(g / 16), n_chunks, B) with g = Hq / Hkv (the kv head fastest, see decode.cuh)
 template <int NB>
 __global__ void __launch_bounds__(kDec8Threads, 2)
 fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -49,12 +49,12 @@ fa_decode_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __gri
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const int c = blockIdx.x;
+    const int c = blockIdx.y;
     const int b = blockIdx.z;
     const int g_all = p.Hq / p.Hkv;
     const int n_sub = (g_all + 15) / 16;           // CTAs per kv head when more than 16 heads share it
-    const int hk = blockIdx.y / n_sub;
-    const int sub = blockIdx.y % n_sub;
+    const int hk = blockIdx.x / n_sub;
+    const int sub = blockIdx.x % n_sub;
     const int h0 = hk * g_all + sub * 16;          // first query head of this CTA
     const int G = min(16, g_all - sub * 16);       // its number of query heads
 

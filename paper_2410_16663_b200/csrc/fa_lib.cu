@@ -759,7 +759,7 @@ int decode_launch(const CUtensorMap& tk, const CUtensorMap& tv, const fa::Decode
                                                  : fa::fa_decode_split_mma_kernel<false, __half, D>));
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
-        dim3 grid(dp.n_chunks, Hkv * ((g * Sq + 15) / 16), B);   // 16 (token, head) rows per CTA
+        dim3 grid(Hkv * ((g * Sq + 15) / 16), dp.n_chunks, B);   // 16 (token, head) rows per CTA
         kern<<<grid, fa::kDecMmaThreads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e);
@@ -794,6 +794,7 @@ int decode_impl(const void* q, const void* k_cache, const void* v_cache, void* o
     dp.Sq = Sq;
     dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max, true) : 256;
     dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
+    if (dp.n_chunks > 65535) return FA_ERR_UNSUPPORTED;   // the chunks are the grid's second dimension
     dp.o_part = static_cast<float*>(workspace);
     dp.lse_part = dp.o_part + (size_t)B * Sq * Hq * dp.n_chunks * d;
     dp.scale_log2 = scale * 1.4426950408889634f;
@@ -862,6 +863,7 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
     dp.B = B; dp.Hq = Hq; dp.Hkv = Hkv; dp.Smax = Skv_max;
     dp.chunk = Skv_max > 0 ? decode_chunk(B, Hkv, Skv_max) : 256;
     dp.n_chunks = Skv_max > 0 ? (Skv_max + dp.chunk - 1) / dp.chunk : 1;
+    if (dp.n_chunks > 65535) return FA_ERR_UNSUPPORTED;   // the chunks are the grid's second dimension
     dp.o_part = static_cast<float*>(workspace);
     dp.lse_part = dp.o_part + (size_t)B * Hq * dp.n_chunks * 128;
     dp.scale_log2 = scale * k_scale * 1.4426950408889634f;   // the scores are q . (k_scale * k8)
@@ -891,7 +893,7 @@ static int decode_fp8_impl(const void* q, const void* k_cache, const void* v_cac
         auto kern = (g > 8) ? fa::fa_decode_split_fp8_kernel<2> : fa::fa_decode_split_fp8_kernel<1>;
         if (int ce = fa::prepare_big_smem_kernel(reinterpret_cast<const void*>(kern), smem, &sm_count))
             return cuda_fail(static_cast<cudaError_t>(ce));
-        dim3 grid(dp.n_chunks, Hkv * ((g + 15) / 16), B);
+        dim3 grid(Hkv * ((g + 15) / 16), dp.n_chunks, B);
         kern<<<grid, fa::kDec8Threads, smem, st>>>(tk, tv, dp);
         cudaError_t e = cudaGetLastError();
         rc = e == cudaSuccess ? FA_OK : cuda_fail(e);
